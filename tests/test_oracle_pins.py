@@ -1,0 +1,441 @@
+"""Pins for the CPU oracle: each test ties a part of it to something other than itself --
+values the paper prints, closed forms, brute force, a separately written restatement,
+a library routine on the special case it covers, finite differences.  CPU only."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_15105_b200.workloads import (HgaConfig, bf16_bits_to_f64, f32_to_bf16_bits,
+                                              make_inputs)
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def tiny(**kw):
+    base = dict(name="tiny", batch=1, n_q_heads=2, n_kv_heads=1, head_dim=16, total_len=128,
+                seg_len=64, chunk=8, group=2, q_block=8, topk_chunks=3, topk_groups=2, sink=8,
+                local=16, topics=4, needles=0, backward=True, seed=7)
+    base.update(kw)
+    return HgaConfig(**base)
+
+
+def read_table(name):
+    rows = []
+    for line in open(os.path.join(GOLDEN, name)):
+        line = line.strip()
+        if line and not line.startswith("#"):
+            rows.append([float(x) for x in line.split()])
+    return rows
+
+
+# ---------------------------------------------------------------- rounding (P1)
+
+def test_bf16_rounding_matches_library_conversion():
+    # torch's float64 -> bfloat16 conversion is an independent round-to-nearest-even
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.standard_normal(4000), rng.standard_normal(2000) * 1e-3,
+                        rng.standard_normal(2000) * 1e4, [0.0, -0.0, 1.0, -1.0, 3.0e38, 1e-40, 5e-41]])
+    x = x.astype(np.float32).astype(np.float64)   # exactly representable in fp32: no double rounding in torch
+    want = torch.from_numpy(x).to(torch.float32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    got = np.array([oracle.f64_to_bf16(v) for v in x], np.uint16)
+    assert np.array_equal(got, want)
+
+
+def test_bf16_rounding_ties_and_single_rounding():
+    # 1 + 2^-8 is exactly half way between bf16 neighbours 1.0 (even) and 1 + 2^-7
+    assert oracle.f64_to_bf16(1.0 + 2.0 ** -8) == 0x3F80
+    assert oracle.f64_to_bf16(1.0 + 2.0 ** -7 + 2.0 ** -8) == 0x3F82   # tie -> even (up)
+    # just above the tie by less than fp32 resolution: a detour through fp32 would round
+    # to the tie first and then to even (down); direct rounding goes up
+    assert oracle.f64_to_bf16(1.0 + 2.0 ** -8 + 2.0 ** -40) == 0x3F81
+    assert oracle.f64_to_bf16(-(1.0 + 2.0 ** -8 + 2.0 ** -40)) == 0xBF81
+    assert oracle.f64_to_bf16(2.0 - 2.0 ** -9) == 0x4000              # mantissa carry into exponent
+
+
+# ---------------------------------------------------------------- summaries (P1)
+
+def test_summaries_constant_chunks_and_mean():
+    cfg = tiny()
+    rng = np.random.default_rng(1)
+    L, d, c, g = cfg.total_len, cfg.head_dim, cfg.chunk, cfg.group
+    # constant keys inside each chunk: every summary of that chunk is that constant
+    const = f32_to_bf16_bits(rng.standard_normal((L // c, d)).astype(np.float32))
+    K = np.repeat(const, c, axis=0)[None, None]
+    cs, gs = oracle.build_summaries(cfg, np.ascontiguousarray(K))
+    assert np.array_equal(cs[0, 0], const)
+    assert np.array_equal(gs[0, 0], np.repeat(const, c // g, axis=0))
+    # random keys: numpy's float64 mean then torch's rounding (independent of the oracle)
+    Kb = f32_to_bf16_bits(rng.standard_normal((1, 1, L, d)).astype(np.float32))
+    cs, gs = oracle.build_summaries(cfg, Kb)
+    kf = bf16_bits_to_f64(Kb)[0, 0]
+    for summ, width in ((cs, c), (gs, g)):
+        mean = kf.reshape(L // width, width, d).mean(axis=1)
+        assert np.all(mean.astype(np.float32).astype(np.float64) == mean)   # exact in fp32 here
+        want = torch.from_numpy(mean).to(torch.float32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        assert np.array_equal(summ[0, 0], want)
+
+
+def test_summaries_partial_range_leaves_rest_untouched():
+    cfg = tiny()
+    K = make_inputs(cfg)["K"]
+    full_c, full_g = oracle.build_summaries(cfg, K)
+    cs = np.full_like(full_c, 0xABCD)
+    gs = np.full_like(full_g, 0xABCD)
+    oracle.build_summaries(cfg, K, 64, 128, cs, gs)
+    assert np.array_equal(cs[:, :, 8:], full_c[:, :, 8:]) and np.all(cs[:, :, :8] == 0xABCD)
+    assert np.array_equal(gs[:, :, 32:], full_g[:, :, 32:]) and np.all(gs[:, :, :32] == 0xABCD)
+
+
+# ---------------------------------------------------------------- window geometry (P2)
+
+def _attended_pairs(cfg, group_idx, n_groups):
+    """Count (query position, key) pairs from the oracle's routed token lists."""
+    H, Bq = cfg.history, cfg.q_block
+    pairs = 0
+    for qb in range(cfg.n_q_blocks):
+        tok = oracle.routed_tokens(cfg, qb, group_idx[qb, :n_groups[qb]])
+        assert np.all(np.diff(tok) > 0)
+        pos = H + qb * Bq + np.arange(Bq)
+        pairs += int((tok[None, :] <= pos[:, None]).sum())
+    return pairs
+
+
+@pytest.mark.parametrize("row", read_table("table1_selection_density.txt"))
+def test_selection_density_reproduces_table1(row):
+    # Table 1: one segment, chunk 64, 8 routed chunks opened completely, sink 64, local 128.
+    L, printed = int(row[0]), row[1]
+    cfg = HgaConfig("t1", 1, 1, 1, 8, L, L, 64, 8, 64, 8, 8, 64, 128, topics=0, needles=0,
+                    backward=False, seed=3)
+    x = make_inputs(cfg, with_dO=False)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    r = oracle.route(cfg, x["Q"], cs, gs)
+    pairs = _attended_pairs(cfg, r["group_idx"][0, 0], r["n_groups"][0, 0])
+    density = 100.0 * pairs / (L * (L + 1) / 2)
+    assert abs(density - printed) <= 0.45, (L, density, printed)
+
+
+def test_tokens_per_second_definition_table2():
+    for tokens, total_ms, printed in read_table("table2_tokens_per_second.txt"):
+        assert abs(tokens / (total_ms * 1e-3) - printed) < 0.01
+
+
+def test_window_geometry_cases():
+    cfg = HgaConfig("w", 1, 1, 1, 8, 1024, 512, 64, 8, 64, 4, 4, 64, 128, 0, 0, False, 0)
+    assert oracle.window(cfg, 0) == (512 - 128, 64)          # p0 = 512
+    assert oracle.window(cfg, 7) == (960 - 128, 64)
+    one = cfg.scaled(total_len=512, seg_len=512)
+    assert oracle.window(one, 0) == (0, 0)                     # nothing before the block
+    assert oracle.window(one, 1) == (0, 0)                     # local window reaches position 0
+    assert oracle.window(one, 2) == (0, 0)
+    assert oracle.window(one, 3) == (64, 64)                   # sink exactly fills the gap
+    assert oracle.window(one, 4) == (128, 64)                  # first block with a candidate
+    big = cfg.scaled(q_block=128, total_len=1024, seg_len=512)
+    assert oracle.window(big, 1) == (512 + 128 - 128, 64)
+
+
+# ---------------------------------------------------------------- top-k (P3, P7)
+
+def _scores_from_definition(cfg, Q, summ, qb, ids):
+    """max over the block's rows of the raw dot product, straight from the definition."""
+    G, Bq = cfg.gqa, cfg.q_block
+    rows = bf16_bits_to_f64(Q[0, :G, qb * Bq:(qb + 1) * Bq]).reshape(G * Bq, -1)
+    return np.array([max(float(np.dot(r, bf16_bits_to_f64(summ[0, 0, j]))) for r in rows) for j in ids])
+
+
+def test_topk_brute_force_with_ties():
+    cfg = tiny(total_len=128, seg_len=32, topk_chunks=3, topk_groups=2)
+    x = make_inputs(cfg)
+    K = x["K"].copy()
+    c = cfg.chunk
+    # duplicate chunks (identical keys => identical scores): 3 copies of chunk 2, 2 of chunk 5
+    for dst, src in ((4, 2), (9, 2), (7, 5)):
+        K[0, 0, dst * c:(dst + 1) * c] = K[0, 0, src * c:(src + 1) * c]
+    # and duplicate groups inside chunk 2 (hence inside its copies)
+    g = cfg.group
+    K[0, 0, 2 * c + 2 * g:2 * c + 3 * g] = K[0, 0, 2 * c:2 * c + g]
+    for dst in (4, 9):
+        K[0, 0, dst * c:(dst + 1) * c] = K[0, 0, 2 * c:3 * c]
+    cs, gs = oracle.build_summaries(cfg, K)
+    r = oracle.route(cfg, x["Q"], cs, gs, want_scores=True)
+    per = c // g
+    saw_tie = False
+    for qb in range(cfg.n_q_blocks):
+        ls, se = oracle.window(cfg, qb)
+        cand = list(range(se // c, ls // c))
+        sc = _scores_from_definition(cfg, x["Q"], cs, qb, cand)
+        assert np.allclose(r["chunk_scores"][0, 0, qb, cand], sc, rtol=0, atol=1e-12)
+        k = min(cfg.topk_chunks, len(cand))
+        best = max(itertools.combinations(range(len(cand)), k),
+                   key=lambda s: (sum(sc[i] for i in s), [-i for i in s]))   # max sum, then lowest ids
+        # a k-subset maximises the sum iff it is a top-k set; among equal sums the tuple
+        # comparison on negated ids picks the lexicographically smallest
+        got = [j for j in r["chunk_idx"][0, 0, qb] if j >= 0]
+        assert got == [cand[i] for i in best], (qb, got)
+        saw_tie |= len(set(np.round(sc, 12))) < len(sc)
+        n = 0
+        for j in got:
+            ids = list(range(j * per, (j + 1) * per))
+            sg = _scores_from_definition(cfg, x["Q"], gs, qb, ids)
+            bestg = max(itertools.combinations(range(per), cfg.topk_groups),
+                        key=lambda s: (sum(sg[i] for i in s), [-i for i in s]))
+            want = [ids[i] for i in bestg]
+            assert list(r["group_idx"][0, 0, qb, n:n + len(want)]) == want
+            n += len(want)
+        assert r["n_groups"][0, 0, qb] == n
+        assert np.all(r["group_idx"][0, 0, qb, n:] == -1)
+    assert saw_tie
+
+
+def test_router_structure_and_permutation():
+    cfg = tiny(n_q_heads=4, n_kv_heads=2, total_len=256, seg_len=64, topk_chunks=4)
+    x = make_inputs(cfg)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    r = oracle.route(cfg, x["Q"], cs, gs)
+    c, g, per, kge = cfg.chunk, cfg.group, cfg.chunk // cfg.group, cfg.kg_eff
+    for h in range(2):
+        for qb in range(cfg.n_q_blocks):
+            ls, se = oracle.window(cfg, qb)
+            n_cand = (ls - se) // c
+            ci = r["chunk_idx"][0, h, qb]
+            sel = ci[ci >= 0]
+            assert len(sel) == min(cfg.topk_chunks, n_cand)
+            assert np.all(np.diff(sel) > 0) and np.all(ci[len(sel):] == -1)
+            assert np.all((sel >= se // c) & (sel < ls // c))
+            gi = r["group_idx"][0, h, qb]
+            ng = r["n_groups"][0, h, qb]
+            assert ng == len(sel) * kge and np.all(np.diff(gi[:ng]) > 0)
+            assert np.array_equal(np.unique(gi[:ng] // per), sel)
+            assert np.all(np.bincount(gi[:ng] // per, minlength=cfg.total_len // c)[sel] == kge)
+    # moving the contents of two candidate chunks moves the selection with them
+    # (history chunks 3 and 11 are candidates of every block; ties have probability zero here)
+    K2 = x["K"].copy()
+    a, b = 3, 11
+    K2[:, :, a * c:(a + 1) * c], K2[:, :, b * c:(b + 1) * c] = \
+        x["K"][:, :, b * c:(b + 1) * c], x["K"][:, :, a * c:(a + 1) * c]
+    cs2, gs2 = oracle.build_summaries(cfg, K2)
+    r2 = oracle.route(cfg, x["Q"], cs2, gs2)
+    swap = {a: b, b: a}
+    for h in range(2):
+        for qb in range(cfg.n_q_blocks):
+            s1 = {swap.get(int(j), int(j)) for j in r["chunk_idx"][0, h, qb] if j >= 0}
+            s2 = {int(j) for j in r2["chunk_idx"][0, h, qb] if j >= 0}
+            assert s1 == s2
+
+
+# ---------------------------------------------------------------- attention (P4, P5, P9)
+
+def _mask_from_definition(cfg, h, group_idx, n_groups):
+    """S x L boolean mask written from the definition of the routed set, per query position."""
+    H, S, L, Bq, c, g = cfg.history, cfg.seg_len, cfg.total_len, cfg.q_block, cfg.chunk, cfg.group
+    mask = np.zeros((S, L), bool)
+    for t in range(S):
+        pos = H + t
+        qb = t // Bq
+        block_start = H + qb * Bq
+        local_start = max(0, ((block_start - cfg.local) // c) * c) if block_start - cfg.local > 0 else 0
+        sink_end = min(cfg.sink, local_start)
+        allowed = np.zeros(L, bool)
+        allowed[:sink_end] = True
+        allowed[local_start:] = True
+        for m in group_idx[0, h, qb, :n_groups[0, h, qb]]:
+            allowed[m * g:(m + 1) * g] = True
+        allowed[pos + 1:] = False                     # causal
+        mask[t] = allowed
+    return mask
+
+
+def _masked_attention_numpy(q, k, v, mask, scale):
+    s = (q @ k.T) * scale
+    s = np.where(mask, s, -np.inf)
+    m = s.max(axis=1, keepdims=True)
+    e = np.exp(s - m)
+    z = e.sum(axis=1, keepdims=True)
+    return (e / z) @ v, (m + np.log(z))[:, 0]
+
+
+@pytest.mark.parametrize("hist", [64, 0])
+def test_routed_attention_equals_masked_dense_restatement(hist):
+    cfg = tiny(n_q_heads=4, n_kv_heads=2, total_len=64 + hist if hist else 128,
+               seg_len=64 if hist else 128)
+    x = make_inputs(cfg)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    r = oracle.route(cfg, x["Q"], cs, gs)
+    O, LSE = oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], r["group_idx"], r["n_groups"])
+    scale = 1.0 / np.sqrt(cfg.head_dim)
+    G = cfg.gqa
+    for hq in range(cfg.n_q_heads):
+        h = hq // G
+        mask = _mask_from_definition(cfg, h, r["group_idx"], r["n_groups"])
+        o, lse = _masked_attention_numpy(bf16_bits_to_f64(x["Q"][0, hq]), bf16_bits_to_f64(x["K"][0, h]),
+                                         bf16_bits_to_f64(x["V"][0, h]), mask, scale)
+        assert np.max(np.abs(o - O[0, hq])) < 1e-12
+        assert np.max(np.abs(lse - LSE[0, hq])) < 1e-12
+
+
+def _torch_attention_grads(cfg, x, mask_fn):
+    """Library special case: torch SDPA in fp64 with autograd (boolean mask or causal)."""
+    G, H = cfg.gqa, cfg.history
+    q = torch.from_numpy(bf16_bits_to_f64(x["Q"])).requires_grad_(True)
+    k = torch.from_numpy(bf16_bits_to_f64(x["K"])).requires_grad_(True)
+    v = torch.from_numpy(bf16_bits_to_f64(x["V"])).requires_grad_(True)
+    go = torch.from_numpy(bf16_bits_to_f64(x["dO"]))
+    ke = k.repeat_interleave(G, dim=1)
+    ve = v.repeat_interleave(G, dim=1)
+    mask = torch.stack([torch.from_numpy(mask_fn(hq // G)) for hq in range(cfg.n_q_heads)])[None]
+    o = torch.nn.functional.scaled_dot_product_attention(q, ke, ve, attn_mask=mask)
+    (o * go).sum().backward()
+    return (o.detach().numpy(), q.grad.numpy(), k.grad[:, :, H:].numpy(), v.grad[:, :, H:].numpy(),
+            k.grad[:, :, :H].numpy())
+
+
+@pytest.mark.parametrize("hist", [0, 64])
+def test_full_budget_equals_dense_causal_attention(hist):
+    # "dense timing is obtained by disabling the router" (Section 4.2): with a budget that
+    # covers every candidate chunk and every group, HGA is dense causal attention.
+    cfg = tiny(n_q_heads=4, n_kv_heads=2, total_len=128 + hist, seg_len=128,
+               topk_chunks=(128 + hist) // 8, topk_groups=4)
+    x = make_inputs(cfg)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    r = oracle.route(cfg, x["Q"], cs, gs)
+    O, LSE = oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], r["group_idx"], r["n_groups"])
+    dQ, dK, dV = oracle.attn_bwd(cfg, x["Q"], x["K"], x["V"], x["dO"], r["group_idx"], r["n_groups"])
+    S, L, H = cfg.seg_len, cfg.total_len, cfg.history
+    causal = np.tril(np.ones((L, L), bool))[H:]
+    o, gq, gk, gv, _ = _torch_attention_grads(cfg, x, lambda h: causal)
+    assert np.max(np.abs(o - O)) < 1e-12
+    assert np.max(np.abs(gq - dQ)) < 1e-11
+    assert np.max(np.abs(gk - dK)) < 1e-11
+    assert np.max(np.abs(gv - dV)) < 1e-11
+    # and the log-sum-exp against a direct evaluation
+    qf, kf = bf16_bits_to_f64(x["Q"]), bf16_bits_to_f64(x["K"])
+    s = np.einsum("sd,ld->sl", qf[0, 3], kf[0, 1]) / np.sqrt(cfg.head_dim)
+    s = np.where(causal, s, -np.inf)
+    assert np.max(np.abs(np.log(np.exp(s).sum(1)) - LSE[0, 3])) < 1e-12
+
+
+def test_backward_matches_autograd_on_routed_mask_and_detaches_history():
+    cfg = tiny(n_q_heads=4, n_kv_heads=2, total_len=192, seg_len=64)
+    x = make_inputs(cfg)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    r = oracle.route(cfg, x["Q"], cs, gs)
+    dQ, dK, dV = oracle.attn_bwd(cfg, x["Q"], x["K"], x["V"], x["dO"], r["group_idx"], r["n_groups"])
+    o, gq, gk, gv, gk_hist = _torch_attention_grads(
+        cfg, x, lambda h: _mask_from_definition(cfg, h, r["group_idx"], r["n_groups"]))
+    assert np.max(np.abs(gq - dQ)) < 1e-11
+    assert np.max(np.abs(gk - dK)) < 1e-11
+    assert np.max(np.abs(gv - dV)) < 1e-11
+    # Section 2.2: history K/V is read (autograd would give it a gradient) but detached:
+    # the oracle returns rows for the S active positions only
+    assert np.abs(gk_hist).max() > 0
+    assert dK.shape == (1, 2, cfg.seg_len, cfg.head_dim) and dV.shape == dK.shape
+
+
+def test_backward_finite_differences():
+    cfg = tiny(n_q_heads=2, n_kv_heads=1, total_len=96, seg_len=32)
+    x = make_inputs(cfg)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    r = oracle.route(cfg, x["Q"], cs, gs)
+    gi, ng = r["group_idx"], r["n_groups"]
+    Q, K, V, dO = (bf16_bits_to_f64(x[n]) for n in ("Q", "K", "V", "dO"))
+    dQ, dK, dV = oracle.attn_bwd_f64(cfg, Q, K, V, dO, gi, ng)
+    # the bf16 and the f64 entry points are the same arithmetic
+    dQb, dKb, dVb = oracle.attn_bwd(cfg, x["Q"], x["K"], x["V"], x["dO"], gi, ng)
+    assert np.array_equal(dQ, dQb) and np.allclose(dK, dKb, rtol=0, atol=1e-13) and np.allclose(dV, dVb, rtol=0, atol=1e-13)
+
+    def f(q, k, v):
+        return float((oracle.attn_fwd_f64(cfg, q, k, v, gi, ng)[0] * dO).sum())
+
+    rng = np.random.default_rng(5)
+    H, h = cfg.history, 1e-5
+    worst = 0.0
+    for name, arr, grad, off in (("Q", Q, dQ, 0), ("K", K, dK, H), ("V", V, dV, H)):
+        for _ in range(40):
+            idx = tuple(int(rng.integers(0, n)) for n in grad.shape)
+            full = (idx[0], idx[1], idx[2] + off, idx[3])
+            plus = [Q.copy(), K.copy(), V.copy()]
+            minus = [Q.copy(), K.copy(), V.copy()]
+            which = "QKV".index(name)
+            plus[which][full] += h
+            minus[which][full] -= h
+            fd = (f(*plus) - f(*minus)) / (2 * h)
+            worst = max(worst, abs(fd - grad[idx]) / max(1.0, abs(fd)))
+    assert worst < 1e-7, worst
+
+
+def test_no_leak_contracts():
+    cfg = tiny(n_q_heads=2, n_kv_heads=1, total_len=192, seg_len=64)
+    x = make_inputs(cfg)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    r = oracle.route(cfg, x["Q"], cs, gs)
+    gi, ng = r["group_idx"], r["n_groups"]
+    O, LSE = oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], gi, ng)
+    dQ, dK, dV = oracle.attn_bwd(cfg, x["Q"], x["K"], x["V"], x["dO"], gi, ng)
+    routed = set()
+    for qb in range(cfg.n_q_blocks):
+        routed |= set(oracle.routed_tokens(cfg, qb, gi[0, 0, qb, :ng[0, 0, qb]]).tolist())
+    unrouted = sorted(set(range(cfg.total_len)) - routed)
+    assert unrouted, "test needs some token no block attends to"
+    K2, V2 = x["K"].copy(), x["V"].copy()
+    K2[0, 0, unrouted] ^= 0x00F3
+    V2[0, 0, unrouted] ^= 0x00F3
+    O2, LSE2 = oracle.attn_fwd(cfg, x["Q"], K2, V2, gi, ng)
+    g2 = oracle.attn_bwd(cfg, x["Q"], K2, V2, x["dO"], gi, ng)
+    assert np.array_equal(O, O2) and np.array_equal(LSE, LSE2)
+    assert all(np.array_equal(a, b) for a, b in zip((dQ, dK, dV), g2))
+    # active rows nobody attends to get exactly zero dK/dV
+    H = cfg.history
+    dead = [t - H for t in unrouted if t >= H]
+    assert np.all(dK[0, 0, dead] == 0) and np.all(dV[0, 0, dead] == 0)
+    # row identity: sum_k dS_ik = 0  <=>  sum_d dQ_i . q_i  = sum_k dS_ik s_ik ... checked via
+    # the gradient of a shift-invariant softmax: adding a constant to all logits of a row
+    # changes nothing, i.e. f(Q) is invariant under K -> K + 1 u^T only through q.u; instead
+    # check sum over keys of dK contributions equals what dQ implies on a single-row case below.
+
+
+def test_row_identity_on_single_query_row():
+    # One query row (Bq = c = 8 forces 8 rows; use G = 1 and inspect a row via f64 entry):
+    # for softmax attention, sum_k dS_k = 0, hence sum_k dK_k = scale * (sum_k dS_k) q = 0
+    # when every key is visited by exactly one row.  Use S = Bq = 8, zero dO on all rows but one.
+    cfg = tiny(n_q_heads=1, n_kv_heads=1, total_len=8, seg_len=8, topk_chunks=0, sink=0, local=0)
+    rng = np.random.default_rng(11)
+    Q = rng.standard_normal((1, 1, 8, 16))
+    K = rng.standard_normal((1, 1, 8, 16))
+    V = rng.standard_normal((1, 1, 8, 16))
+    dO = np.zeros((1, 1, 8, 16))
+    dO[0, 0, 7] = rng.standard_normal(16)
+    gi = np.full((1, 1, 1, 0), -1, np.int32)
+    ng = np.zeros((1, 1, 1), np.int32)
+    dQ, dK, dV = oracle.attn_bwd_f64(cfg, Q, K, V, dO, gi, ng)
+    assert np.max(np.abs(dK[0, 0].sum(axis=0))) < 1e-12
+    assert np.abs(dK).max() > 1e-3
+    # dV = P^T dO: columns sum to dO since probabilities sum to one
+    assert np.max(np.abs(dV[0, 0].sum(axis=0) - dO[0, 0, 7])) < 1e-12
+
+
+def test_k_zero_and_no_history_edge_cases():
+    cfg = tiny(total_len=64, seg_len=64, topk_chunks=0)
+    x = make_inputs(cfg)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    r = oracle.route(cfg, x["Q"], cs, gs)
+    assert r["group_idx"].shape[-1] == 0 and np.all(r["n_groups"] == 0)
+    O, _ = oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], r["group_idx"], r["n_groups"])
+    # first position attends to itself only
+    assert np.allclose(O[0, :, 0], bf16_bits_to_f64(x["V"])[0, 0, 0], rtol=0, atol=1e-14)
+
+
+def test_attention_rejects_invalid_indices():
+    cfg = tiny()
+    x = make_inputs(cfg)
+    gi = np.full((1, 1, cfg.n_q_blocks, cfg.topk_chunks * cfg.kg_eff), -1, np.int32)
+    ng = np.zeros((1, 1, cfg.n_q_blocks), np.int32)
+    gi[0, 0, 0, :2] = (9, 9)      # duplicate
+    ng[0, 0, 0] = 2
+    with pytest.raises(RuntimeError):
+        oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], gi, ng)
+    gi[0, 0, 0, :2] = (0, 9)      # group 0 lies inside the sink
+    with pytest.raises(RuntimeError):
+        oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], gi, ng)
