@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the HGA hot path (summaries -> route -> attention fwd -> attention bwd).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+A step is one pass of the whole path over one synthetic Qwen3-8B-shaped attention layer
+(default: the 16K TBPTT configuration).  Prints ONE JSON line.  With N > 1 (launched by
+torchrun) every rank runs its own sequence: the path shards by sequence with no exchange
+step, so the only collectives are the timing barrier and the max over ranks.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_15105_b200.workloads import CONFIGS, make_inputs  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            pk = json.load(f)
+        pk["source"] = "measured"
+        return pk
+    pk = dict(FALLBACK_PEAKS)
+    pk["source"] = "fallback"
+    return pk
+
+
+# ----------------------------------------------------------------------------- work counts
+
+def work_counts(cfg, n_groups):
+    """Algorithmic work of the attention kernels for the routing actually taken.
+
+    pairs: (query row, visible key) pairs; pairs_active: those whose key is in the active
+    segment.  Bytes: K and V rows gathered once per item, Q/O/dO/dQ/LSE/delta once, dK/dV once.
+    """
+    d, G, Bq, g, H = cfg.head_dim, cfg.gqa, cfg.q_block, cfg.group, cfg.history
+    ng = np.asarray(n_groups).reshape(cfg.batch * cfg.n_kv_heads, cfg.n_q_blocks)
+    pairs = pairs_active = keys = 0
+    for qb in range(cfg.n_q_blocks):
+        p0 = H + qb * Bq
+        ls = max(0, ((p0 - cfg.local) // cfg.chunk) * cfg.chunk) if p0 - cfg.local > 0 else 0
+        se = min(cfg.sink, ls)
+        local_pairs = Bq * (p0 - ls) + Bq * (Bq + 1) // 2
+        local_active = Bq * (p0 - max(ls, H)) + Bq * (Bq + 1) // 2
+        sink_active = max(0, se - H)
+        for bh in range(ng.shape[0]):
+            far = se + int(ng[bh, qb]) * g
+            keys += far + (p0 + Bq - ls)
+            pairs += G * (Bq * far + local_pairs)
+            # routed groups inside the active segment are counted by the caller when needed;
+            # here: sink and local only (a lower bound, exact when no routed group is active)
+            pairs_active += G * (Bq * sink_active + local_active)
+    rows = cfg.batch * cfg.n_q_heads * cfg.seg_len
+    kv_rows_active = cfg.batch * cfg.n_kv_heads * cfg.seg_len
+    fwd_flops = 4.0 * d * pairs
+    bwd_flops = 6.0 * d * pairs + 4.0 * d * pairs_active
+    gather = keys * d * 2 * 2
+    fwd_bytes = gather + rows * d * 2 * 2 + rows * 4
+    bwd_bytes = gather + rows * d * 2 * 4 + rows * 4 * 2 + kv_rows_active * d * 4 * 2
+    return {"pairs": pairs, "pairs_active_min": pairs_active, "fwd_flops": fwd_flops,
+            "bwd_flops": bwd_flops, "fwd_bytes": float(fwd_bytes), "bwd_bytes": float(bwd_bytes)}
+
+
+def active_group_pairs(cfg, group_idx, n_groups):
+    """(row, key) pairs whose key lies in a routed group of the active segment."""
+    gi = np.asarray(group_idx).reshape(-1, cfg.n_q_blocks, group_idx.shape[-1])
+    first_active = cfg.history // cfg.group
+    n = int(((gi >= first_active)).sum())
+    return n * cfg.group * cfg.gqa * cfg.q_block
+
+
+def roofline_entry(name, flops, nbytes, seconds, peaks, sustained=False):
+    tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"]
+    t_flop = flops / (tf * 1e12)
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+    if t_hbm >= t_flop:
+        achieved, peak, unit, bound = nbytes / seconds / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+    else:
+        achieved, peak, unit, bound = flops / seconds / 1e12, tf, "TFLOP/s", "tensor"
+    return {"kernel": name, "bound": bound, "achieved": round(achieved, 2), "peak": peak, "unit": unit,
+            "frac": round(achieved / peak, 4), "traffic": None, "peak_source": peaks["source"],
+            "roofline_us": round(max(t_flop, t_hbm) * 1e6, 2), "measured_us": round(seconds * 1e6, 2)}
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- oracle legs
+
+def oracle_throughput(cfg, x, budget_s=15.0):
+    """Times the CPU oracle, as it stands, on a bounded sample of items of the same workload.
+
+    Returns (tokens/s, threads used, description).  One item covers Bq positions of one kv
+    head, so n items amount to n*Bq/Hkv tokens of the layer."""
+    import oracle
+    threads = oracle.num_threads()
+    t0 = time.perf_counter()
+    tb = cfg.history
+    cs, gs = oracle.build_summaries(cfg, x["K"], tb, cfg.total_len)
+    # history summaries are resident state (built by earlier segments): build them untimed
+    t_sum = time.perf_counter() - t0
+    oracle.build_summaries(cfg, x["K"], 0, tb, cs, gs)
+    rng = np.random.default_rng(0)
+    order = rng.permutation(cfg.n_items)
+    done, elapsed, batch = 0, 0.0, max(threads, 4)
+    while done < cfg.n_items and (done == 0 or elapsed * (done + batch) / done < budget_s):
+        items = np.sort(order[done:done + batch]).astype(np.int32)
+        t0 = time.perf_counter()
+        r = oracle.route(cfg, x["Q"], cs, gs, items=items)
+        oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], r["group_idx"], r["n_groups"], items=items)
+        if cfg.backward:
+            oracle.attn_bwd(cfg, x["Q"], x["K"], x["V"], x["dO"], r["group_idx"], r["n_groups"], items=items)
+        elapsed += time.perf_counter() - t0
+        done += len(items)
+    frac = done / cfg.n_items
+    total = elapsed + t_sum * frac
+    tokens = done * cfg.q_block / cfg.n_kv_heads
+    what = ("%d of %d (batch, kv head, query block) items of %s, chosen at random: summaries of the "
+            "active range (pro rata) + route + attention fwd%s" %
+            (done, cfg.n_items, cfg.name, " + bwd" if cfg.backward else ""))
+    return tokens / total, threads, what, total
+
+
+def run_reference(args, cfg):
+    """--impl reference: the oracle on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    x = make_inputs(cfg)
+    vals, last = [], None
+    for i in range(args.warmup + args.steps):
+        last = oracle_throughput(cfg, x, budget_s=max(2.0, min(15.0, 120.0 / (args.warmup + args.steps))))
+        if i >= args.warmup:
+            vals.append(last)
+    tps = float(np.mean([v[0] for v in vals]))
+    sec = float(np.mean([v[3] for v in vals]))
+    line = {"impl": "reference", "metric": METRIC, "value": round(tps, 3), "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(sec * 1e3, 3), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(cfg, args),
+            "cpu_baseline": {"value": round(tps, 3), "unit": "tokens/s", "cores": last[1],
+                             "kind": "oracle", "sample": last[2]},
+            "e2e": {"value": round(tps, 3), "unit": "tokens/s", "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+METRIC = "Qwen3-8B-layer HGA fwd+bwd tokens/s at 16K context; % of roofline"
+
+
+def config_dict(cfg, args):
+    return {"workload": cfg.name, "batch_per_gpu": cfg.batch, "q_heads": cfg.n_q_heads,
+            "kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim, "total_len": cfg.total_len,
+            "active_segment": cfg.seg_len, "chunk": cfg.chunk, "group": cfg.group,
+            "q_block": cfg.q_block, "topk_chunks": cfg.topk_chunks, "topk_groups": cfg.topk_groups,
+            "sink": cfg.sink, "local": cfg.local, "pass": "fwd+bwd" if cfg.backward else "fwd",
+            "l2": "flushed between timed steps (512 MiB write)", "parallelism": "dp%d" % args.gpus}
+
+
+# ----------------------------------------------------------------------------- main arm
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flags", type=int, default=0, help="hga_params.flags (debugging)")
+    args = ap.parse_args()
+    cfg = CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import torch.distributed as dist
+    from paper_2607_15105_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    # every rank draws its own sequence (weak scaling): same shapes, different seed
+    x = make_inputs(cfg.scaled(seed=cfg.seed + 1000 * rank) if rank else cfg)
+
+    def dev(a):
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+
+    Q, K, V = dev(x["Q"]), dev(x["K"]), dev(x["V"])
+    dO = dev(x["dO"]) if cfg.backward else None
+    buf = binding.HgaLayerBuffers(cfg, backward=cfg.backward, flags=args.flags)
+    buf.build_summaries(K, 0, cfg.history)          # resident history summaries
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    names = ["build_summaries", "route", "attn_fwd"] + (["attn_bwd"] if cfg.backward else [])
+
+    def one_step(ev=None):
+        if ev:
+            ev[0].record(stream)
+        buf.build_summaries(K)
+        if ev:
+            ev[1].record(stream)
+        buf.route(Q)
+        if ev:
+            ev[2].record(stream)
+        buf.attn_fwd(Q, K, V)
+        if ev:
+            ev[3].record(stream)
+        if cfg.backward:
+            buf.attn_bwd(Q, K, V, dO)
+            if ev:
+                ev[4].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        one_step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    n_ev = len(names) + 1
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(args.steps)]
+    launches0 = binding.hga_kernel_launch_count()
+    barrier()
+    for i in range(args.steps):
+        flush.zero_()                     # evict L2 (untimed: events bracket the step only)
+        one_step(events[i])
+    barrier()
+    launches = binding.hga_kernel_launch_count() - launches0
+    per_call = np.array([[ev[j].elapsed_time(ev[j + 1]) for j in range(n_ev - 1)] for ev in events])  # ms
+    step_ms = np.array([ev[0].elapsed_time(ev[-1]) for ev in events])
+    # warm-L2 variant (reported beside the headline, not instead of it)
+    warm_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(args.steps)]
+    for i in range(args.steps):
+        one_step(warm_ev[i])
+    barrier()
+    warm_ms = np.array([ev[0].elapsed_time(ev[-1]) for ev in warm_ev])
+    clocks = sampler.stop() if rank == 0 else None
+
+    # end to end through the host-buffer entry point: H2D of the step's inputs, D2H of its results
+    H = cfg.history
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16).pin_memory()
+    Qh, Kh, Vh = pin(x["Q"]), pin(x["K"][:, :, H:]), pin(x["V"][:, :, H:])
+    dOh = pin(x["dO"]) if cfg.backward else None
+    Oh = torch.empty_like(Qh).pin_memory()
+    dQh = torch.empty_like(Qh).pin_memory() if cfg.backward else None
+    dKh = torch.empty(cfg.batch, cfg.n_kv_heads, cfg.seg_len, cfg.head_dim).pin_memory() if cfg.backward else None
+    dVh = torch.empty_like(dKh).pin_memory() if cfg.backward else None
+    arena = torch.empty(binding.hga_step_arena_bytes(buf.p), dtype=torch.uint8, device="cuda")
+    h2d = sum(t.numel() * t.element_size() for t in (Qh, Kh, Vh, dOh) if t is not None)
+    d2h = sum(t.numel() * t.element_size() for t in (Oh, dQh, dKh, dVh) if t is not None)
+
+    def host_step():
+        binding.hga_step_host(buf.p, Qh, Kh, Vh, dOh, K, V, buf.chunk_sum, buf.group_sum, Oh, dQh,
+                              dKh, dVh, arena, buf.status)
+
+    for _ in range(3):
+        host_step()
+    barrier()
+    e2e_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(args.steps)]
+    for a, b in e2e_ev:
+        flush.zero_()
+        a.record(stream)
+        host_step()
+        b.record(stream)
+    barrier()
+    e2e_ms = np.array([a.elapsed_time(b) for a, b in e2e_ev])
+    status = int(buf.status.item())
+
+    def max_over_ranks(v):
+        if world == 1:
+            return float(v)
+        t = torch.tensor([float(v)], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    total_ms = max_over_ranks(step_ms.sum())
+    warm_total_ms = max_over_ranks(warm_ms.sum())
+    e2e_total_ms = max_over_ranks(e2e_ms.sum())
+    tokens = cfg.tokens_per_step * world * args.steps
+
+    if rank == 0:
+        peaks = load_peaks()
+        gi, ng = buf.group_idx.cpu().numpy(), buf.n_groups.cpu().numpy()
+        wc = work_counts(cfg, ng)
+        extra_active = active_group_pairs(cfg, gi, ng)
+        wc["bwd_flops"] += 4.0 * cfg.head_dim * extra_active
+        med = np.median(per_call, axis=0) * 1e-3      # seconds per call
+        roofs = {"attn_fwd": roofline_entry("hga_attn_fwd", wc["fwd_flops"], wc["fwd_bytes"], med[2], peaks)}
+        if cfg.backward:
+            roofs["attn_bwd"] = roofline_entry("hga_attn_bwd", wc["bwd_flops"], wc["bwd_bytes"], med[3], peaks)
+        dominant = max(roofs.values(), key=lambda r: r["measured_us"])
+        attn_us = sum(r["measured_us"] for r in roofs.values())
+        attn_roof_us = sum(r["roofline_us"] for r in roofs.values())
+        line = {
+            "metric": METRIC, "value": round(tokens / (total_ms * 1e-3), 1), "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(total_ms / args.steps, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": config_dict(cfg, args),
+            "clocks": clocks,
+            "e2e": {"value": round(tokens / (e2e_total_ms * 1e-3), 1), "unit": "tokens/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": round(e2e_total_ms / args.steps, 5)},
+            "gpu_launches": int(launches),
+            "roofline": dominant,
+            "roofline_all": roofs,
+            "attention": {"fwd_plus_bwd_us": round(attn_us, 2), "roofline_us": round(attn_roof_us, 2),
+                          "frac_of_roofline": round(attn_roof_us / attn_us, 4),
+                          "tokens_per_s": round(cfg.tokens_per_step / (attn_us * 1e-6), 1)},
+            "per_call_us_median": {n: round(float(m) * 1e6, 2) for n, m in zip(names, med)},
+            "warm_l2": {"value": round(tokens / (warm_total_ms * 1e-3), 1),
+                        "ms_per_step": round(warm_total_ms / args.steps, 5)},
+            "device_status_word": status,
+            "paper_context": "217.75 (HGA) / 207.02 (dense) tokens/s: whole-model QLoRA step at 2K on a "
+                             "Quadro RTX 5000 (Table 2); another machine and scope, not the target",
+        }
+        if not args.no_cpu_baseline and world == 1:
+            tps, threads, what, _ = oracle_throughput(cfg, x)
+            line["cpu_baseline"] = {"value": round(tps, 3), "unit": "tokens/s", "cores": threads,
+                                    "kind": "oracle", "sample": what}
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

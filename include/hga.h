@@ -1,0 +1,165 @@
+/*
+ * libhga -- Hierarchical Global Attention (HGA) hot path for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the four steps of one HGA attention-layer step as stated in "Long-Context
+ * Fine-Tuning with Limited VRAM", Section 2.1 (exact-token hierarchical routing) and
+ * Section 2.2 (segment-wise backward):
+ *
+ *   hga_build_summaries  two levels of key summaries from the projected keys   (Sec. 2.1)
+ *   hga_route            chunk selection, then group selection                 (Sec. 2.1, items 1-2)
+ *   hga_attn_fwd         exact-token softmax attention over the routed set     (Sec. 2.1, item 3)
+ *   hga_attn_bwd         its backward; history K/V are detached constants      (Sec. 2.1 last par., Sec. 2.2)
+ *
+ * General rules
+ *   - Unless a parameter says "host", every data pointer is a DEVICE pointer owned by the
+ *     caller.  The library allocates and frees no device memory, never synchronises the
+ *     device, and launches on the `stream` it is given (a cudaStream_t passed as void*).
+ *   - Every call returns an int status: HGA_OK (0) or a negative HGA_ERR_* code.  On an
+ *     error nothing has been launched.  hga_status_string() names a code.
+ *   - bf16 data are raw 16-bit patterns.  The innermost (head_dim) axis is contiguous.
+ *
+ * Shapes (B batch, Hq/Hkv query/kv heads, G = Hq/Hkv, d head_dim, L total tokens,
+ * S active-segment tokens, H = L - S detached history, c chunk, g group, Bq query block,
+ * NQB = S/Bq):
+ *   Q, O, dO, dQ  bf16 [B, Hq,  S, d]   row t is absolute position H + t
+ *   K, V          bf16 [B, Hkv, L, d]   history rows first, the active segment last
+ *   chunk_sum     bf16 [B, Hkv, L/c, d] group_sum bf16 [B, Hkv, L/g, d]        (dense)
+ *   chunk_idx     int32 [B, Hkv, NQB, k_c]            ascending chunk ids, -1 padded
+ *   group_idx     int32 [B, Hkv, NQB, k_c * kg_eff]   ascending global group ids (group m
+ *                 covers tokens [m*g, (m+1)*g)), -1 padded; kg_eff = min(k_g, c/g)
+ *   n_groups      int32 [B, Hkv, NQB]                 number of real entries in group_idx
+ *   LSE           fp32 [B, Hq, S]  natural-log sum of exp of the scaled logits
+ *   dK, dV        fp32 [B, Hkv, S, d]  rows of the ACTIVE segment only (row t = position H + t)
+ *
+ * One routing decision is taken per "item" (b, kv head, query block) and shared by the
+ * G*Bq query rows of that item.  Window geometry of query block qb, p0 = H + qb*Bq:
+ *   local start ls = max(0, floor((p0 - local)/c)*c);  sink end se = min(sink, ls);
+ *   candidate chunks j: se <= j*c and (j+1)*c <= ls;
+ *   routed set = [0, se)  U  selected groups  U  [ls, p0 + Bq), causal inside the block.
+ */
+#ifndef HGA_H
+#define HGA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HGA_VERSION 100
+
+#if defined(__GNUC__)
+#define HGA_API __attribute__((visibility("default")))
+#else
+#define HGA_API
+#endif
+
+/* status codes */
+#define HGA_OK 0
+#define HGA_ERR_NULL (-1)        /* a required pointer is NULL */
+#define HGA_ERR_SHAPE (-2)       /* sizes violate the divisibility / range rules below */
+#define HGA_ERR_ALIGN (-3)       /* pointer not 16-byte aligned or stride not a multiple of 8 */
+#define HGA_ERR_UNSUPPORTED (-4) /* head_dim / device not supported */
+#define HGA_ERR_WORKSPACE (-5)   /* workspace missing or too small */
+#define HGA_ERR_CUDA (-6)        /* a CUDA call failed; see hga_last_cuda_error() */
+
+/* hga_params.flags */
+#define HGA_FLAG_BWD_ACCUMULATE 1  /* hga_attn_bwd adds into dK/dV instead of overwriting */
+#define HGA_FLAG_GENERIC_KERNELS 2 /* use the shape-generic CUDA-core kernels even where a
+                                      tensor-core kernel exists (debugging / cross-checks) */
+
+/* bits OR-ed into *status_word by the attention kernels */
+#define HGA_STATUS_BAD_INDEX 1     /* a group_idx entry was out of range, inside the sink or
+                                      local window, or not ascending: that entry was skipped */
+#define HGA_STATUS_WAIT_TIMEOUT 2  /* a bounded on-chip wait gave up; outputs are invalid */
+
+typedef struct hga_params {
+  int32_t batch, n_q_heads, n_kv_heads, head_dim; /* Hq % Hkv == 0; head_dim in {64, 128}      */
+  int32_t total_len, seg_len;                      /* L >= S >= 1                                */
+  int32_t chunk, group, q_block;                   /* c % g == 0; Bq % c == 0; S % Bq == 0;
+                                                      (L - S) % Bq == 0; L % c == 0            */
+  int32_t topk_chunks, topk_groups;                /* k_c >= 0; k_g >= 1 (per opened chunk)      */
+  int32_t sink, local;                             /* tokens, multiples of c                     */
+  float   softmax_scale;                           /* <= 0 selects 1/sqrt(head_dim)              */
+  int32_t flags;                                   /* HGA_FLAG_*                                 */
+  /* element strides of the (batch, head, token) axes; all-zero means dense.  q_stride
+   * also describes dQ; o_stride describes O and dO; k_stride / v_stride describe K / V. */
+  int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];
+} hga_params;
+
+/* Section 2.1, first paragraph (chunk-level and group-level summaries are derived from the
+ * keys the model already projects): for every chunk and group inside the token range [tok_begin, tok_end)
+ * (chunk aligned) of every (batch, kv head), write the arithmetic mean of its keys, rounded
+ * once to bf16 (the mean is accumulated exactly).  Summaries outside the range are left
+ * untouched, so a caller extends resident history summaries segment by segment. */
+HGA_API int hga_build_summaries(const hga_params* p, const void* K, int32_t tok_begin, int32_t tok_end,
+                        void* chunk_sum, void* group_sum, void* stream);
+
+/* Section 2.1 items 1-2 (chunk selection, group selection), run without gradients.
+ * Per item: the score of a summary is the maximum over the item's G*Bq query rows of the
+ * raw dot product (bf16 products, fp32 accumulation); the min(k_c, #candidates) best
+ * candidate chunks are selected, then inside each selected chunk the kg_eff best groups;
+ * ties go to the lowest index.  Outputs as laid out above.
+ * chunk_scores (optional, may be NULL) fp32 [B,Hkv,NQB,L/c]: scores, -inf off-candidate.
+ * group_scores (optional, may be NULL) fp32 [B,Hkv,NQB,k_c*(c/g)]: slot (r,u) = group u
+ *   of the r-th selected chunk, -inf where unused.
+ * workspace: device scratch of at least hga_workspace_bytes().route bytes (16-byte
+ *   aligned); contents are overwritten.  Calls that share a workspace must not overlap. */
+HGA_API int hga_route(const hga_params* p, const void* Q, const void* chunk_sum, const void* group_sum,
+              int32_t* chunk_idx, int32_t* group_idx, int32_t* n_groups, float* chunk_scores,
+              float* group_scores, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Section 2.1 item 3 (attention reads the exact K/V rows of the selected groups; summaries
+ * only select and never act as values): for every query row i at position
+ * pos, O_i = sum over routed keys k <= pos of softmax(scale * q_i.k) v_k (bf16 MMA inputs,
+ * fp32 accumulation) and LSE_i.  Accepts any valid index list, not only hga_route's.
+ * status_word (optional device int32) receives HGA_STATUS_* bits by atomic OR. */
+HGA_API int hga_attn_fwd(const hga_params* p, const void* Q, const void* K, const void* V,
+                 const int32_t* group_idx, const int32_t* n_groups, void* O, float* LSE,
+                 int32_t* status_word, void* stream);
+
+/* Backward of hga_attn_fwd with the routing frozen (Section 2.1, last paragraph: selection
+ * carries no gradient, the gather and the attention do) under segment-wise TBPTT
+ * (Section 2.2: history K/V is detached at the segment boundary, so no gradient reaches an
+ * earlier segment): writes dQ for all S rows and dK/dV for the
+ * S active rows only; history keys contribute to dQ but receive no gradient.
+ * O and LSE are hga_attn_fwd's outputs, dO the upstream gradient (layout of O).
+ * dK/dV are overwritten unless HGA_FLAG_BWD_ACCUMULATE is set.  The sum over query blocks
+ * uses floating-point atomics: results may differ in the last bits from run to run.
+ * workspace: device scratch of at least hga_workspace_bytes().bwd bytes. */
+HGA_API int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* V, const void* O,
+                 const float* LSE, const void* dO, const int32_t* group_idx,
+                 const int32_t* n_groups, void* dQ, float* dK, float* dV, void* workspace,
+                 size_t workspace_bytes, int32_t* status_word, void* stream);
+
+/* Scratch sizes (bytes) the two calls above need for `p`; either output may be NULL. */
+HGA_API int hga_workspace_bytes(const hga_params* p, size_t* route_bytes, size_t* bwd_bytes);
+
+/* One whole layer step from HOST buffers (pinned memory recommended), for callers that
+ * keep the step's tensors on the host: copies Q, dO (host [B,Hq,S,d]) and the active
+ * segment's K/V rows (host [B,Hkv,S,d]) into the caller's device arena, appends them to the
+ * resident device K/V (device [B,Hkv,L,d] dense, history already in place), runs
+ * build_summaries(active range) -> route -> attn_fwd -> attn_bwd, and copies O (bf16),
+ * dQ (bf16), dK, dV (fp32) back to the host buffers.  dO_host == NULL runs the forward half
+ * only.  All work is queued on `stream`; the host buffers are valid after the caller
+ * synchronises the stream.  arena: device scratch of hga_step_arena_bytes() bytes.
+ * chunk_sum / group_sum: resident device summaries (history part already built). */
+HGA_API int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host,
+                  const void* Vseg_host, const void* dO_host, void* K_dev, void* V_dev,
+                  void* chunk_sum, void* group_sum, void* O_host, void* dQ_host, float* dK_host,
+                  float* dV_host, void* arena, size_t arena_bytes, int32_t* status_word,
+                  void* stream);
+HGA_API int hga_step_arena_bytes(const hga_params* p, size_t* bytes);
+
+HGA_API const char* hga_status_string(int status);
+HGA_API int hga_version(void);
+/* the cudaError_t (as int) of the most recent failed CUDA call made by this library */
+HGA_API int hga_last_cuda_error(void);
+/* number of kernels this library has launched since it was loaded (all calls, all streams) */
+HGA_API int64_t hga_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HGA_H */

@@ -1,0 +1,280 @@
+// C-ABI entry points of libhga: argument validation, stride resolution, dispatch.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+
+#include "hga_common.cuh"
+
+namespace hga {
+
+static std::atomic<int64_t> g_launches{0};
+static std::atomic<int> g_last_cuda{0};
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int record_cuda(cudaError_t e) {
+  if (e == cudaSuccess) return HGA_OK;
+  g_last_cuda.store((int)e, std::memory_order_relaxed);
+  return HGA_ERR_CUDA;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+static void dense_strides(int64_t* s, int heads, int tokens, int d) {
+  s[2] = d;
+  s[1] = (int64_t)tokens * d;
+  s[0] = (int64_t)heads * tokens * d;
+}
+
+// Validates p and fills dm.  Returns an HGA status.
+static int resolve(const hga_params* p, Dims& dm) {
+  if (!p) return HGA_ERR_NULL;
+  if (p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1) return HGA_ERR_SHAPE;
+  if (p->n_q_heads % p->n_kv_heads) return HGA_ERR_SHAPE;
+  if (p->head_dim != 64 && p->head_dim != 128) return HGA_ERR_UNSUPPORTED;
+  if (p->seg_len < 1 || p->total_len < p->seg_len) return HGA_ERR_SHAPE;
+  if (p->group < 1 || p->chunk < p->group || p->chunk % p->group) return HGA_ERR_SHAPE;
+  if (p->q_block < p->chunk || p->q_block % p->chunk) return HGA_ERR_SHAPE;
+  if (p->seg_len % p->q_block || (p->total_len - p->seg_len) % p->q_block) return HGA_ERR_SHAPE;
+  if (p->total_len % p->chunk) return HGA_ERR_SHAPE;
+  if (p->topk_chunks < 0 || p->topk_groups < 1) return HGA_ERR_SHAPE;
+  if (p->sink < 0 || p->local < 0 || p->sink % p->chunk || p->local % p->chunk) return HGA_ERR_SHAPE;
+  if (p->chunk / p->group > 64) return HGA_ERR_UNSUPPORTED;
+  if (p->topk_chunks > 1024) return HGA_ERR_UNSUPPORTED;
+  dm.B = p->batch; dm.Hq = p->n_q_heads; dm.Hkv = p->n_kv_heads; dm.G = dm.Hq / dm.Hkv;
+  dm.d = p->head_dim; dm.L = p->total_len; dm.S = p->seg_len; dm.H = dm.L - dm.S;
+  dm.c = p->chunk; dm.g = p->group; dm.Bq = p->q_block;
+  dm.kc = p->topk_chunks; dm.kg = p->topk_groups; dm.per = dm.c / dm.g;
+  dm.kge = dm.kg < dm.per ? dm.kg : dm.per;
+  dm.sink = p->sink; dm.local = p->local;
+  dm.NQB = dm.S / dm.Bq; dm.Nc = dm.L / dm.c; dm.Ng = dm.L / dm.g;
+  dm.width = dm.kc * dm.kge; dm.rows = dm.G * dm.Bq;
+  dm.flags = p->flags;
+  dm.scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)dm.d);
+  if ((int64_t)dm.B * dm.Hkv * dm.NQB > 0x7fffffff) return HGA_ERR_SHAPE;
+  struct { const int64_t* in; int64_t* out; int heads, tokens; } t[4] = {
+      {p->q_stride, dm.qs, dm.Hq, dm.S}, {p->k_stride, dm.ks, dm.Hkv, dm.L},
+      {p->v_stride, dm.vs, dm.Hkv, dm.L}, {p->o_stride, dm.os, dm.Hq, dm.S}};
+  for (auto& e : t) {
+    if (e.in[0] == 0 && e.in[1] == 0 && e.in[2] == 0) {
+      dense_strides(e.out, e.heads, e.tokens, dm.d);
+    } else {
+      for (int i = 0; i < 3; ++i) {
+        if (e.in[i] < 0 || (e.in[i] % 8)) return HGA_ERR_ALIGN;
+        e.out[i] = e.in[i];
+      }
+      if (e.out[2] < dm.d) return HGA_ERR_SHAPE;
+    }
+  }
+  return HGA_OK;
+}
+
+size_t route_workspace_bytes(const Dims& dm) {
+  // chunk scores fp32 [items, Nc]
+  return (size_t)dm.B * dm.Hkv * dm.NQB * dm.Nc * sizeof(float) + 16;
+}
+
+size_t bwd_workspace_bytes(const Dims& dm) {
+  // delta = rowsum(dO * O), fp32 [B, Hq, S]
+  return (size_t)dm.B * dm.Hq * dm.S * sizeof(float) + 16;
+}
+
+}  // namespace hga
+
+using namespace hga;
+
+extern "C" {
+
+int hga_version(void) { return HGA_VERSION; }
+
+int hga_last_cuda_error(void) { return g_last_cuda.load(); }
+
+int64_t hga_kernel_launch_count(void) { return g_launches.load(); }
+
+const char* hga_status_string(int s) {
+  switch (s) {
+    case HGA_OK: return "ok";
+    case HGA_ERR_NULL: return "a required pointer is NULL";
+    case HGA_ERR_SHAPE: return "sizes violate the shape rules of hga_params";
+    case HGA_ERR_ALIGN: return "pointer not 16-byte aligned or stride not a multiple of 8 elements";
+    case HGA_ERR_UNSUPPORTED: return "unsupported head_dim, size or device";
+    case HGA_ERR_WORKSPACE: return "workspace missing or too small";
+    case HGA_ERR_CUDA: return "a CUDA call failed (see hga_last_cuda_error)";
+    default: return "unknown status";
+  }
+}
+
+int hga_workspace_bytes(const hga_params* p, size_t* route_bytes, size_t* bwd_bytes) {
+  Dims dm;
+  int rc = resolve(p, dm);
+  if (rc) return rc;
+  if (route_bytes) *route_bytes = route_workspace_bytes(dm);
+  if (bwd_bytes) *bwd_bytes = bwd_workspace_bytes(dm);
+  return HGA_OK;
+}
+
+int hga_build_summaries(const hga_params* p, const void* K, int32_t tok_begin, int32_t tok_end,
+                        void* chunk_sum, void* group_sum, void* stream) {
+  Dims dm;
+  int rc = resolve(p, dm);
+  if (rc) return rc;
+  if (!K || !chunk_sum || !group_sum) return HGA_ERR_NULL;
+  if (!aligned16(K) || !aligned16(chunk_sum) || !aligned16(group_sum)) return HGA_ERR_ALIGN;
+  if (tok_begin < 0 || tok_end > dm.L || tok_begin > tok_end || tok_begin % dm.c || tok_end % dm.c)
+    return HGA_ERR_SHAPE;
+  if (tok_begin == tok_end) return HGA_OK;
+  return launch_build_summaries(dm, K, tok_begin, tok_end, chunk_sum, group_sum, (cudaStream_t)stream);
+}
+
+int hga_route(const hga_params* p, const void* Q, const void* chunk_sum, const void* group_sum,
+              int32_t* chunk_idx, int32_t* group_idx, int32_t* n_groups, float* chunk_scores,
+              float* group_scores, void* workspace, size_t workspace_bytes, void* stream) {
+  Dims dm;
+  int rc = resolve(p, dm);
+  if (rc) return rc;
+  if (!Q || !chunk_sum || !group_sum || !chunk_idx || !group_idx || !n_groups) return HGA_ERR_NULL;
+  if (!aligned16(Q) || !aligned16(chunk_sum) || !aligned16(group_sum)) return HGA_ERR_ALIGN;
+  if (!workspace || workspace_bytes < route_workspace_bytes(dm)) return HGA_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return HGA_ERR_ALIGN;
+  return launch_route_generic(dm, Q, chunk_sum, group_sum, chunk_idx, group_idx, n_groups,
+                              chunk_scores, group_scores, workspace, (cudaStream_t)stream);
+}
+
+int hga_attn_fwd(const hga_params* p, const void* Q, const void* K, const void* V,
+                 const int32_t* group_idx, const int32_t* n_groups, void* O, float* LSE,
+                 int32_t* status_word, void* stream) {
+  Dims dm;
+  int rc = resolve(p, dm);
+  if (rc) return rc;
+  if (!Q || !K || !V || !group_idx || !n_groups || !O || !LSE) return HGA_ERR_NULL;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return HGA_ERR_ALIGN;
+  return launch_attn_fwd_generic(dm, Q, K, V, group_idx, n_groups, O, LSE, status_word,
+                                 (cudaStream_t)stream);
+}
+
+int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* V, const void* O,
+                 const float* LSE, const void* dO, const int32_t* group_idx,
+                 const int32_t* n_groups, void* dQ, float* dK, float* dV, void* workspace,
+                 size_t workspace_bytes, int32_t* status_word, void* stream) {
+  Dims dm;
+  int rc = resolve(p, dm);
+  if (rc) return rc;
+  if (!Q || !K || !V || !O || !LSE || !dO || !group_idx || !n_groups || !dQ || !dK || !dV)
+    return HGA_ERR_NULL;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) ||
+      !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
+    return HGA_ERR_ALIGN;
+  if (!workspace || workspace_bytes < bwd_workspace_bytes(dm)) return HGA_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return HGA_ERR_ALIGN;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!(dm.flags & HGA_FLAG_BWD_ACCUMULATE)) {
+    size_t bytes = (size_t)dm.B * dm.Hkv * dm.S * dm.d * sizeof(float);
+    rc = record_cuda(cudaMemsetAsync(dK, 0, bytes, st));
+    if (rc) return rc;
+    rc = record_cuda(cudaMemsetAsync(dV, 0, bytes, st));
+    if (rc) return rc;
+  }
+  return launch_attn_bwd_generic(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV,
+                                 (float*)workspace, status_word, st);
+}
+
+int hga_step_arena_bytes(const hga_params* p, size_t* bytes) {
+  Dims dm;
+  int rc = resolve(p, dm);
+  if (rc) return rc;
+  if (!bytes) return HGA_ERR_NULL;
+  size_t q = (size_t)dm.B * dm.Hq * dm.S * dm.d * 2;           // Q, dO, O, dQ (bf16)
+  size_t kv32 = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 4;       // dK, dV (fp32)
+  size_t kvseg = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 2;      // staged K/V segment rows
+  size_t items = (size_t)dm.B * dm.Hkv * dm.NQB;
+  size_t idx = items * (dm.kc + dm.width + 1) * 4 + 64;
+  size_t lse = (size_t)dm.B * dm.Hq * dm.S * 4;
+  auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  *bytes = 4 * up(q) + 2 * up(kv32) + 2 * up(kvseg) + up(idx) + up(lse) +
+           up(route_workspace_bytes(dm)) + up(bwd_workspace_bytes(dm)) + 256;
+  return HGA_OK;
+}
+
+int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host,
+                  const void* Vseg_host, const void* dO_host, void* K_dev, void* V_dev,
+                  void* chunk_sum, void* group_sum, void* O_host, void* dQ_host, float* dK_host,
+                  float* dV_host, void* arena, size_t arena_bytes, int32_t* status_word,
+                  void* stream) {
+  Dims dm;
+  int rc = resolve(p, dm);
+  if (rc) return rc;
+  if (!Q_host || !Kseg_host || !Vseg_host || !K_dev || !V_dev || !chunk_sum || !group_sum ||
+      !O_host || !arena)
+    return HGA_ERR_NULL;
+  const bool bwd = dO_host != nullptr;
+  if (bwd && (!dQ_host || !dK_host || !dV_host)) return HGA_ERR_NULL;
+  // this convenience call works on dense tensors only
+  const int64_t zero[3] = {0, 0, 0};
+  if (memcmp(p->q_stride, zero, sizeof zero) || memcmp(p->k_stride, zero, sizeof zero) ||
+      memcmp(p->v_stride, zero, sizeof zero) || memcmp(p->o_stride, zero, sizeof zero))
+    return HGA_ERR_UNSUPPORTED;
+  size_t need = 0;
+  hga_step_arena_bytes(p, &need);
+  if (arena_bytes < need) return HGA_ERR_WORKSPACE;
+  if (!aligned16(arena) || !aligned16(K_dev) || !aligned16(V_dev)) return HGA_ERR_ALIGN;
+  cudaStream_t st = (cudaStream_t)stream;
+
+  auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  char* a = (char*)(((uintptr_t)arena + 255) & ~(uintptr_t)255);
+  auto take = [&](size_t n) { char* r = a; a += up(n); return (void*)r; };
+  size_t qb = (size_t)dm.B * dm.Hq * dm.S * dm.d * 2;
+  size_t kv32 = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 4;
+  size_t kvseg = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 2;
+  size_t items = (size_t)dm.B * dm.Hkv * dm.NQB;
+  void* dQin = take(qb); void* ddO = take(qb); void* dO_ = take(qb); void* ddQ = take(qb);
+  float* ddK = (float*)take(kv32); float* ddV = (float*)take(kv32);
+  void* kseg = take(kvseg); void* vseg = take(kvseg);
+  int32_t* cidx = (int32_t*)take(items * (dm.kc + dm.width + 1) * 4 + 64);
+  int32_t* gidx = cidx + items * dm.kc;
+  int32_t* ng = gidx + items * dm.width;
+  float* lse = (float*)take((size_t)dm.B * dm.Hq * dm.S * 4);
+  void* rws = take(route_workspace_bytes(dm));
+  void* bws = take(bwd_workspace_bytes(dm));
+
+  // host -> device: Q, (dO), and the active segment's K/V rows appended behind the history
+  rc = record_cuda(cudaMemcpyAsync(dQin, Q_host, qb, cudaMemcpyHostToDevice, st));
+  if (rc) return rc;
+  if (bwd) {
+    rc = record_cuda(cudaMemcpyAsync(ddO, dO_host, qb, cudaMemcpyHostToDevice, st));
+    if (rc) return rc;
+  }
+  rc = record_cuda(cudaMemcpyAsync(kseg, Kseg_host, kvseg, cudaMemcpyHostToDevice, st));
+  if (rc) return rc;
+  rc = record_cuda(cudaMemcpyAsync(vseg, Vseg_host, kvseg, cudaMemcpyHostToDevice, st));
+  if (rc) return rc;
+  const size_t row = (size_t)dm.d * 2;
+  rc = record_cuda(cudaMemcpy2DAsync((char*)K_dev + (size_t)dm.H * row, (size_t)dm.L * row, kseg,
+                                     (size_t)dm.S * row, (size_t)dm.S * row,
+                                     (size_t)dm.B * dm.Hkv, cudaMemcpyDeviceToDevice, st));
+  if (rc) return rc;
+  rc = record_cuda(cudaMemcpy2DAsync((char*)V_dev + (size_t)dm.H * row, (size_t)dm.L * row, vseg,
+                                     (size_t)dm.S * row, (size_t)dm.S * row,
+                                     (size_t)dm.B * dm.Hkv, cudaMemcpyDeviceToDevice, st));
+  if (rc) return rc;
+
+  rc = hga_build_summaries(p, K_dev, dm.H, dm.L, chunk_sum, group_sum, stream);
+  if (rc) return rc;
+  rc = hga_route(p, dQin, chunk_sum, group_sum, cidx, gidx, ng, nullptr, nullptr, rws,
+                 route_workspace_bytes(dm), stream);
+  if (rc) return rc;
+  rc = hga_attn_fwd(p, dQin, K_dev, V_dev, gidx, ng, dO_, lse, status_word, stream);
+  if (rc) return rc;
+  rc = record_cuda(cudaMemcpyAsync(O_host, dO_, qb, cudaMemcpyDeviceToHost, st));
+  if (rc) return rc;
+  if (!bwd) return HGA_OK;
+  rc = hga_attn_bwd(p, dQin, K_dev, V_dev, dO_, lse, ddO, gidx, ng, ddQ, ddK, ddV, bws,
+                    bwd_workspace_bytes(dm), status_word, stream);
+  if (rc) return rc;
+  rc = record_cuda(cudaMemcpyAsync(dQ_host, ddQ, qb, cudaMemcpyDeviceToHost, st));
+  if (rc) return rc;
+  rc = record_cuda(cudaMemcpyAsync(dK_host, ddK, kv32, cudaMemcpyDeviceToHost, st));
+  if (rc) return rc;
+  return record_cuda(cudaMemcpyAsync(dV_host, ddV, kv32, cudaMemcpyDeviceToHost, st));
+}
+
+}  // extern "C"

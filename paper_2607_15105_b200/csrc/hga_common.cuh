@@ -1,0 +1,75 @@
+// Internal definitions shared by the libhga translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hga.h"
+
+namespace hga {
+
+// Resolved problem description handed to kernels by value.
+struct Dims {
+  int B, Hq, Hkv, G, d;
+  int L, S, H;          // total, active segment, history = L - S
+  int c, g, Bq;         // chunk, group, query block
+  int kc, kg, kge, per; // k_c, k_g, min(k_g, c/g), c/g
+  int sink, local;
+  int NQB, Nc, Ng;      // query blocks per sequence, chunks, groups
+  int width;            // group_idx entries per item = kc * kge
+  int rows;             // G * Bq query rows per item
+  int flags;
+  float scale;          // softmax scale
+  int64_t qs[3], ks[3], vs[3], os[3];  // element strides (batch, head, token)
+};
+
+// Window geometry of a query block (local start, sink end), see hga.h.
+struct Window {
+  int p0, ls, se;
+};
+
+__host__ __device__ inline Window window_of(const Dims& dm, int qb) {
+  Window w;
+  w.p0 = dm.H + qb * dm.Bq;
+  int l = w.p0 - dm.local;
+  w.ls = l <= 0 ? 0 : (l / dm.c) * dm.c;
+  w.se = dm.sink < w.ls ? dm.sink : w.ls;
+  return w;
+}
+
+__host__ __device__ inline void item_coords(const Dims& dm, int item, int& b, int& h, int& qb) {
+  qb = item % dm.NQB;
+  int bh = item / dm.NQB;
+  h = bh % dm.Hkv;
+  b = bh / dm.Hkv;
+}
+
+// Upper bound of routed tokens per item (sink + groups + local window + the block itself).
+__host__ __device__ inline int max_routed_tokens(const Dims& dm) {
+  return dm.sink + dm.width * dm.g + dm.local + dm.Bq + dm.c;
+}
+
+// Launch bookkeeping (hga_api.cu).
+void count_launch(int n = 1);
+int record_cuda(cudaError_t e);  // returns HGA_OK or HGA_ERR_CUDA and remembers the code
+
+// Kernel launchers, one per translation unit.  All return an HGA status.
+int launch_build_summaries(const Dims& dm, const void* K, int tok_begin, int tok_end,
+                           void* chunk_sum, void* group_sum, cudaStream_t st);
+int launch_route_generic(const Dims& dm, const void* Q, const void* chunk_sum,
+                         const void* group_sum, int32_t* chunk_idx, int32_t* group_idx,
+                         int32_t* n_groups, float* chunk_scores, float* group_scores,
+                         void* workspace, cudaStream_t st);
+int launch_attn_fwd_generic(const Dims& dm, const void* Q, const void* K, const void* V,
+                            const int32_t* group_idx, const int32_t* n_groups, void* O, float* LSE,
+                            int32_t* status_word, cudaStream_t st);
+int launch_attn_bwd_generic(const Dims& dm, const void* Q, const void* K, const void* V,
+                            const void* O, const float* LSE, const void* dO,
+                            const int32_t* group_idx, const int32_t* n_groups, void* dQ, float* dK,
+                            float* dV, float* delta_ws, int32_t* status_word, cudaStream_t st);
+
+size_t route_workspace_bytes(const Dims& dm);
+size_t bwd_workspace_bytes(const Dims& dm);
+
+}  // namespace hga

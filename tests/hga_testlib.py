@@ -1,0 +1,92 @@
+"""Helpers shared by the parity tests: moving the seeded inputs to the device and comparing
+the CUDA library's outputs with the CPU oracle's.  No method arithmetic lives here."""
+import numpy as np
+import torch
+
+import oracle
+
+SCORE_GAP = 1e-3   # routing: an index may differ only where the score gap to the k-th is below this
+TOL_O = 1e-2       # attention forward: max abs error on O (unit-scale bf16 inputs)
+TOL_LSE = 1e-3     # attention forward: max abs error on LSE
+TOL_GRAD = 2e-2    # backward: relative Frobenius error per gradient tensor
+
+
+def to_dev(bits: np.ndarray) -> torch.Tensor:
+    """uint16 bf16 bit patterns -> CUDA bfloat16 tensor (same bits)."""
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def bits_of(t: torch.Tensor) -> np.ndarray:
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def bf16_to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def rel_fro(a: np.ndarray, ref: np.ndarray) -> float:
+    den = float(np.linalg.norm(ref.ravel()))
+    num = float(np.linalg.norm((a - ref).ravel()))
+    return num / den if den > 0 else num
+
+
+def check_routing(cfg, ref, chunk_idx, group_idx, n_groups, items=None):
+    """Compare GPU routing with the oracle's (ref holds oracle indices and fp64 scores).
+
+    Index sets must be equal, except that an index in the symmetric difference is excused
+    when its oracle score lies within SCORE_GAP of the oracle's k-th best score; set sizes
+    must match.  Groups are compared inside chunks both sides selected.
+    Returns (items checked, items with an excused chunk, chunks with an excused group).
+    """
+    per, kge = cfg.chunk // cfg.group, min(cfg.topk_groups, cfg.chunk // cfg.group)
+    nqb, Hkv = cfg.n_q_blocks, cfg.n_kv_heads
+    all_items = range(cfg.n_items) if items is None else items
+    exc_c = exc_g = 0
+    for item in all_items:
+        qb = item % nqb
+        h = (item // nqb) % Hkv
+        b = item // (nqb * Hkv)
+        o_c = [int(j) for j in ref["chunk_idx"][b, h, qb] if j >= 0]
+        g_c = [int(j) for j in chunk_idx[b, h, qb] if j >= 0]
+        assert len(o_c) == len(g_c), (item, o_c, g_c)
+        assert g_c == sorted(set(g_c)), ("chunk list not ascending/unique", item, g_c)
+        ls, se = oracle.window(cfg, qb)
+        assert all(se <= j * cfg.chunk and (j + 1) * cfg.chunk <= ls for j in g_c), (item, g_c)
+        sc = ref["chunk_scores"][b, h, qb]
+        if set(o_c) != set(g_c):
+            kth = min(sc[j] for j in o_c)
+            for j in set(o_c) ^ set(g_c):
+                assert abs(sc[j] - kth) < SCORE_GAP, ("chunk not excused", item, j, sc[j], kth)
+            exc_c += 1
+        ng = int(n_groups[b, h, qb])
+        assert ng == len(g_c) * kge, (item, ng)
+        g_g = [int(m) for m in group_idx[b, h, qb, :ng]]
+        assert g_g == sorted(set(g_g)) and np.all(group_idx[b, h, qb, ng:] == -1), (item, g_g)
+        for r, j in enumerate(o_c):
+            if j not in g_c:
+                continue
+            o_set = {int(m) for m in ref["group_idx"][b, h, qb] if m >= 0 and m // per == j}
+            g_set = {m for m in g_g if m // per == j}
+            assert len(g_set) == kge, (item, j, g_set)
+            if o_set != g_set:
+                sg = ref["group_scores"][b, h, qb, r * per:(r + 1) * per]
+                kth = min(sg[m - j * per] for m in o_set)
+                for m in o_set ^ g_set:
+                    assert abs(sg[m - j * per] - kth) < SCORE_GAP, ("group not excused", item, m)
+                exc_g += 1
+    return len(list(all_items)), exc_c, exc_g
+
+
+def item_rows(cfg, items):
+    """(b, hq, s) index arrays of every query row belonging to the listed items."""
+    G, Bq, nqb, Hkv = cfg.gqa, cfg.q_block, cfg.n_q_blocks, cfg.n_kv_heads
+    bs, hs, ss = [], [], []
+    for item in items:
+        qb = item % nqb
+        h = (item // nqb) % Hkv
+        b = item // (nqb * Hkv)
+        for a in range(G):
+            bs.append(np.full(Bq, b))
+            hs.append(np.full(Bq, h * G + a))
+            ss.append(qb * Bq + np.arange(Bq))
+    return np.concatenate(bs), np.concatenate(hs), np.concatenate(ss)

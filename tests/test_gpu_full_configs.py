@@ -1,0 +1,86 @@
+"""The five benchmark configurations at full size, in the launch configuration bench.py times:
+the whole path runs on the GPU; the oracle recomputes sampled items (all query blocks of one
+(batch, kv head) so that its dK/dV rows are complete, plus a few scattered items)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_15105_b200 import binding
+from paper_2607_15105_b200.workloads import CONFIGS, make_inputs
+
+from hga_testlib import (TOL_GRAD, TOL_LSE, TOL_O, bf16_to_f64, bits_of, check_routing, item_rows,
+                         rel_fro, to_dev)
+
+pytestmark = pytest.mark.gpu
+
+
+def sample_items(cfg, full_head, extra, seed):
+    """All items of one (b, h) plus `extra` random others."""
+    nqb = cfg.n_q_blocks
+    b, h = full_head
+    head = [((b * cfg.n_kv_heads + h) * nqb) + qb for qb in range(nqb)]
+    rng = np.random.default_rng(seed)
+    rest = [int(i) for i in rng.choice(cfg.n_items, size=min(extra, cfg.n_items), replace=False)]
+    return head, sorted(set(head) | set(rest))
+
+
+# routed keys per item (a data-independent count) for the last query block of each config
+ROUTED_KEYS_LAST_BLOCK = {1: 320, 2: 512, 3: 768, 4: 768, 5: 2560}
+
+
+@pytest.mark.parametrize("n,full_head,extra", [(1, (0, 0), 4), (2, (0, 5), 12), (3, (0, 3), 12),
+                                               (4, (0, 6), 0), (5, (2, 5), 0)])
+def test_config_against_oracle(n, full_head, extra):
+    cfg = CONFIGS[n]
+    x = make_inputs(cfg)
+    Q, K, V = to_dev(x["Q"]), to_dev(x["K"]), to_dev(x["V"])
+    dO = to_dev(x["dO"]) if cfg.backward else None
+    buf = binding.HgaLayerBuffers(cfg, backward=cfg.backward)
+    # history summaries come from earlier segments; the step itself adds the active range
+    buf.build_summaries(K, 0, cfg.history)
+    buf.step(Q, K, V, dO)
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    head, items = sample_items(cfg, full_head, extra, seed=n)
+    if n == 4:
+        head, items = [], head[::2]          # forward only: 16 items are plenty
+
+    # summaries: bit exact, everywhere
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    assert np.array_equal(bits_of(buf.chunk_sum), cs)
+    assert np.array_equal(bits_of(buf.group_sum), gs)
+
+    # routing on the sampled items
+    ref = oracle.route(cfg, x["Q"], cs, gs, items=items, want_scores=True)
+    gi, ng = buf.group_idx.cpu().numpy(), buf.n_groups.cpu().numpy()
+    checked, ec, eg = check_routing(cfg, ref, buf.chunk_idx.cpu().numpy(), gi, ng, items=items)
+    assert ec <= max(2, checked // 4), (checked, ec, eg)
+    # data-independent counts, everywhere
+    keys = cfg.sink + ng[:, :, -1] * cfg.group + cfg.local + cfg.q_block
+    assert np.all(keys == ROUTED_KEYS_LAST_BLOCK[n])
+
+    # attention on the GPU's own indices (the oracle takes the same lists)
+    O, LSE = oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], gi, ng, items=items)
+    bi, hi, si = item_rows(cfg, items)
+    assert np.max(np.abs(bf16_to_f64(buf.O)[bi, hi, si] - O[bi, hi, si])) <= TOL_O
+    assert np.max(np.abs(buf.LSE.cpu().numpy().astype(np.float64)[bi, hi, si] - LSE[bi, hi, si])) <= TOL_LSE
+    if not cfg.backward:
+        return
+    # dK/dV rows are complete only for the (b, h) whose every query block was recomputed
+    b, h = full_head
+    dQ, dKo, dVo = oracle.attn_bwd(cfg, x["Q"], x["K"], x["V"], x["dO"], gi, ng, items=head)
+    rest = sorted(set(items) - set(head))
+    if rest:
+        dQ += oracle.attn_bwd(cfg, x["Q"], x["K"], x["V"], x["dO"], gi, ng, items=rest)[0]   # disjoint rows
+    assert rel_fro(bf16_to_f64(buf.dQ)[bi, hi, si], dQ[bi, hi, si]) <= TOL_GRAD
+    assert rel_fro(buf.dK[b, h].cpu().numpy().astype(np.float64), dKo[b, h]) <= TOL_GRAD
+    assert rel_fro(buf.dV[b, h].cpu().numpy().astype(np.float64), dVo[b, h]) <= TOL_GRAD
+    # rows of the active segment that no query block routes to get exactly zero
+    H = cfg.history
+    touched = np.zeros(cfg.seg_len, bool)
+    for qb in range(cfg.n_q_blocks):
+        tok = oracle.routed_tokens(cfg, qb, gi[b, h, qb, :ng[b, h, qb]])
+        touched[tok[tok >= H] - H] = True
+    if (~touched).any():
+        assert float(buf.dK[b, h][torch.from_numpy(~touched).cuda()].abs().max()) == 0.0

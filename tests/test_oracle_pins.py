@@ -294,8 +294,9 @@ def _torch_attention_grads(cfg, x, mask_fn):
 
 @pytest.mark.parametrize("hist", [0, 64])
 def test_full_budget_equals_dense_causal_attention(hist):
-    # "dense timing is obtained by disabling the router" (Section 4.2): with a budget that
-    # covers every candidate chunk and every group, HGA is dense causal attention.
+    # Section 4.2 takes its dense timings from the same module with the router switched off:
+    # with a budget that covers every candidate chunk and every group, HGA is dense causal
+    # attention.
     cfg = tiny(n_q_heads=4, n_kv_heads=2, total_len=128 + hist, seg_len=128,
                topk_chunks=(128 + hist) // 8, topk_groups=4)
     x = make_inputs(cfg)
