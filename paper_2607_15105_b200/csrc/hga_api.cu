@@ -132,7 +132,8 @@ int hga_route(const hga_params* p, const void* Q, const void* chunk_sum, const v
   Dims dm;
   int rc = resolve(p, dm);
   if (rc) return rc;
-  if (!Q || !chunk_sum || !group_sum || !chunk_idx || !group_idx || !n_groups) return HGA_ERR_NULL;
+  if (!Q || !chunk_sum || !group_sum || !n_groups) return HGA_ERR_NULL;
+  if (dm.kc > 0 && (!chunk_idx || !group_idx)) return HGA_ERR_NULL;   // zero-width lists may be NULL
   if (!aligned16(Q) || !aligned16(chunk_sum) || !aligned16(group_sum)) return HGA_ERR_ALIGN;
   if (!workspace || workspace_bytes < route_workspace_bytes(dm)) return HGA_ERR_WORKSPACE;
   if (!aligned16(workspace)) return HGA_ERR_ALIGN;
@@ -146,8 +147,12 @@ int hga_attn_fwd(const hga_params* p, const void* Q, const void* K, const void* 
   Dims dm;
   int rc = resolve(p, dm);
   if (rc) return rc;
-  if (!Q || !K || !V || !group_idx || !n_groups || !O || !LSE) return HGA_ERR_NULL;
+  if (!Q || !K || !V || (!group_idx && dm.width > 0) || !n_groups || !O || !LSE) return HGA_ERR_NULL;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return HGA_ERR_ALIGN;
+  if (attn_fwd_sm100_supported(dm)) {
+    rc = launch_attn_fwd_sm100(dm, Q, K, V, group_idx, n_groups, O, LSE, status_word, (cudaStream_t)stream);
+    if (rc != HGA_ERR_UNSUPPORTED) return rc;
+  }
   return launch_attn_fwd_generic(dm, Q, K, V, group_idx, n_groups, O, LSE, status_word,
                                  (cudaStream_t)stream);
 }
@@ -159,7 +164,7 @@ int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* 
   Dims dm;
   int rc = resolve(p, dm);
   if (rc) return rc;
-  if (!Q || !K || !V || !O || !LSE || !dO || !group_idx || !n_groups || !dQ || !dK || !dV)
+  if (!Q || !K || !V || !O || !LSE || !dO || (!group_idx && dm.width > 0) || !n_groups || !dQ || !dK || !dV)
     return HGA_ERR_NULL;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) ||
       !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
@@ -226,7 +231,7 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   size_t kv32 = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 4;
   size_t kvseg = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 2;
   size_t items = (size_t)dm.B * dm.Hkv * dm.NQB;
-  void* dQin = take(qb); void* ddO = take(qb); void* dO_ = take(qb); void* ddQ = take(qb);
+  void* dQin = take(qb); void* ddO = take(qb); void* dOut = take(qb); void* ddQ = take(qb);
   float* ddK = (float*)take(kv32); float* ddV = (float*)take(kv32);
   void* kseg = take(kvseg); void* vseg = take(kvseg);
   int32_t* cidx = (int32_t*)take(items * (dm.kc + dm.width + 1) * 4 + 64);
@@ -262,12 +267,12 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   rc = hga_route(p, dQin, chunk_sum, group_sum, cidx, gidx, ng, nullptr, nullptr, rws,
                  route_workspace_bytes(dm), stream);
   if (rc) return rc;
-  rc = hga_attn_fwd(p, dQin, K_dev, V_dev, gidx, ng, dO_, lse, status_word, stream);
+  rc = hga_attn_fwd(p, dQin, K_dev, V_dev, gidx, ng, dOut, lse, status_word, stream);
   if (rc) return rc;
-  rc = record_cuda(cudaMemcpyAsync(O_host, dO_, qb, cudaMemcpyDeviceToHost, st));
+  rc = record_cuda(cudaMemcpyAsync(O_host, dOut, qb, cudaMemcpyDeviceToHost, st));
   if (rc) return rc;
   if (!bwd) return HGA_OK;
-  rc = hga_attn_bwd(p, dQin, K_dev, V_dev, dO_, lse, ddO, gidx, ng, ddQ, ddK, ddV, bws,
+  rc = hga_attn_bwd(p, dQin, K_dev, V_dev, dOut, lse, ddO, gidx, ng, ddQ, ddK, ddV, bws,
                     bwd_workspace_bytes(dm), status_word, stream);
   if (rc) return rc;
   rc = record_cuda(cudaMemcpyAsync(dQ_host, ddQ, qb, cudaMemcpyDeviceToHost, st));

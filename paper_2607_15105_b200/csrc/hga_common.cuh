@@ -69,6 +69,12 @@ int launch_attn_bwd_generic(const Dims& dm, const void* Q, const void* K, const 
                             const int32_t* group_idx, const int32_t* n_groups, void* dQ, float* dK,
                             float* dV, float* delta_ws, int32_t* status_word, cudaStream_t st);
 
+// tensor-core (tcgen05 / TMEM / TMA) kernels; *_supported says whether the shape qualifies
+bool attn_fwd_sm100_supported(const Dims& dm);
+int launch_attn_fwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V,
+                          const int32_t* group_idx, const int32_t* n_groups, void* O, float* LSE,
+                          int32_t* status_word, cudaStream_t st);
+
 size_t route_workspace_bytes(const Dims& dm);
 size_t bwd_workspace_bytes(const Dims& dm);
 
