@@ -1,0 +1,428 @@
+// hga_attn_bwd for sm_100a (head_dim 128): backward of routed exact-token attention with the
+// routing frozen (Section 2.1, last paragraph) and history K/V detached (Section 2.2).
+//
+// Work unit (one CTA): one 128-row M-tile of one item, swept over the item's routed keys in
+// 64-key tiles (8 octets, gathered by TMA exactly as in the forward kernel).  Per tile:
+//   S  = Q K^T          (smem x smem)  -> TMEM          dP = dO V^T     (smem x smem) -> TMEM
+//   P  = 2^(S*c - LSE*log2e),  dS = scale * P o (dP - delta)            (one thread per row)
+//   dQ += dS K          (dS K-major from smem, K tile MN-major)          -> TMEM, kept for all tiles
+//   and, only for tiles that hold keys of the active segment (position >= H):
+//   dV^T = dO^T P,  dK^T = Q^T dS   (M = head_dim, N = 64 keys, K = 128 rows) -> TMEM
+// dK^T/dV^T are produced transposed so that a reduction warp's 32 lanes hold 32 consecutive
+// elements of one key row: its red.global.add.f32 is one coalesced 128-byte request.  History
+// tiles skip two of the five GEMMs and all atomics.
+//
+// Warp roles (320 threads): warp 0 producer (TMA), warp 1 MMA issuer, warps 2-5 one thread
+// per query row (delta, P, dS, dQ epilogue), warps 6-9 dK/dV reduction (thread = head_dim lane).
+// TMEM (512 columns): S[2] dP[2] (64 each, double buffered) | dQ 128 | dV^T 64 | dK^T 64.
+// Shared memory: Q, dO (32 KB each), 3-stage K/V ring (16 + 16 KB per stage), P, dS (16 KB each).
+#include "hga_common.cuh"
+#include "hga_sm100.cuh"
+
+namespace hga {
+
+using namespace sm100;
+
+constexpr int kBwdThreads = 320;
+constexpr int kBwdStages = 3;
+constexpr int kBwdD = 128;
+constexpr int kKT = 64;                         // keys per tile
+constexpr int kOct = 8 * kBwdD * 2;             // bytes of one octet of K/V/Q/dO rows (2 panels)
+
+struct BwdSmem {
+  alignas(1024) uint8_t q[128 * kBwdD * 2];
+  alignas(1024) uint8_t dO[128 * kBwdD * 2];
+  alignas(1024) uint8_t k[kBwdStages][kKT * kBwdD * 2];
+  alignas(1024) uint8_t v[kBwdStages][kKT * kBwdD * 2];
+  alignas(1024) uint8_t p[128 * kKT * 2];       // [16 row octets][8 rows][128 B], 128-byte swizzle
+  alignas(1024) uint8_t ds[128 * kKT * 2];
+  uint64_t q_full, kv_full[kBwdStages], kv_empty[kBwdStages];
+  uint64_t sdp_full[2], sdp_free[2], pds_full, pds_free, dkv_full, dkv_free, dq_done;
+  uint32_t tmem_base;
+  int n_oct, first_active;
+  volatile int abort;
+  int oct_row[1];
+};
+
+__device__ __forceinline__ bool bwd_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+  for (uint32_t i = 0; i < (1u << 20); ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 255u && *abort) return false;
+  }
+  *abort = 1;
+  return false;
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+__global__ void __launch_bounds__(kBwdThreads, 1)
+k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
+                 const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                 const uint16_t* __restrict__ O, const uint16_t* __restrict__ dOg,
+                 const float* __restrict__ LSE, const int32_t* __restrict__ group_idx,
+                 const int32_t* __restrict__ n_groups, Dims dm, uint16_t* __restrict__ dQ,
+                 float* __restrict__ dK, float* __restrict__ dV, int32_t* status_word) {
+  constexpr int D = kBwdD;
+  constexpr uint32_t kColSdP = 0;       // S[b] at 128*b, dP[b] at 128*b + 64
+  constexpr uint32_t kColDQ = 256, kColDV = 384, kColDK = 448;
+  extern __shared__ uint8_t smem_raw[];
+  BwdSmem& sm = *reinterpret_cast<BwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_mt_item = dm.rows / 128;
+  const int item = blockIdx.x / n_mt_item;
+  const int mt = blockIdx.x % n_mt_item;
+  int b, h, qb;
+  item_coords(dm, item, b, h, qb);
+  const Window w = window_of(dm, qb);
+
+  if (tid == 0) {
+    mbar_init(&sm.q_full, 1);
+    for (int s = 0; s < kBwdStages; ++s) { mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&sm.sdp_full[s], 1); mbar_init(&sm.sdp_free[s], 128); }
+    mbar_init(&sm.pds_full, 128); mbar_init(&sm.pds_free, 1);
+    mbar_init(&sm.dkv_full, 1); mbar_init(&sm.dkv_free, 128);
+    mbar_init(&sm.dq_done, 1);
+    sm.abort = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&sm.tmem_base, 512);
+    tmem_relinquish();
+  }
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tensormap(&map_q); prefetch_tensormap(&map_do);
+      prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
+      const int32_t* gi = group_idx + (int64_t)item * dm.width;
+      int ng = n_groups[item], n = w.se / 8, prev = -1;
+      if (ng > dm.width) ng = dm.width;
+      if (ng < 0) ng = 0;
+      const int opg = dm.g / 8;
+      for (int i = 0; i < ng; ++i) {      // invalid entries are skipped, as in the forward kernel
+        const int m = gi[i];
+        if (m > prev && (int64_t)m * dm.g >= w.se && ((int64_t)m + 1) * dm.g <= w.ls) {
+          for (int u = 0; u < opg; ++u) sm.oct_row[n++] = m * dm.g + 8 * u;
+          prev = m;
+        }
+      }
+      sm.n_oct = n;
+    }
+    __syncwarp();
+    const int n_far = sm.n_oct;
+    for (int o = lane; o < w.se / 8; o += 32) sm.oct_row[o] = 8 * o;
+    const int n_local = (w.p0 + dm.Bq - w.ls) / 8;
+    for (int o = lane; o < n_local; o += 32) sm.oct_row[n_far + o] = w.ls + 8 * o;
+    __syncwarp();
+    if (lane == 0) {
+      const int n_oct = n_far + n_local;
+      sm.n_oct = n_oct;
+      // rows ascend, so the tiles holding active keys (position >= H) are a suffix
+      const int n_tiles = (n_oct + 7) / 8;
+      int fa = n_tiles;
+      for (int j = n_tiles - 1; j >= 0; --j) {
+        const int last = 8 * j + 7 < n_oct ? 8 * j + 7 : n_oct - 1;
+        if (sm.oct_row[last] + 8 > dm.H) fa = j; else break;
+      }
+      sm.first_active = fa;
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+
+  const uint32_t tmem = sm.tmem_base;
+  const int n_oct = sm.n_oct;
+  const int n_keys = n_oct * 8;
+  const int n_tiles = (n_oct + 7) / 8;
+  const int first_active = sm.first_active;
+  volatile int* abort = &sm.abort;
+  constexpr uint32_t kStageBytes = 2 * kKT * D * 2;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) mbar_arrive_expect_tx(&sm.q_full, 2 * 128 * D * 2);
+    __syncwarp();
+    {
+      const int o = lane & 15;
+      const int r = mt * 128 + 8 * o;
+      const int a = r / dm.Bq, t = r % dm.Bq;
+      if (lane < 16) tma_load_5d(sm.q + o * kOct, &map_q, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
+      else tma_load_5d(sm.dO + o * kOct, &map_do, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
+    }
+    bool ok = true;
+    int issued = 0;
+    for (int j = 0; j < n_tiles; ++j) {
+      const int s = j % kBwdStages, use = j / kBwdStages;
+      if (lane == 0 && use > 0) ok = bwd_wait(&sm.kv_empty[s], (use - 1) & 1, abort);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane == 0) mbar_arrive_expect_tx(&sm.kv_full[s], kStageBytes);
+      __syncwarp();
+      const int o = 8 * j + (lane & 7);
+      const int row = o < n_oct ? sm.oct_row[o] : dm.L;    // past the list: zeros
+      if (lane < 8) tma_load_5d(sm.k[s] + lane * kOct, &map_k, &sm.kv_full[s], 0, row, 0, h, b);
+      else if (lane < 16) tma_load_5d(sm.v[s] + (lane - 8) * kOct, &map_v, &sm.kv_full[s], 0, row, 0, h, b);
+      issued = j + 1;
+    }
+    if (*abort && lane == 0) {
+      mbar_wait(&sm.q_full, 0);
+      for (int j = issued > kBwdStages ? issued - kBwdStages : 0; j < issued; ++j)
+        mbar_wait(&sm.kv_full[j % kBwdStages], (j / kBwdStages) & 1);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_sdp = idesc_bf16_f32(128, kKT, 0, 0);   // rows x keys, both K-major
+      constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);      // dS K-major, K tile MN-major
+      constexpr uint32_t idesc_dkv = idesc_bf16_f32(D, kKT, 1, 1);     // both MN-major
+      const uint32_t qa = smem_u32(sm.q), doa = smem_u32(sm.dO), pa = smem_u32(sm.p), dsa = smem_u32(sm.ds);
+      auto issue_sdp = [&](int j) {
+        const int st = j % kBwdStages, buf = j & 1;
+        const uint32_t ka = smem_u32(sm.k[st]), va = smem_u32(sm.v[st]);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
+          mma_ss(tmem + kColSdP + buf * 128, smem_desc_sw128(qa + off, 16, kOct),
+                 smem_desc_sw128(ka + off, 16, kOct), idesc_sdp, kk > 0);
+        }
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
+          mma_ss(tmem + kColSdP + buf * 128 + 64, smem_desc_sw128(doa + off, 16, kOct),
+                 smem_desc_sw128(va + off, 16, kOct), idesc_sdp, kk > 0);
+        }
+        mma_commit(&sm.sdp_full[buf]);
+      };
+      bool ok = bwd_wait(&sm.q_full, 0, abort) && bwd_wait(&sm.kv_full[0], 0, abort);
+      if (ok) {
+        tc_fence_after_sync();
+        issue_sdp(0);
+      }
+      int n_active_done = 0;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int st = j % kBwdStages;
+        if (j + 1 < n_tiles) {
+          ok = bwd_wait(&sm.kv_full[(j + 1) % kBwdStages], ((j + 1) / kBwdStages) & 1, abort);
+          // buffer (j+1)&1 held tile j-1: its rows have been read once sdp_free completed
+          if (ok && j >= 1) ok = bwd_wait(&sm.sdp_free[(j + 1) & 1], ((j - 1) >> 1) & 1, abort);
+          if (!ok) break;
+          tc_fence_after_sync();
+          issue_sdp(j + 1);
+        }
+        ok = bwd_wait(&sm.pds_full, j & 1, abort);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t ka = smem_u32(sm.k[st]);
+#pragma unroll
+        for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per step
+          mma_ss(tmem + kColDQ, smem_desc_sw128(dsa + kk * 32, 16, 1024),
+                 smem_desc_sw128(ka + kk * 2 * kOct, 1024, kOct), idesc_dq, (j > 0 || kk > 0));
+        if (j >= first_active) {
+          if (n_active_done > 0) {
+            ok = bwd_wait(&sm.dkv_free, (n_active_done - 1) & 1, abort);
+            if (!ok) break;
+            tc_fence_after_sync();
+          }
+#pragma unroll
+          for (int kk = 0; kk < 128 / 16; ++kk) {   // 16 query rows per step (2 row octets)
+            mma_ss(tmem + kColDV, smem_desc_sw128(doa + kk * 2 * kOct, 1024, kOct),
+                   smem_desc_sw128(pa + kk * 2048, 16, 1024), idesc_dkv, kk > 0);
+          }
+#pragma unroll
+          for (int kk = 0; kk < 128 / 16; ++kk) {
+            mma_ss(tmem + kColDK, smem_desc_sw128(qa + kk * 2 * kOct, 1024, kOct),
+                   smem_desc_sw128(dsa + kk * 2048, 16, 1024), idesc_dkv, kk > 0);
+          }
+          mma_commit(&sm.dkv_full);
+          ++n_active_done;
+        }
+        mma_commit(&sm.pds_free);
+        mma_commit(&sm.kv_empty[st]);
+      }
+      if (ok) mma_commit(&sm.dq_done);
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ one thread per query row
+    const int quarter = warp & 3;
+    const int row_in_tile = quarter * 32 + lane;
+    const int r = mt * 128 + row_in_tile;
+    const int a = r / dm.Bq, t = r % dm.Bq;
+    const int hq = h * dm.G + a, srow = qb * dm.Bq + t;
+    const int limit = n_keys - dm.Bq + t + 1;
+    const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+    const float sl2 = dm.scale * 1.4426950408889634f;
+    // delta = rowsum(dO o O); LSE in log2 units
+    float delta = 0.f;
+    {
+      const uint4* o4 = reinterpret_cast<const uint4*>(O + b * dm.os[0] + hq * dm.os[1] + (int64_t)srow * dm.os[2]);
+      const uint4* g4 = reinterpret_cast<const uint4*>(dOg + b * dm.os[0] + hq * dm.os[1] + (int64_t)srow * dm.os[2]);
+#pragma unroll 4
+      for (int i = 0; i < D / 8; ++i) {
+        const uint4 x = o4[i], y = g4[i];
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          delta = fmaf(__uint_as_float(xs[e] << 16), __uint_as_float(ys[e] << 16), delta);
+          delta = fmaf(__uint_as_float(xs[e] & 0xffff0000u), __uint_as_float(ys[e] & 0xffff0000u), delta);
+        }
+      }
+    }
+    const float neg_lse2 = -LSE[((int64_t)b * dm.Hq + hq) * dm.S + srow] * 1.4426950408889634f;
+    const float neg_delta_s = -delta * dm.scale;
+    // this row's 128-byte line inside the P / dS buffers, and its swizzle key
+    const uint32_t line = (uint32_t)(row_in_tile >> 3) * 1024 + (uint32_t)(row_in_tile & 7) * 128;
+    const uint32_t key = (uint32_t)(row_in_tile & 7);
+    const uint32_t p_line = smem_u32(sm.p) + line, ds_line = smem_u32(sm.ds) + line;
+    bool ok = true;
+    for (int j = 0; j < n_tiles; ++j) {
+      const int buf = j & 1;
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[buf], (j >> 1) & 1, abort));
+      if (!ok) break;
+      tc_fence_after_sync();
+      const int vis = limit - kKT * j;
+      uint32_t pk[32], dk[32];
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t s[32], dp[32];
+        tmem_ld32(lane_base + kColSdP + buf * 128 + half * 32, s);
+        tmem_ld32(lane_base + kColSdP + buf * 128 + 64 + half * 32, dp);
+        tmem_wait_ld();
+        if (half == 1) {
+          // both halves are in registers: the MMA warp may overwrite this S/dP buffer
+          tc_fence_before_sync();
+          mbar_arrive(&sm.sdp_free[buf]);
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), sl2, neg_lse2));
+          float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), sl2, neg_lse2));
+          if (half * 32 + 2 * i >= vis) p0 = 0.f;
+          if (half * 32 + 2 * i + 1 >= vis) p1 = 0.f;
+          const float d0 = p0 * fmaf(__uint_as_float(dp[2 * i]), dm.scale, neg_delta_s);
+          const float d1 = p1 * fmaf(__uint_as_float(dp[2 * i + 1]), dm.scale, neg_delta_s);
+          pk[half * 16 + i] = pack_bf16(p0, p1);
+          dk[half * 16 + i] = pack_bf16(d0, d1);
+        }
+      }
+      if (j > 0) {
+        ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_free, (j - 1) & 1, abort));
+        if (!ok) break;
+      }
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {    // 8 chunks of 16 bytes (8 keys) per row, XOR-swizzled
+        const uint32_t off = ((uint32_t)c ^ key) * 16;
+        st_shared_v4(p_line + off, pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        st_shared_v4(ds_line + off, dk[4 * c], dk[4 * c + 1], dk[4 * c + 2], dk[4 * c + 3]);
+      }
+      fence_proxy_async_smem();
+      mbar_arrive(&sm.pds_full);
+    }
+    if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.dq_done, 0, abort));
+    if (ok) {
+      tc_fence_after_sync();
+      uint16_t* qrow = dQ + b * dm.qs[0] + hq * dm.qs[1] + (int64_t)srow * dm.qs[2];
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t x[32];
+        tmem_ld32(lane_base + kColDQ + c * 32, x);
+        tmem_wait_ld();
+        uint4* dst = reinterpret_cast<uint4*>(qrow + c * 32);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          dst[i] = make_uint4(pack_bf16(__uint_as_float(x[8 * i]), __uint_as_float(x[8 * i + 1])),
+                              pack_bf16(__uint_as_float(x[8 * i + 2]), __uint_as_float(x[8 * i + 3])),
+                              pack_bf16(__uint_as_float(x[8 * i + 4]), __uint_as_float(x[8 * i + 5])),
+                              pack_bf16(__uint_as_float(x[8 * i + 6]), __uint_as_float(x[8 * i + 7])));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ dK / dV reduction
+    const int quarter = warp & 3;
+    const int e = quarter * 32 + lane;                       // head_dim element = TMEM lane
+    const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+    float* dKb = dK + ((int64_t)(b * dm.Hkv + h) * dm.S) * D + e;
+    float* dVb = dV + ((int64_t)(b * dm.Hkv + h) * dm.S) * D + e;
+    bool ok = true;
+    for (int j = first_active, n = 0; j < n_tiles; ++j, ++n) {
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.dkv_full, n & 1, abort));
+      if (!ok) break;
+      tc_fence_after_sync();
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t gv[32], gk[32];
+        tmem_ld32(lane_base + kColDV + half * 32, gv);
+        tmem_ld32(lane_base + kColDK + half * 32, gk);
+        tmem_wait_ld();
+        if (half == 1) {
+          tc_fence_before_sync();
+          mbar_arrive(&sm.dkv_free);
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int o = 8 * j + half * 4 + (i >> 3);
+          if (o < n_oct) {
+            const int pos = sm.oct_row[o] + (i & 7);
+            if (pos >= dm.H) {            // warp-uniform: active-segment key
+              atomicAdd(dVb + (int64_t)(pos - dm.H) * D, __uint_as_float(gv[i]));
+              atomicAdd(dKb + (int64_t)(pos - dm.H) * D, __uint_as_float(gk[i]));
+            }
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (tid == 0 && sm.abort && status_word) atomicOr(status_word, HGA_STATUS_WAIT_TIMEOUT);
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+bool attn_bwd_sm100_supported(const Dims& dm) {
+  if (dm.flags & HGA_FLAG_GENERIC_KERNELS) return false;
+  return dm.d == 128 && dm.rows % 128 == 0 && dm.g % 8 == 0;
+}
+
+int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
+                          const float* LSE, const void* dO, const int32_t* group_idx,
+                          const int32_t* n_groups, void* dQ, float* dK, float* dV,
+                          int32_t* status_word, cudaStream_t st) {
+  constexpr int D = kBwdD;
+  CUtensorMap mq, mdo, mk, mv;
+  const uint32_t box[5] = {64, 8, 2, 1, 1};
+  const uint64_t dq[5] = {64, (uint64_t)dm.S, 2, (uint64_t)dm.Hq, (uint64_t)dm.B};
+  const uint64_t dk[5] = {64, (uint64_t)dm.L, 2, (uint64_t)dm.Hkv, (uint64_t)dm.B};
+  const uint64_t sq[4] = {(uint64_t)dm.qs[2] * 2, 128, (uint64_t)dm.qs[1] * 2, (uint64_t)dm.qs[0] * 2};
+  const uint64_t so[4] = {(uint64_t)dm.os[2] * 2, 128, (uint64_t)dm.os[1] * 2, (uint64_t)dm.os[0] * 2};
+  const uint64_t sk[4] = {(uint64_t)dm.ks[2] * 2, 128, (uint64_t)dm.ks[1] * 2, (uint64_t)dm.ks[0] * 2};
+  const uint64_t sv[4] = {(uint64_t)dm.vs[2] * 2, 128, (uint64_t)dm.vs[1] * 2, (uint64_t)dm.vs[0] * 2};
+  if (encode_tensor_map_bf16(&mq, Q, 5, dq, sq, box, true) ||
+      encode_tensor_map_bf16(&mdo, dO, 5, dq, so, box, true) ||
+      encode_tensor_map_bf16(&mk, K, 5, dk, sk, box, true) ||
+      encode_tensor_map_bf16(&mv, V, 5, dk, sv, box, true))
+    return HGA_ERR_UNSUPPORTED;
+  const size_t smem = sizeof(BwdSmem) + sizeof(int) * (max_routed_tokens(dm) / 8 + 8) + 1024;
+  if (smem > 227 * 1024) return HGA_ERR_UNSUPPORTED;
+  cudaError_t e = cudaFuncSetAttribute(k_attn_bwd_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return record_cuda(e);
+  const int units = dm.B * dm.Hkv * dm.NQB * (dm.rows / 128);
+  k_attn_bwd_sm100<<<units, kBwdThreads, smem, st>>>(mq, mdo, mk, mv, (const uint16_t*)O, (const uint16_t*)dO,
+                                                    LSE, group_idx, n_groups, dm, (uint16_t*)dQ, dK, dV,
+                                                    status_word);
+  count_launch();
+  (void)D;
+  return record_cuda(cudaGetLastError());
+}
+
+}  // namespace hga

@@ -75,6 +75,12 @@ int launch_attn_fwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
                           const int32_t* group_idx, const int32_t* n_groups, void* O, float* LSE,
                           int32_t* status_word, cudaStream_t st);
 
+bool attn_bwd_sm100_supported(const Dims& dm);
+int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
+                          const float* LSE, const void* dO, const int32_t* group_idx,
+                          const int32_t* n_groups, void* dQ, float* dK, float* dV,
+                          int32_t* status_word, cudaStream_t st);
+
 size_t route_workspace_bytes(const Dims& dm);
 size_t bwd_workspace_bytes(const Dims& dm);
 
