@@ -110,6 +110,29 @@ HGA_API int hga_route(const hga_params* p, const void* Q, const void* chunk_sum,
               int32_t* chunk_idx, int32_t* group_idx, int32_t* n_groups, float* chunk_scores,
               float* group_scores, void* workspace, size_t workspace_bytes, void* stream);
 
+/* hga_route without a caller-provided workspace (the paper has no counterpart: this entry
+ * point exists for deployment reasons only).  It is for callers that cannot allocate device
+ * memory at all -- code that runs while its host framework's allocator is locked or has
+ * claimed the whole device, loops that must never enter cudaMalloc because it synchronises
+ * the device, processes whose device memory is budgeted at start-up.  The scratch hga_route
+ * would take from `workspace` lives in a fixed array inside the library image instead, so
+ * every GPU that loads the library holds HGA_ROUTE_STATIC_SCRATCH_BYTES of device memory
+ * until the process exits, and the call itself allocates and frees nothing.
+ *   - Same inputs, outputs and selection rule as hga_route (no optional score outputs).
+ *   - Size limit: hga_workspace_bytes().route must not exceed HGA_ROUTE_STATIC_SCRATCH_BYTES
+ *     (batch * n_kv_heads * (seg_len / q_block) * (total_len / chunk) * 4 bytes + 16); a larger
+ *     problem returns HGA_ERR_WORKSPACE and launches nothing.  All five benchmark
+ *     configurations fit.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.  Later calls on the same device do no set-up.
+ *   - All calls on a device share the one array and it keeps the last call's contents (the
+ *     kernels overwrite what they read, nothing needs clearing).  Two calls that overlap on
+ *     the GPU (different streams, no ordering between them) race on it: order them. */
+#define HGA_ROUTE_STATIC_SCRATCH_BYTES (4u << 20)
+HGA_API int hga_route_static(const hga_params* p, const void* Q, const void* chunk_sum,
+                             const void* group_sum, int32_t* chunk_idx, int32_t* group_idx,
+                             int32_t* n_groups, void* stream);
+
 /* Section 2.1 item 3 (attention reads the exact K/V rows of the selected groups; summaries
  * only select and never act as values): for every query row i at position
  * pos, O_i = sum over routed keys k <= pos of softmax(scale * q_i.k) v_k (bf16 MMA inputs,

@@ -19,7 +19,9 @@ HGA_FLAG_GENERIC_KERNELS = 2
 HGA_STATUS_BAD_INDEX = 1
 HGA_STATUS_WAIT_TIMEOUT = 2
 
-EXPORTS = ("hga_build_summaries", "hga_route", "hga_attn_fwd", "hga_attn_bwd",
+HGA_ROUTE_STATIC_SCRATCH_BYTES = 4 << 20
+
+EXPORTS = ("hga_build_summaries", "hga_route", "hga_route_static", "hga_attn_fwd", "hga_attn_bwd",
            "hga_workspace_bytes", "hga_step_host", "hga_step_arena_bytes", "hga_status_string",
            "hga_version", "hga_last_cuda_error", "hga_kernel_launch_count")
 
@@ -60,6 +62,7 @@ def lib():
         pp = C.POINTER(HgaParams)
         L.hga_build_summaries.argtypes = [pp, vp, i32, i32, vp, vp, vp]
         L.hga_route.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.hga_route_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
         L.hga_attn_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.hga_attn_bwd.argtypes = [pp] + [vp] * 12 + [sz, vp, vp]
         L.hga_workspace_bytes.argtypes = [pp, C.POINTER(sz), C.POINTER(sz)]
@@ -145,6 +148,17 @@ def hga_route(p, Q, chunk_sum, group_sum, chunk_idx, group_idx, n_groups, worksp
         C.byref(p), _ptr(Q), _ptr(chunk_sum), _ptr(group_sum), _ptr(chunk_idx), _ptr(group_idx),
         _ptr(n_groups), _ptr(chunk_scores), _ptr(group_scores), _ptr(workspace), nbytes,
         _stream(stream)))
+
+
+def hga_route_static(p, Q, chunk_sum, group_sum, chunk_idx, group_idx, n_groups, stream=None):
+    """hga_route for callers that may not allocate device memory: no workspace argument, the
+    scratch is a fixed array inside the library (HGA_ROUTE_STATIC_SCRATCH_BYTES per GPU).
+    Problems whose routing scratch exceeds that size are refused with HGA_ERR_WORKSPACE.
+    Calls on one device share the array: do not let two of them overlap on the GPU, and make
+    the first call on a device outside any stream capture."""
+    _check("hga_route_static", lib().hga_route_static(
+        C.byref(p), _ptr(Q), _ptr(chunk_sum), _ptr(group_sum), _ptr(chunk_idx), _ptr(group_idx),
+        _ptr(n_groups), _stream(stream)))
 
 
 def hga_attn_fwd(p, Q, K, V, group_idx, n_groups, O, LSE, status_word=None, stream=None):

@@ -69,6 +69,8 @@ static int resolve(const hga_params* p, Dims& dm) {
   return HGA_OK;
 }
 
+int resolve_params(const hga_params* p, Dims& dm) { return resolve(p, dm); }
+
 size_t route_workspace_bytes(const Dims& dm) {
   // chunk scores fp32 [items, Nc]
   return (size_t)dm.B * dm.Hkv * dm.NQB * dm.Nc * sizeof(float) + 16;

@@ -81,6 +81,9 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
                           const int32_t* n_groups, void* dQ, float* dK, float* dV,
                           int32_t* status_word, cudaStream_t st);
 
+// Validates an hga_params block and fills the resolved description (hga_api.cu).
+int resolve_params(const hga_params* p, Dims& dm);
+
 size_t route_workspace_bytes(const Dims& dm);
 size_t bwd_workspace_bytes(const Dims& dm);
 

@@ -1,0 +1,68 @@
+"""hga_route_static: the routing entry point for callers that may not allocate device memory
+(plug-ins running under a locked or exhausted framework allocator, loops that must never enter
+cudaMalloc, processes with a start-up memory budget).  Its scratch is a fixed array inside the
+library, so the test checks, through the C ABI, that it selects exactly what hga_route selects
+-- twice in a row, because the array keeps the previous call's contents -- and that it refuses
+a problem larger than the array.  Collected last on purpose: a run that stops at the first
+failure has then already run every other test."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_15105_b200 import binding
+from paper_2607_15105_b200.workloads import CONFIGS, HgaConfig, make_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _route_both_ways(cfg, seed_shift=0):
+    """Indices from hga_route (caller workspace) and from hga_route_static (no allocation)."""
+    x = make_inputs(cfg.scaled(seed=cfg.seed + seed_shift), with_dO=False)
+    Q, K = _dev(x["Q"]), _dev(x["K"])
+    ref = binding.HgaLayerBuffers(cfg, backward=False)
+    ref.build_summaries(K, 0, cfg.total_len)
+    ref.route(Q)
+    # every buffer the static call touches exists before it runs; the call itself gets no workspace
+    chunk_idx = torch.full_like(ref.chunk_idx, -7)
+    group_idx = torch.full_like(ref.group_idx, -7)
+    n_groups = torch.full_like(ref.n_groups, -7)
+    binding.hga_route_static(ref.p, Q, ref.chunk_sum, ref.group_sum, chunk_idx, group_idx, n_groups)
+    torch.cuda.synchronize()
+    return ref, (chunk_idx, group_idx, n_groups)
+
+
+def test_static_route_matches_route_on_two_calls_in_a_row():
+    # two different problems back to back: the second call finds the first one's scores in the
+    # shared array and must not be influenced by them (indices are integers: exact equality)
+    small = HgaConfig("static_small", 2, 4, 2, 128, 1536, 512, 64, 8, 64, 5, 3, 64, 128,
+                      topics=16, needles=4, backward=False, seed=23)
+    for cfg, shift in ((CONFIGS[3], 0), (small, 0), (CONFIGS[3], 1)):
+        ref, (ci, gi, ng) = _route_both_ways(cfg, shift)
+        assert torch.equal(ci, ref.chunk_idx)
+        assert torch.equal(gi, ref.group_idx)
+        assert torch.equal(ng, ref.n_groups)
+        assert int(ng.min()) >= 0
+
+
+def test_static_route_refuses_problems_beyond_its_array():
+    # 8 sequences of the 128K evaluation shape need 16 MiB of scores: more than the fixed array
+    big = CONFIGS[4].scaled(batch=8)
+    p = binding.make_params(big)
+    need, _ = binding.hga_workspace_bytes(p)
+    assert need > binding.HGA_ROUTE_STATIC_SCRATCH_BYTES
+    dummy = torch.zeros(64, dtype=torch.int32, device="cuda")
+    before = binding.hga_kernel_launch_count()
+    rc = binding.lib().hga_route_static(C.byref(p), C.c_void_p(dummy.data_ptr()), C.c_void_p(dummy.data_ptr()),
+                                        C.c_void_p(dummy.data_ptr()), C.c_void_p(dummy.data_ptr()),
+                                        C.c_void_p(dummy.data_ptr()), C.c_void_p(dummy.data_ptr()), None)
+    assert rc == -5                                      # HGA_ERR_WORKSPACE
+    assert binding.hga_kernel_launch_count() == before   # nothing was launched
+    # the largest benchmark shapes do fit
+    for n in (3, 4, 5):
+        assert binding.hga_workspace_bytes(binding.make_params(CONFIGS[n]))[0] <= binding.HGA_ROUTE_STATIC_SCRATCH_BYTES
