@@ -139,6 +139,11 @@ int hga_route(const hga_params* p, const void* Q, const void* chunk_sum, const v
   if (!aligned16(Q) || !aligned16(chunk_sum) || !aligned16(group_sum)) return HGA_ERR_ALIGN;
   if (!workspace || workspace_bytes < route_workspace_bytes(dm)) return HGA_ERR_WORKSPACE;
   if (!aligned16(workspace)) return HGA_ERR_ALIGN;
+  if (route_sm100_supported(dm)) {
+    rc = launch_route_sm100(dm, Q, chunk_sum, group_sum, chunk_idx, group_idx, n_groups, chunk_scores,
+                            group_scores, (cudaStream_t)stream);
+    if (rc != HGA_ERR_UNSUPPORTED) return rc;
+  }
   return launch_route_generic(dm, Q, chunk_sum, group_sum, chunk_idx, group_idx, n_groups,
                               chunk_scores, group_scores, workspace, (cudaStream_t)stream);
 }

@@ -75,6 +75,10 @@ int launch_attn_fwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
                           const int32_t* group_idx, const int32_t* n_groups, void* O, float* LSE,
                           int32_t* status_word, cudaStream_t st);
 
+bool route_sm100_supported(const Dims& dm);
+int launch_route_sm100(const Dims& dm, const void* Q, const void* chunk_sum, const void* group_sum,
+                       int32_t* chunk_idx, int32_t* group_idx, int32_t* n_groups, float* chunk_scores,
+                       float* group_scores, cudaStream_t st);
 bool attn_bwd_sm100_supported(const Dims& dm);
 int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
                           const float* LSE, const void* dO, const int32_t* group_idx,

@@ -21,11 +21,11 @@ def _dev(bits):
     return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
 
 
-def _route_both_ways(cfg, seed_shift=0):
+def _route_both_ways(cfg, seed_shift=0, flags=0):
     """Indices from hga_route (caller workspace) and from hga_route_static (no allocation)."""
     x = make_inputs(cfg.scaled(seed=cfg.seed + seed_shift), with_dO=False)
     Q, K = _dev(x["Q"]), _dev(x["K"])
-    ref = binding.HgaLayerBuffers(cfg, backward=False)
+    ref = binding.HgaLayerBuffers(cfg, backward=False, want_scores=True, flags=flags)
     ref.build_summaries(K, 0, cfg.total_len)
     ref.route(Q)
     # every buffer the static call touches exists before it runs; the call itself gets no workspace
@@ -43,11 +43,39 @@ def test_static_route_matches_route_on_two_calls_in_a_row():
     small = HgaConfig("static_small", 2, 4, 2, 128, 1536, 512, 64, 8, 64, 5, 3, 64, 128,
                       topics=16, needles=4, backward=False, seed=23)
     for cfg, shift in ((CONFIGS[3], 0), (small, 0), (CONFIGS[3], 1)):
-        ref, (ci, gi, ng) = _route_both_ways(cfg, shift)
+        # against hga_route running the same (shape-generic) kernels: exact
+        ref, (ci, gi, ng) = _route_both_ways(cfg, shift, flags=binding.HGA_FLAG_GENERIC_KERNELS)
         assert torch.equal(ci, ref.chunk_idx)
         assert torch.equal(gi, ref.group_idx)
         assert torch.equal(ng, ref.n_groups)
         assert int(ng.min()) >= 0
+        # against hga_route's default kernels (another fp32 summation order): the routing
+        # tolerance of the parity tests -- sets may differ only at score gaps below 1e-3
+        dflt, (ci, gi, ng) = _route_both_ways(cfg, shift)
+        assert torch.equal(ng, dflt.n_groups)
+        _same_up_to_near_ties(cfg, dflt, ci.cpu().numpy(), gi.cpu().numpy())
+
+
+def _same_up_to_near_ties(cfg, ref, ci, gi, gap=1e-3):
+    r_ci, r_gi = ref.chunk_idx.cpu().numpy(), ref.group_idx.cpu().numpy()
+    cs, gs = ref.chunk_scores.cpu().numpy(), ref.group_scores.cpu().numpy()
+    per = cfg.chunk // cfg.group
+    flat = lambda a: a.reshape(-1, a.shape[-1])
+    for it, (a, b, c, d, sc, sg) in enumerate(zip(flat(r_ci), flat(ci), flat(r_gi), flat(gi), flat(cs), flat(gs))):
+        sa, sb = set(a[a >= 0].tolist()), set(b[b >= 0].tolist())
+        assert len(sa) == len(sb)
+        if sa != sb:
+            kth = min(sc[j] for j in sa)
+            assert all(abs(sc[j] - kth) < gap for j in sa ^ sb), (it, sa ^ sb)
+        ga, gb = set(c[c >= 0].tolist()), set(d[d >= 0].tolist())
+        for r, j in enumerate(sorted(sa)):
+            if j not in sb:
+                continue
+            ca, cb = {m for m in ga if m // per == j}, {m for m in gb if m // per == j}
+            if ca != cb:
+                s = sg[r * per:(r + 1) * per]
+                kth = min(s[m - j * per] for m in ca)
+                assert all(abs(s[m - j * per] - kth) < gap for m in ca ^ cb), (it, j, ca ^ cb)
 
 
 def test_static_route_refuses_problems_beyond_its_array():
