@@ -17,6 +17,7 @@
 // TMEM (512 columns): S[2] dP[2] (64 each, double buffered) | dQ 128 | dV^T 64 | dK^T 64.
 // Shared memory: Q, dO (32 KB each), 3-stage K/V ring (16 + 16 KB per stage), P, dS (16 KB each).
 #include "hga_common.cuh"
+#include "hga_octets.cuh"
 #include "hga_sm100.cuh"
 
 namespace hga {
@@ -98,31 +99,23 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     tmem_relinquish();
   }
   if (warp == 0) {
+    // Q and dO do not depend on the routing: start their copies first
     if (lane == 0) {
       prefetch_tensormap(&map_q); prefetch_tensormap(&map_do);
       prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
-      const int32_t* gi = group_idx + (int64_t)item * dm.width;
-      int ng = n_groups[item], n = w.se / 8, prev = -1;
-      if (ng > dm.width) ng = dm.width;
-      if (ng < 0) ng = 0;
-      const int opg = dm.g / 8;
-      for (int i = 0; i < ng; ++i) {      // invalid entries are skipped, as in the forward kernel
-        const int m = gi[i];
-        if (m > prev && (int64_t)m * dm.g >= w.se && ((int64_t)m + 1) * dm.g <= w.ls) {
-          for (int u = 0; u < opg; ++u) sm.oct_row[n++] = m * dm.g + 8 * u;
-          prev = m;
-        }
-      }
-      sm.n_oct = n;
+      mbar_arrive_expect_tx(&sm.q_full, 2 * 128 * kBwdD * 2);
     }
     __syncwarp();
-    const int n_far = sm.n_oct;
-    for (int o = lane; o < w.se / 8; o += 32) sm.oct_row[o] = 8 * o;
-    const int n_local = (w.p0 + dm.Bq - w.ls) / 8;
-    for (int o = lane; o < n_local; o += 32) sm.oct_row[n_far + o] = w.ls + 8 * o;
-    __syncwarp();
+    {
+      const int o = lane & 15;
+      const int r = mt * 128 + 8 * o;
+      const int a = r / dm.Bq, t = r % dm.Bq;
+      if (lane < 16) tma_load_5d(sm.q + o * kOct, &map_q, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
+      else tma_load_5d(sm.dO + o * kOct, &map_do, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
+    }
+    bool bad;   // invalid entries are skipped exactly as in the forward kernel (which reports them)
+    const int n_oct = build_octet_table(dm, w, group_idx + (int64_t)item * dm.width, n_groups + item, sm.oct_row, &bad);
     if (lane == 0) {
-      const int n_oct = n_far + n_local;
       sm.n_oct = n_oct;
       // rows ascend, so the tiles holding active keys (position >= H) are a suffix
       const int n_tiles = (n_oct + 7) / 8;
@@ -148,15 +141,6 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
-    if (lane == 0) mbar_arrive_expect_tx(&sm.q_full, 2 * 128 * D * 2);
-    __syncwarp();
-    {
-      const int o = lane & 15;
-      const int r = mt * 128 + 8 * o;
-      const int a = r / dm.Bq, t = r % dm.Bq;
-      if (lane < 16) tma_load_5d(sm.q + o * kOct, &map_q, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
-      else tma_load_5d(sm.dO + o * kOct, &map_do, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
-    }
     bool ok = true;
     int issued = 0;
     for (int j = 0; j < n_tiles; ++j) {
@@ -183,23 +167,33 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       constexpr uint32_t idesc_sdp = idesc_bf16_f32(128, kKT, 0, 0);   // rows x keys, both K-major
       constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);      // dS K-major, K tile MN-major
       constexpr uint32_t idesc_dkv = idesc_bf16_f32(D, kKT, 1, 1);     // both MN-major
-      const uint32_t qa = smem_u32(sm.q), doa = smem_u32(sm.dO), pa = smem_u32(sm.p), dsa = smem_u32(sm.ds);
+      // Descriptors are built once; inside the loops an MMA costs two integer adds.
+      constexpr uint32_t kKvTile = kKT * D * 2;
+      const uint64_t q_k = smem_desc_sw128(smem_u32(sm.q), 16, kOct);        // Q  as K-major A   (S)
+      const uint64_t do_k = smem_desc_sw128(smem_u32(sm.dO), 16, kOct);      // dO as K-major A   (dP)
+      const uint64_t q_mn = smem_desc_sw128(smem_u32(sm.q), 1024, kOct);     // Q^T  as MN-major A (dK^T)
+      const uint64_t do_mn = smem_desc_sw128(smem_u32(sm.dO), 1024, kOct);   // dO^T as MN-major A (dV^T)
+      const uint64_t k_k0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, kOct);    // K tile, K-major B  (S)
+      const uint64_t v_k0 = smem_desc_sw128(smem_u32(sm.v[0]), 16, kOct);    // V tile, K-major B  (dP)
+      const uint64_t k_mn0 = smem_desc_sw128(smem_u32(sm.k[0]), 1024, kOct); // K tile, MN-major B (dQ)
+      const uint64_t ds_k = smem_desc_sw128(smem_u32(sm.ds), 16, 1024);      // dS as K-major A   (dQ)
+      const uint64_t ds_mn = smem_desc_sw128(smem_u32(sm.ds), 16, 1024);     // dS as MN-major B  (dK^T)
+      const uint64_t p_mn = smem_desc_sw128(smem_u32(sm.p), 16, 1024);       // P  as MN-major B  (dV^T)
       auto issue_sdp = [&](int j) {
-        const int st = j % kBwdStages, buf = j & 1;
-        const uint32_t ka = smem_u32(sm.k[st]), va = smem_u32(sm.v[st]);
+        const uint32_t st_off = (uint32_t)(j % kBwdStages) * kKvTile;
+        const uint64_t kd = desc_advance(k_k0, st_off), vd = desc_advance(v_k0, st_off);
+        const uint32_t s_acc = tmem + kColSdP + (j & 1) * 128;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-          mma_ss(tmem + kColSdP + buf * 128, smem_desc_sw128(qa + off, 16, kOct),
-                 smem_desc_sw128(ka + off, 16, kOct), idesc_sdp, kk > 0);
+          mma_ss(s_acc, desc_advance(q_k, off), desc_advance(kd, off), idesc_sdp, kk > 0);
         }
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-          mma_ss(tmem + kColSdP + buf * 128 + 64, smem_desc_sw128(doa + off, 16, kOct),
-                 smem_desc_sw128(va + off, 16, kOct), idesc_sdp, kk > 0);
+          mma_ss(s_acc + 64, desc_advance(do_k, off), desc_advance(vd, off), idesc_sdp, kk > 0);
         }
-        mma_commit(&sm.sdp_full[buf]);
+        mma_commit(&sm.sdp_full[j & 1]);
       };
       bool ok = bwd_wait(&sm.q_full, 0, abort) && bwd_wait(&sm.kv_full[0], 0, abort);
       if (ok) {
@@ -220,11 +214,11 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ok = bwd_wait(&sm.pds_full, j & 1, abort);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t ka = smem_u32(sm.k[st]);
+        const uint64_t kmn = desc_advance(k_mn0, (uint32_t)st * kKvTile);
 #pragma unroll
         for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per step
-          mma_ss(tmem + kColDQ, smem_desc_sw128(dsa + kk * 32, 16, 1024),
-                 smem_desc_sw128(ka + kk * 2 * kOct, 1024, kOct), idesc_dq, (j > 0 || kk > 0));
+          mma_ss(tmem + kColDQ, desc_advance(ds_k, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
+                 (j > 0 || kk > 0));
         if (j >= first_active) {
           if (n_active_done > 0) {
             ok = bwd_wait(&sm.dkv_free, (n_active_done - 1) & 1, abort);
@@ -232,15 +226,11 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             tc_fence_after_sync();
           }
 #pragma unroll
-          for (int kk = 0; kk < 128 / 16; ++kk) {   // 16 query rows per step (2 row octets)
-            mma_ss(tmem + kColDV, smem_desc_sw128(doa + kk * 2 * kOct, 1024, kOct),
-                   smem_desc_sw128(pa + kk * 2048, 16, 1024), idesc_dkv, kk > 0);
-          }
+          for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per step (2 row octets)
+            mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2 * kOct), desc_advance(p_mn, kk * 2048), idesc_dkv, kk > 0);
 #pragma unroll
-          for (int kk = 0; kk < 128 / 16; ++kk) {
-            mma_ss(tmem + kColDK, smem_desc_sw128(qa + kk * 2 * kOct, 1024, kOct),
-                   smem_desc_sw128(dsa + kk * 2048, 16, 1024), idesc_dkv, kk > 0);
-          }
+          for (int kk = 0; kk < 128 / 16; ++kk)
+            mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2 * kOct), desc_advance(ds_mn, kk * 2048), idesc_dkv, kk > 0);
           mma_commit(&sm.dkv_full);
           ++n_active_done;
         }

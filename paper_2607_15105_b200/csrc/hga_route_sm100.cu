@@ -147,13 +147,13 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             if (use > 0) ok = rt_wait(&sm.acc_free[buf], (use - 1) & 1, abort);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t aa = smem_u32(sm.a[s]);
-            const uint32_t ba = smem_u32(q_smem) + (uint32_t)hf * (uint32_t)(rows_half / 8) * kOctBytes;
+            const uint64_t ad = smem_desc_sw128(smem_u32(sm.a[s]), 16, kOctBytes);
+            const uint64_t bd = smem_desc_sw128(
+                smem_u32(q_smem) + (uint32_t)hf * (uint32_t)(rows_half / 8) * kOctBytes, 16, kOctBytes);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
               const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-              mma_ss(tmem + buf * 256, smem_desc_sw128(aa + off, 16, kOctBytes),
-                     smem_desc_sw128(ba + off, 16, kOctBytes), idesc, kk > 0);
+              mma_ss(tmem + buf * 256, desc_advance(ad, off), desc_advance(bd, off), idesc, kk > 0);
             }
             mma_commit(&sm.acc_full[buf]);
           }

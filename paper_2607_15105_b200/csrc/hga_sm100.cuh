@@ -167,6 +167,13 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
   return d;
 }
 
+// A descriptor whose start address is `byte_off` further on (byte_off a multiple of 16; shared
+// memory is < 256 KB, so the 14-bit address field cannot overflow).  One integer add: the single
+// MMA-issuing thread is latency-bound, so descriptors are built once and only advanced in loops.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t byte_off) {
+  return desc + (uint64_t)(byte_off >> 4);
+}
+
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, dense.
 //   a_mn_major / b_mn_major: 0 = K-major operand, 1 = MN-major operand.
 __host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N, int a_mn_major, int b_mn_major) {
