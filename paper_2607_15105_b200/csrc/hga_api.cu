@@ -187,7 +187,8 @@ int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* 
     if (rc) return rc;
   }
   if (attn_bwd_sm100_supported(dm)) {
-    rc = launch_attn_bwd_sm100(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV, status_word, st);
+    rc = launch_attn_bwd_sm100(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV, (float*)workspace,
+                               status_word, st);
     if (rc != HGA_ERR_UNSUPPORTED) return rc;
   }
   return launch_attn_bwd_generic(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV,

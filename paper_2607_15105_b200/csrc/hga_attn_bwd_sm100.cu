@@ -12,33 +12,49 @@
 // elements of one key row: its red.global.add.f32 is one coalesced 128-byte request.  History
 // tiles skip two of the five GEMMs and all atomics.
 //
+// Tiles are processed in DESCENDING key order.  The keys of the active segment are a suffix of the
+// ascending key list, so their tiles come first and their atomics drain while the history tiles
+// are still being computed, instead of forming a tail at the end of the CTA.
+//
 // Warp roles (320 threads): warp 0 producer (TMA), warp 1 MMA issuer, warps 2-5 one thread
 // per query row (delta, P, dS, dQ epilogue), warps 6-9 dK/dV reduction (thread = head_dim lane).
 // TMEM (512 columns): S[2] dP[2] (64 each, double buffered) | dQ 128 | dV^T 64 | dK^T 64.
-// Shared memory: Q, dO (32 KB each), 3-stage K/V ring (16 + 16 KB per stage), P, dS (16 KB each).
+// Shared memory: Q, dO (32 KB each), K ring (3 x 16 KB; a K tile is held until its dQ GEMM),
+// V ring (2 x 16 KB; a V tile is free once dP is issued), P and dS double buffered (4 x 16 KB), so
+// the row threads of tile s+1 never wait for the GEMMs that read P/dS of tile s.
 #include "hga_common.cuh"
 #include "hga_octets.cuh"
 #include "hga_sm100.cuh"
+
+// Optional phase timers: a profiling harness defines these three macros; otherwise no-ops.
+#ifndef HGA_TRACE_POINT
+#define HGA_TRACE_DECL
+#define HGA_TRACE_POINT(tag)
+#define HGA_TRACE_DUMP
+#endif
 
 namespace hga {
 
 using namespace sm100;
 
 constexpr int kBwdThreads = 320;
-constexpr int kBwdStages = 3;
+constexpr int kBwdKStages = 3;
+constexpr int kBwdVStages = 2;
 constexpr int kBwdD = 128;
 constexpr int kKT = 64;                         // keys per tile
 constexpr int kOct = 8 * kBwdD * 2;             // bytes of one octet of K/V/Q/dO rows (2 panels)
+constexpr int kKvTile = kKT * kBwdD * 2;        // bytes of one K or V tile
+constexpr int kPdsTile = 128 * kKT * 2;         // bytes of one P or dS tile
 
 struct BwdSmem {
   alignas(1024) uint8_t q[128 * kBwdD * 2];
   alignas(1024) uint8_t dO[128 * kBwdD * 2];
-  alignas(1024) uint8_t k[kBwdStages][kKT * kBwdD * 2];
-  alignas(1024) uint8_t v[kBwdStages][kKT * kBwdD * 2];
-  alignas(1024) uint8_t p[128 * kKT * 2];       // [16 row octets][8 rows][128 B], 128-byte swizzle
-  alignas(1024) uint8_t ds[128 * kKT * 2];
-  uint64_t q_full, kv_full[kBwdStages], kv_empty[kBwdStages];
-  uint64_t sdp_full[2], sdp_free[2], pds_full, pds_free, dkv_full, dkv_free, dq_done;
+  alignas(1024) uint8_t k[kBwdKStages][kKvTile];
+  alignas(1024) uint8_t v[kBwdVStages][kKvTile];
+  alignas(1024) uint8_t p[2][kPdsTile];         // [16 row octets][8 rows][128 B], 128-byte swizzle
+  alignas(1024) uint8_t ds[2][kPdsTile];
+  uint64_t q_full, k_full[kBwdKStages], k_empty[kBwdKStages], v_full[kBwdVStages], v_empty[kBwdVStages];
+  uint64_t sdp_full[2], sdp_free[2], pds_full[2], pds_free[2], dkv_full, dkv_free, dq_done;
   uint32_t tmem_base;
   int n_oct, first_active;
   volatile int abort;
@@ -63,11 +79,18 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+__device__ __forceinline__ float dot4_bf16(uint2 x, uint2 y) {
+  float s = __uint_as_float(x.x << 16) * __uint_as_float(y.x << 16);
+  s = fmaf(__uint_as_float(x.x & 0xffff0000u), __uint_as_float(y.x & 0xffff0000u), s);
+  s = fmaf(__uint_as_float(x.y << 16), __uint_as_float(y.y << 16), s);
+  s = fmaf(__uint_as_float(x.y & 0xffff0000u), __uint_as_float(y.y & 0xffff0000u), s);
+  return s;
+}
+
 __global__ void __launch_bounds__(kBwdThreads, 1)
 k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
                  const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                 const uint16_t* __restrict__ O, const uint16_t* __restrict__ dOg,
-                 const float* __restrict__ LSE, const int32_t* __restrict__ group_idx,
+                 const float* __restrict__ delta_ws, const float* __restrict__ LSE, const int32_t* __restrict__ group_idx,
                  const int32_t* __restrict__ n_groups, Dims dm, uint16_t* __restrict__ dQ,
                  float* __restrict__ dK, float* __restrict__ dV, int32_t* status_word) {
   constexpr int D = kBwdD;
@@ -77,6 +100,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   BwdSmem& sm = *reinterpret_cast<BwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  HGA_TRACE_DECL;
   const int n_mt_item = dm.rows / 128;
   const int item = blockIdx.x / n_mt_item;
   const int mt = blockIdx.x % n_mt_item;
@@ -86,9 +110,12 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < kBwdStages; ++s) { mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&sm.sdp_full[s], 1); mbar_init(&sm.sdp_free[s], 128); }
-    mbar_init(&sm.pds_full, 128); mbar_init(&sm.pds_free, 1);
+    for (int s = 0; s < kBwdKStages; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
+    for (int s = 0; s < kBwdVStages; ++s) { mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sm.sdp_full[s], 1); mbar_init(&sm.sdp_free[s], 128);
+      mbar_init(&sm.pds_full[s], 128); mbar_init(&sm.pds_free[s], 1);
+    }
     mbar_init(&sm.dkv_full, 1); mbar_init(&sm.dkv_free, 128);
     mbar_init(&sm.dq_done, 1);
     sm.abort = 0;
@@ -127,6 +154,16 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       sm.first_active = fa;
     }
   }
+  // Row threads: LSE and delta = rowsum(dO o O) of the thread's own row (delta comes from a
+  // coalesced pre-pass, k_bwd_delta_sm100).  Loaded here so the latency hides behind the set-up.
+  float delta = 0.f, row_lse = 0.f;
+  if (warp >= 2 && warp < 6) {
+    const int r = mt * 128 + (warp & 3) * 32 + lane;
+    const int64_t row = ((int64_t)b * dm.Hq + h * dm.G + r / dm.Bq) * dm.S + qb * dm.Bq + r % dm.Bq;
+    delta = delta_ws[row];
+    row_lse = LSE[row];
+  }
+  __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -135,31 +172,42 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const int n_oct = sm.n_oct;
   const int n_keys = n_oct * 8;
   const int n_tiles = (n_oct + 7) / 8;
-  const int first_active = sm.first_active;
+  const int n_active = n_tiles - sm.first_active;   // steps 0 .. n_active-1 hold active-segment keys
   volatile int* abort = &sm.abort;
-  constexpr uint32_t kStageBytes = 2 * kKT * D * 2;
+  HGA_TRACE_POINT(1);
+  // step s (processing order) handles tile j = n_tiles - 1 - s (ascending key order)
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
     bool ok = true;
     int issued = 0;
-    for (int j = 0; j < n_tiles; ++j) {
-      const int s = j % kBwdStages, use = j / kBwdStages;
-      if (lane == 0 && use > 0) ok = bwd_wait(&sm.kv_empty[s], (use - 1) & 1, abort);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      if (lane == 0) mbar_arrive_expect_tx(&sm.kv_full[s], kStageBytes);
-      __syncwarp();
+    for (int s = 0; s < n_tiles; ++s) {
+      const int j = n_tiles - 1 - s;
+      const int ks = s % kBwdKStages, vs = s % kBwdVStages;
       const int o = 8 * j + (lane & 7);
       const int row = o < n_oct ? sm.oct_row[o] : dm.L;    // past the list: zeros
-      if (lane < 8) tma_load_5d(sm.k[s] + lane * kOct, &map_k, &sm.kv_full[s], 0, row, 0, h, b);
-      else if (lane < 16) tma_load_5d(sm.v[s] + (lane - 8) * kOct, &map_v, &sm.kv_full[s], 0, row, 0, h, b);
-      issued = j + 1;
+      if (lane == 0 && s >= kBwdKStages) ok = bwd_wait(&sm.k_empty[ks], (s / kBwdKStages - 1) & 1, abort);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane == 0) mbar_arrive_expect_tx(&sm.k_full[ks], kKvTile);
+      __syncwarp();
+      if (lane < 8) tma_load_5d(sm.k[ks] + lane * kOct, &map_k, &sm.k_full[ks], 0, row, 0, h, b);
+      if (lane == 0 && s >= kBwdVStages) ok = bwd_wait(&sm.v_empty[vs], (s / kBwdVStages - 1) & 1, abort);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane == 0) mbar_arrive_expect_tx(&sm.v_full[vs], kKvTile);
+      __syncwarp();
+      if (lane >= 8 && lane < 16) tma_load_5d(sm.v[vs] + (lane - 8) * kOct, &map_v, &sm.v_full[vs], 0, row, 0, h, b);
+      issued = s + 1;
+      HGA_TRACE_POINT(2);
     }
     if (*abort && lane == 0) {
+      // giving up: let the copies still in flight land before shared memory is released
       mbar_wait(&sm.q_full, 0);
-      for (int j = issued > kBwdStages ? issued - kBwdStages : 0; j < issued; ++j)
-        mbar_wait(&sm.kv_full[j % kBwdStages], (j / kBwdStages) & 1);
+      for (int s = issued > kBwdKStages ? issued - kBwdKStages : 0; s < issued; ++s)
+        mbar_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1);
+      for (int s = issued > kBwdVStages ? issued - kBwdVStages : 0; s < issued; ++s)
+        mbar_wait(&sm.v_full[s % kBwdVStages], (s / kBwdVStages) & 1);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -168,7 +216,6 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);      // dS K-major, K tile MN-major
       constexpr uint32_t idesc_dkv = idesc_bf16_f32(D, kKT, 1, 1);     // both MN-major
       // Descriptors are built once; inside the loops an MMA costs two integer adds.
-      constexpr uint32_t kKvTile = kKT * D * 2;
       const uint64_t q_k = smem_desc_sw128(smem_u32(sm.q), 16, kOct);        // Q  as K-major A   (S)
       const uint64_t do_k = smem_desc_sw128(smem_u32(sm.dO), 16, kOct);      // dO as K-major A   (dP)
       const uint64_t q_mn = smem_desc_sw128(smem_u32(sm.q), 1024, kOct);     // Q^T  as MN-major A (dK^T)
@@ -176,13 +223,12 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const uint64_t k_k0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, kOct);    // K tile, K-major B  (S)
       const uint64_t v_k0 = smem_desc_sw128(smem_u32(sm.v[0]), 16, kOct);    // V tile, K-major B  (dP)
       const uint64_t k_mn0 = smem_desc_sw128(smem_u32(sm.k[0]), 1024, kOct); // K tile, MN-major B (dQ)
-      const uint64_t ds_k = smem_desc_sw128(smem_u32(sm.ds), 16, 1024);      // dS as K-major A   (dQ)
-      const uint64_t ds_mn = smem_desc_sw128(smem_u32(sm.ds), 16, 1024);     // dS as MN-major B  (dK^T)
-      const uint64_t p_mn = smem_desc_sw128(smem_u32(sm.p), 16, 1024);       // P  as MN-major B  (dV^T)
-      auto issue_sdp = [&](int j) {
-        const uint32_t st_off = (uint32_t)(j % kBwdStages) * kKvTile;
-        const uint64_t kd = desc_advance(k_k0, st_off), vd = desc_advance(v_k0, st_off);
-        const uint32_t s_acc = tmem + kColSdP + (j & 1) * 128;
+      const uint64_t ds0 = smem_desc_sw128(smem_u32(sm.ds[0]), 16, 1024);    // dS: K-major A (dQ) and MN-major B (dK^T)
+      const uint64_t p0 = smem_desc_sw128(smem_u32(sm.p[0]), 16, 1024);      // P : MN-major B (dV^T)
+      auto issue_sdp = [&](int s) {
+        const uint64_t kd = desc_advance(k_k0, (uint32_t)(s % kBwdKStages) * kKvTile);
+        const uint64_t vd = desc_advance(v_k0, (uint32_t)(s % kBwdVStages) * kKvTile);
+        const uint32_t s_acc = tmem + kColSdP + (s & 1) * 128;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
@@ -193,49 +239,58 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
           mma_ss(s_acc + 64, desc_advance(do_k, off), desc_advance(vd, off), idesc_sdp, kk > 0);
         }
-        mma_commit(&sm.sdp_full[j & 1]);
+        mma_commit(&sm.sdp_full[s & 1]);
+        mma_commit(&sm.v_empty[s % kBwdVStages]);      // the V tile is only needed for dP
       };
-      bool ok = bwd_wait(&sm.q_full, 0, abort) && bwd_wait(&sm.kv_full[0], 0, abort);
+      bool ok = bwd_wait(&sm.q_full, 0, abort) && bwd_wait(&sm.k_full[0], 0, abort) &&
+                bwd_wait(&sm.v_full[0], 0, abort);
       if (ok) {
         tc_fence_after_sync();
         issue_sdp(0);
       }
-      int n_active_done = 0;
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int st = j % kBwdStages;
-        if (j + 1 < n_tiles) {
-          ok = bwd_wait(&sm.kv_full[(j + 1) % kBwdStages], ((j + 1) / kBwdStages) & 1, abort);
-          // buffer (j+1)&1 held tile j-1: its rows have been read once sdp_free completed
-          if (ok && j >= 1) ok = bwd_wait(&sm.sdp_free[(j + 1) & 1], ((j - 1) >> 1) & 1, abort);
+      HGA_TRACE_POINT(3);
+      for (int s = 0; s < n_tiles && ok; ++s) {
+        if (s + 1 < n_tiles) {
+          ok = bwd_wait(&sm.k_full[(s + 1) % kBwdKStages], ((s + 1) / kBwdKStages) & 1, abort) &&
+               bwd_wait(&sm.v_full[(s + 1) % kBwdVStages], ((s + 1) / kBwdVStages) & 1, abort);
+          // TMEM buffer (s+1)&1 held step s-1: its rows have been read once sdp_free completed
+          if (ok && s >= 1) ok = bwd_wait(&sm.sdp_free[(s + 1) & 1], ((s - 1) >> 1) & 1, abort);
           if (!ok) break;
           tc_fence_after_sync();
-          issue_sdp(j + 1);
+          HGA_TRACE_POINT(6);
+          issue_sdp(s + 1);
+          HGA_TRACE_POINT(8);
         }
-        ok = bwd_wait(&sm.pds_full, j & 1, abort);
+        ok = bwd_wait(&sm.pds_full[s & 1], (s >> 1) & 1, abort);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint64_t kmn = desc_advance(k_mn0, (uint32_t)st * kKvTile);
+        HGA_TRACE_POINT(5);
+        const uint64_t kmn = desc_advance(k_mn0, (uint32_t)(s % kBwdKStages) * kKvTile);
+        const uint64_t dsd = desc_advance(ds0, (uint32_t)(s & 1) * kPdsTile);
 #pragma unroll
         for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per step
-          mma_ss(tmem + kColDQ, desc_advance(ds_k, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
-                 (j > 0 || kk > 0));
-        if (j >= first_active) {
-          if (n_active_done > 0) {
-            ok = bwd_wait(&sm.dkv_free, (n_active_done - 1) & 1, abort);
+          mma_ss(tmem + kColDQ, desc_advance(dsd, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
+                 (s > 0 || kk > 0));
+        HGA_TRACE_POINT(7);
+        if (s < n_active) {
+          if (s > 0) {
+            ok = bwd_wait(&sm.dkv_free, (s - 1) & 1, abort);
             if (!ok) break;
             tc_fence_after_sync();
           }
+          HGA_TRACE_POINT(9);
+          const uint64_t pd = desc_advance(p0, (uint32_t)(s & 1) * kPdsTile);
 #pragma unroll
           for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per step (2 row octets)
-            mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2 * kOct), desc_advance(p_mn, kk * 2048), idesc_dkv, kk > 0);
+            mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2 * kOct), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
 #pragma unroll
           for (int kk = 0; kk < 128 / 16; ++kk)
-            mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2 * kOct), desc_advance(ds_mn, kk * 2048), idesc_dkv, kk > 0);
+            mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2 * kOct), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
           mma_commit(&sm.dkv_full);
-          ++n_active_done;
+          HGA_TRACE_POINT(4);
         }
-        mma_commit(&sm.pds_free);
-        mma_commit(&sm.kv_empty[st]);
+        mma_commit(&sm.pds_free[s & 1]);
+        mma_commit(&sm.k_empty[s % kBwdKStages]);
       }
       if (ok) mma_commit(&sm.dq_done);
     }
@@ -249,40 +304,25 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int limit = n_keys - dm.Bq + t + 1;
     const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
     const float sl2 = dm.scale * 1.4426950408889634f;
-    // delta = rowsum(dO o O); LSE in log2 units
-    float delta = 0.f;
-    {
-      const uint4* o4 = reinterpret_cast<const uint4*>(O + b * dm.os[0] + hq * dm.os[1] + (int64_t)srow * dm.os[2]);
-      const uint4* g4 = reinterpret_cast<const uint4*>(dOg + b * dm.os[0] + hq * dm.os[1] + (int64_t)srow * dm.os[2]);
-#pragma unroll 4
-      for (int i = 0; i < D / 8; ++i) {
-        const uint4 x = o4[i], y = g4[i];
-        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          delta = fmaf(__uint_as_float(xs[e] << 16), __uint_as_float(ys[e] << 16), delta);
-          delta = fmaf(__uint_as_float(xs[e] & 0xffff0000u), __uint_as_float(ys[e] & 0xffff0000u), delta);
-        }
-      }
-    }
-    const float neg_lse2 = -LSE[((int64_t)b * dm.Hq + hq) * dm.S + srow] * 1.4426950408889634f;
+    const float neg_lse2 = -row_lse * 1.4426950408889634f;
     const float neg_delta_s = -delta * dm.scale;
+    HGA_TRACE_POINT(10);
     // this row's 128-byte line inside the P / dS buffers, and its swizzle key
     const uint32_t line = (uint32_t)(row_in_tile >> 3) * 1024 + (uint32_t)(row_in_tile & 7) * 128;
     const uint32_t key = (uint32_t)(row_in_tile & 7);
-    const uint32_t p_line = smem_u32(sm.p) + line, ds_line = smem_u32(sm.ds) + line;
     bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
-      const int buf = j & 1;
-      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[buf], (j >> 1) & 1, abort));
+    for (int s = 0; s < n_tiles; ++s) {
+      const int j = n_tiles - 1 - s, buf = s & 1;
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[buf], (s >> 1) & 1, abort));
       if (!ok) break;
       tc_fence_after_sync();
+      HGA_TRACE_POINT(11);
       const int vis = limit - kKT * j;
       uint32_t pk[32], dk[32];
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        uint32_t s[32], dp[32];
-        tmem_ld32(lane_base + kColSdP + buf * 128 + half * 32, s);
+        uint32_t sv[32], dp[32];
+        tmem_ld32(lane_base + kColSdP + buf * 128 + half * 32, sv);
         tmem_ld32(lane_base + kColSdP + buf * 128 + 64 + half * 32, dp);
         tmem_wait_ld();
         if (half == 1) {
@@ -292,20 +332,25 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), sl2, neg_lse2));
-          float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), sl2, neg_lse2));
-          if (half * 32 + 2 * i >= vis) p0 = 0.f;
-          if (half * 32 + 2 * i + 1 >= vis) p1 = 0.f;
+          float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), sl2, neg_lse2));
+          float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), sl2, neg_lse2));
+          if (vis < kKT) {                    // diagonal / ragged tile only
+            if (half * 32 + 2 * i >= vis) p0 = 0.f;
+            if (half * 32 + 2 * i + 1 >= vis) p1 = 0.f;
+          }
           const float d0 = p0 * fmaf(__uint_as_float(dp[2 * i]), dm.scale, neg_delta_s);
           const float d1 = p1 * fmaf(__uint_as_float(dp[2 * i + 1]), dm.scale, neg_delta_s);
           pk[half * 16 + i] = pack_bf16(p0, p1);
           dk[half * 16 + i] = pack_bf16(d0, d1);
         }
       }
-      if (j > 0) {
-        ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_free, (j - 1) & 1, abort));
+      HGA_TRACE_POINT(12);
+      if (s >= 2) {     // the GEMMs that read this P/dS buffer two steps ago must have finished
+        ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_free[buf], ((s - 2) >> 1) & 1, abort));
         if (!ok) break;
       }
+      HGA_TRACE_POINT(13);
+      const uint32_t p_line = smem_u32(sm.p[buf]) + line, ds_line = smem_u32(sm.ds[buf]) + line;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {    // 8 chunks of 16 bytes (8 keys) per row, XOR-swizzled
         const uint32_t off = ((uint32_t)c ^ key) * 16;
@@ -313,24 +358,30 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         st_shared_v4(ds_line + off, dk[4 * c], dk[4 * c + 1], dk[4 * c + 2], dk[4 * c + 3]);
       }
       fence_proxy_async_smem();
-      mbar_arrive(&sm.pds_full);
+      mbar_arrive(&sm.pds_full[buf]);
+      HGA_TRACE_POINT(14);
     }
     if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.dq_done, 0, abort));
+    HGA_TRACE_POINT(20);
     if (ok) {
       tc_fence_after_sync();
       uint16_t* qrow = dQ + b * dm.qs[0] + hq * dm.qs[1] + (int64_t)srow * dm.qs[2];
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t x[32];
-        tmem_ld32(lane_base + kColDQ + c * 32, x);
+      for (int c2 = 0; c2 < D / 64; ++c2) {
+        uint32_t x[2][32];
+        tmem_ld32(lane_base + kColDQ + c2 * 64, x[0]);
+        tmem_ld32(lane_base + kColDQ + c2 * 64 + 32, x[1]);
         tmem_wait_ld();
-        uint4* dst = reinterpret_cast<uint4*>(qrow + c * 32);
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-          dst[i] = make_uint4(pack_bf16(__uint_as_float(x[8 * i]), __uint_as_float(x[8 * i + 1])),
-                              pack_bf16(__uint_as_float(x[8 * i + 2]), __uint_as_float(x[8 * i + 3])),
-                              pack_bf16(__uint_as_float(x[8 * i + 4]), __uint_as_float(x[8 * i + 5])),
-                              pack_bf16(__uint_as_float(x[8 * i + 6]), __uint_as_float(x[8 * i + 7])));
+        for (int c = 0; c < 2; ++c) {
+          uint4* dst = reinterpret_cast<uint4*>(qrow + c2 * 64 + c * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            dst[i] = make_uint4(pack_bf16(__uint_as_float(x[c][8 * i]), __uint_as_float(x[c][8 * i + 1])),
+                                pack_bf16(__uint_as_float(x[c][8 * i + 2]), __uint_as_float(x[c][8 * i + 3])),
+                                pack_bf16(__uint_as_float(x[c][8 * i + 4]), __uint_as_float(x[c][8 * i + 5])),
+                                pack_bf16(__uint_as_float(x[c][8 * i + 6]), __uint_as_float(x[c][8 * i + 7])));
+        }
       }
     }
   } else {
@@ -341,10 +392,12 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     float* dKb = dK + ((int64_t)(b * dm.Hkv + h) * dm.S) * D + e;
     float* dVb = dV + ((int64_t)(b * dm.Hkv + h) * dm.S) * D + e;
     bool ok = true;
-    for (int j = first_active, n = 0; j < n_tiles; ++j, ++n) {
-      ok = __all_sync(0xffffffffu, bwd_wait(&sm.dkv_full, n & 1, abort));
+    for (int s = 0; s < n_active; ++s) {
+      const int j = n_tiles - 1 - s;
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.dkv_full, s & 1, abort));
       if (!ok) break;
       tc_fence_after_sync();
+      HGA_TRACE_POINT(16);
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t gv[32], gk[32];
@@ -367,15 +420,36 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
       }
+      HGA_TRACE_POINT(18);
     }
   }
+  HGA_TRACE_POINT(30);
 
+  // Common exit.  The single-thread roles leave their warps diverged, so every warp reconverges
+  // first: a block barrier reached by part of a warp would count that warp as arrived.
+  __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
+  HGA_TRACE_POINT(31);
+  HGA_TRACE_DUMP;
   if (tid == 0 && sm.abort && status_word) atomicOr(status_word, HGA_STATUS_WAIT_TIMEOUT);
-  if (warp == 1) {
-    __syncwarp();
-    tmem_dealloc(tmem, 512);
+  if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+// delta[row] = sum_e dO[row][e] * O[row][e]: one warp per row, 8-byte loads (a 256-byte row per
+// request), an HBM stream of O and dO at full-GPU bandwidth.
+__global__ void __launch_bounds__(256)
+k_bwd_delta_sm100(const uint16_t* __restrict__ O, const uint16_t* __restrict__ dO, Dims dm,
+                  float* __restrict__ delta) {
+  const int lane = threadIdx.x & 31;
+  const int64_t n_rows = (int64_t)dm.B * dm.Hq * dm.S;
+  for (int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); row < n_rows; row += (int64_t)gridDim.x * 8) {
+    const int s = row % dm.S, hq = (row / dm.S) % dm.Hq, b = row / ((int64_t)dm.S * dm.Hq);
+    const int64_t off = b * dm.os[0] + hq * dm.os[1] + (int64_t)s * dm.os[2] + lane * 4;
+    float part = dot4_bf16(*reinterpret_cast<const uint2*>(O + off), *reinterpret_cast<const uint2*>(dO + off));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if (lane == 0) delta[row] = part;
   }
 }
 
@@ -386,9 +460,8 @@ bool attn_bwd_sm100_supported(const Dims& dm) {
 
 int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
                           const float* LSE, const void* dO, const int32_t* group_idx,
-                          const int32_t* n_groups, void* dQ, float* dK, float* dV,
+                          const int32_t* n_groups, void* dQ, float* dK, float* dV, float* delta_ws,
                           int32_t* status_word, cudaStream_t st) {
-  constexpr int D = kBwdD;
   CUtensorMap mq, mdo, mk, mv;
   const uint32_t box[5] = {64, 8, 2, 1, 1};
   const uint64_t dq[5] = {64, (uint64_t)dm.S, 2, (uint64_t)dm.Hq, (uint64_t)dm.B};
@@ -406,12 +479,15 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
   if (smem > 227 * 1024) return HGA_ERR_UNSUPPORTED;
   cudaError_t e = cudaFuncSetAttribute(k_attn_bwd_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return record_cuda(e);
+  const int64_t n_rows = (int64_t)dm.B * dm.Hq * dm.S;
+  const int delta_blocks = (int)((n_rows + 7) / 8 < 148 * 16 ? (n_rows + 7) / 8 : 148 * 16);
+  k_bwd_delta_sm100<<<delta_blocks, 256, 0, st>>>((const uint16_t*)O, (const uint16_t*)dO, dm, delta_ws);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return record_cuda(e);
   const int units = dm.B * dm.Hkv * dm.NQB * (dm.rows / 128);
-  k_attn_bwd_sm100<<<units, kBwdThreads, smem, st>>>(mq, mdo, mk, mv, (const uint16_t*)O, (const uint16_t*)dO,
-                                                    LSE, group_idx, n_groups, dm, (uint16_t*)dQ, dK, dV,
-                                                    status_word);
-  count_launch();
-  (void)D;
+  k_attn_bwd_sm100<<<units, kBwdThreads, smem, st>>>(mq, mdo, mk, mv, delta_ws, LSE, group_idx, n_groups, dm,
+                                                    (uint16_t*)dQ, dK, dV, status_word);
+  count_launch(2);
   return record_cuda(cudaGetLastError());
 }
 

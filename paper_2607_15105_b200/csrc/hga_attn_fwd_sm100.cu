@@ -128,6 +128,7 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (bad && status_word) atomicOr(status_word, HGA_STATUS_BAD_INDEX);
     }
   }
+  __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -363,6 +364,7 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   // common exit: every role has either finished or given up; tensor memory is released
   HGA_TRACE_POINT(30);
+  __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
   HGA_TRACE_POINT(31);

@@ -82,7 +82,7 @@ int launch_route_sm100(const Dims& dm, const void* Q, const void* chunk_sum, con
 bool attn_bwd_sm100_supported(const Dims& dm);
 int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
                           const float* LSE, const void* dO, const int32_t* group_idx,
-                          const int32_t* n_groups, void* dQ, float* dK, float* dV,
+                          const int32_t* n_groups, void* dQ, float* dK, float* dV, float* delta_ws,
                           int32_t* status_word, cudaStream_t st);
 
 // Validates an hga_params block and fills the resolved description (hga_api.cu).

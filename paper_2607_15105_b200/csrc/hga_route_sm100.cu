@@ -96,6 +96,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   if (warp == 0 && lane == 0) {
     prefetch_tensormap(&map_q); prefetch_tensormap(&map_cs); prefetch_tensormap(&map_gs);
   }
+  __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -205,6 +206,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       group_scores[(int64_t)item * dm.kc * dm.per + i] = -INFINITY;
 
   if (k_sel > 0) run_phase(0, n_ct, false);
+  __syncwarp();          // the roles diverge inside a warp: reconverge before the block barrier
   __syncthreads();
 
   // ---------------------------------------------------------------------- chunk top-k
@@ -242,6 +244,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 
   // ---------------------------------------------------------------------- groups of the opened chunks
   if (k_sel > 0 && !sm.abort) run_phase(n_ct, n_gt, true);
+  __syncwarp();
   __syncthreads();
   if (!sm.abort) {
     int32_t* gi = group_idx + (int64_t)item * dm.width;
@@ -267,6 +270,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     if (tid == 0) n_groups[item] = k_sel * dm.kge;
   }
 
+  __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) {
