@@ -82,6 +82,11 @@ def active_group_pairs(cfg, group_idx, n_groups):
     return n * cfg.group * cfg.gqa * cfg.q_block
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the call's main kernel, from the ncu
+# captures summarised under profiles/ (k_attn_fwd_sm100_cfg3_16k.md, k_attn_bwd_sm100_cfg3_16k.md).
+NCU_TRAFFIC_BYTES = {3: {"hga_attn_fwd": 63.56e6, "hga_attn_bwd": 104.89e6}}
+
+
 def roofline_entry(name, flops, nbytes, seconds, peaks, sustained=False):
     tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"]
     t_flop = flops / (tf * 1e12)
@@ -232,6 +237,7 @@ def main():
     ap.add_argument("--config", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA-graph replay")
     ap.add_argument("--flags", type=int, default=0, help="hga_params.flags (debugging)")
     args = ap.parse_args()
     cfg = CONFIGS[args.config]
@@ -307,14 +313,45 @@ def main():
     barrier()
     launches = binding.hga_kernel_launch_count() - launches0
     per_call = np.array([[ev[j].elapsed_time(ev[j + 1]) for j in range(n_ev - 1)] for ev in events])  # ms
-    step_ms = np.array([ev[0].elapsed_time(ev[-1]) for ev in events])
+    eager_ms = np.array([ev[0].elapsed_time(ev[-1]) for ev in events])
+    step_ms, launch_mode = eager_ms, "eager"
+    if not args.no_graph:
+        # The headline step: the same four C-ABI calls captured once into a CUDA graph and replayed,
+        # which removes the host-side launch gaps between them.  Same K steps, same flush.
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                one_step()                                   # warm the capture stream
+            torch.cuda.current_stream().wait_stream(side)
+            graph = torch.cuda.CUDAGraph()
+            c0 = binding.hga_kernel_launch_count()
+            with torch.cuda.graph(graph):
+                one_step()
+            per_step_launches = binding.hga_kernel_launch_count() - c0
+            for _ in range(3):
+                flush.zero_()
+                graph.replay()
+            barrier()
+            g_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                    for _ in range(args.steps)]
+            for a, b in g_ev:
+                flush.zero_()
+                a.record(stream)
+                graph.replay()
+                b.record(stream)
+            barrier()
+            step_ms = np.array([a.elapsed_time(b) for a, b in g_ev])
+            launches = per_step_launches * args.steps
+            launch_mode = "cuda_graph"
+        except Exception as exc:  # capture unavailable: keep the eager numbers, say why
+            launch_mode = "eager (graph capture failed: %s)" % type(exc).__name__
     # warm-L2 variant (reported beside the headline, not instead of it)
     warm_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(args.steps)]
     for i in range(args.steps):
         one_step(warm_ev[i])
     barrier()
     warm_ms = np.array([ev[0].elapsed_time(ev[-1]) for ev in warm_ev])
-    clocks = sampler.stop() if rank == 0 else None
 
     # end to end through the host-buffer entry point: H2D of the step's inputs, D2H of its results
     H = cfg.history
@@ -345,6 +382,7 @@ def main():
         b.record(stream)
     barrier()
     e2e_ms = np.array([a.elapsed_time(b) for a, b in e2e_ev])
+    clocks = sampler.stop() if rank == 0 else None      # sampled across all timed loops above
     status = int(buf.status.item())
 
     def max_over_ranks(v):
@@ -369,6 +407,10 @@ def main():
         roofs = {"attn_fwd": roofline_entry("hga_attn_fwd", wc["fwd_flops"], wc["fwd_bytes"], med[2], peaks)}
         if cfg.backward:
             roofs["attn_bwd"] = roofline_entry("hga_attn_bwd", wc["bwd_flops"], wc["bwd_bytes"], med[3], peaks)
+        for r in roofs.values():
+            r["traffic"] = NCU_TRAFFIC_BYTES.get(args.config, {}).get(r["kernel"])
+            r["algorithmic_bytes"] = wc["fwd_bytes"] if r["kernel"] == "hga_attn_fwd" else wc["bwd_bytes"]
+            r["algorithmic_flops"] = wc["fwd_flops"] if r["kernel"] == "hga_attn_fwd" else wc["bwd_flops"]
         dominant = max(roofs.values(), key=lambda r: r["measured_us"])
         attn_us = sum(r["measured_us"] for r in roofs.values())
         attn_roof_us = sum(r["roofline_us"] for r in roofs.values())
@@ -389,6 +431,9 @@ def main():
                           "frac_of_roofline": round(attn_roof_us / attn_us, 4),
                           "tokens_per_s": round(cfg.tokens_per_step / (attn_us * 1e-6), 1)},
             "per_call_us_median": {n: round(float(m) * 1e6, 2) for n, m in zip(names, med)},
+            "launch": launch_mode,
+            "eager": {"value": round(cfg.tokens_per_step * args.steps / (eager_ms.sum() * 1e-3), 1),
+                      "ms_per_step": round(float(eager_ms.mean()), 5)},
             "warm_l2": {"value": round(tokens / (warm_total_ms * 1e-3), 1),
                         "ms_per_step": round(warm_total_ms / args.steps, 5)},
             "device_status_word": status,

@@ -441,15 +441,33 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 __global__ void __launch_bounds__(256)
 k_bwd_delta_sm100(const uint16_t* __restrict__ O, const uint16_t* __restrict__ dO, Dims dm,
                   float* __restrict__ delta) {
-  const int lane = threadIdx.x & 31;
+  // half a warp per row (16 lanes x 16 bytes = one 256-byte row), 8 rows per warp in flight
+  const int lane = threadIdx.x & 31, sub = lane >> 4, chunk = lane & 15;
   const int64_t n_rows = (int64_t)dm.B * dm.Hq * dm.S;
-  for (int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); row < n_rows; row += (int64_t)gridDim.x * 8) {
-    const int s = row % dm.S, hq = (row / dm.S) % dm.Hq, b = row / ((int64_t)dm.S * dm.Hq);
-    const int64_t off = b * dm.os[0] + hq * dm.os[1] + (int64_t)s * dm.os[2] + lane * 4;
-    float part = dot4_bf16(*reinterpret_cast<const uint2*>(O + off), *reinterpret_cast<const uint2*>(dO + off));
+  const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  for (int64_t base = warp_id * 8; base < n_rows; base += n_warps * 8) {
+    uint4 x[4], y[4];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-    if (lane == 0) delta[row] = part;
+    for (int u = 0; u < 4; ++u) {
+      const int64_t row = base + 2 * u + sub;
+      x[u] = y[u] = make_uint4(0, 0, 0, 0);
+      if (row < n_rows) {
+        const int s = row % dm.S, hq = (row / dm.S) % dm.Hq, b = row / ((int64_t)dm.S * dm.Hq);
+        const int64_t off = b * dm.os[0] + hq * dm.os[1] + (int64_t)s * dm.os[2] + chunk * 8;
+        x[u] = *reinterpret_cast<const uint4*>(O + off);
+        y[u] = *reinterpret_cast<const uint4*>(dO + off);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      float part = dot4_bf16(make_uint2(x[u].x, x[u].y), make_uint2(y[u].x, y[u].y)) +
+                   dot4_bf16(make_uint2(x[u].z, x[u].w), make_uint2(y[u].z, y[u].w));
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+      const int64_t row = base + 2 * u + sub;
+      if (chunk == 0 && row < n_rows) delta[row] = part;
+    }
   }
 }
 
@@ -480,7 +498,9 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
   cudaError_t e = cudaFuncSetAttribute(k_attn_bwd_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return record_cuda(e);
   const int64_t n_rows = (int64_t)dm.B * dm.Hq * dm.S;
-  const int delta_blocks = (int)((n_rows + 7) / 8 < 148 * 16 ? (n_rows + 7) / 8 : 148 * 16);
+  // one block = 8 warps x 8 rows; a multiple of the SM count when there is enough work
+  const int64_t want_blocks = (n_rows + 63) / 64;
+  const int delta_blocks = (int)(want_blocks < 148 * 8 ? want_blocks : 148 * 8);
   k_bwd_delta_sm100<<<delta_blocks, 256, 0, st>>>((const uint16_t*)O, (const uint16_t*)dO, dm, delta_ws);
   e = cudaGetLastError();
   if (e != cudaSuccess) return record_cuda(e);
