@@ -251,16 +251,15 @@ def main():
     import torch.distributed as dist
     from paper_2607_15105_b200 import binding
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2607_15105_b200 import sharding
+    rank, world, local_rank = sharding.env_rank()
     torch.cuda.set_device(local_rank)
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     # every rank draws its own sequence (weak scaling): same shapes, different seed
-    x = make_inputs(cfg.scaled(seed=cfg.seed + 1000 * rank) if rank else cfg)
+    x = make_inputs(sharding.rank_config(cfg, rank))
 
     def dev(a):
         return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
@@ -386,11 +385,7 @@ def main():
     status = int(buf.status.item())
 
     def max_over_ranks(v):
-        if world == 1:
-            return float(v)
-        t = torch.tensor([float(v)], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return sharding.max_over_ranks(v, device="cuda")
 
     total_ms = max_over_ranks(step_ms.sum())
     warm_total_ms = max_over_ranks(warm_ms.sum())
