@@ -16,8 +16,9 @@
 // ascending key list, so their tiles come first and their atomics drain while the history tiles
 // are still being computed, instead of forming a tail at the end of the CTA.
 //
-// Warp roles (320 threads): warp 0 producer (TMA), warp 1 MMA issuer, warps 2-5 one thread
-// per query row (delta, P, dS, dQ epilogue), warps 6-9 dK/dV reduction (thread = head_dim lane).
+// Warp roles (448 threads): warp 0 producer (TMA), warp 1 MMA issuer, warps 2-5 and 6-9 two
+// warpgroups of one thread per query row (P, dS, dQ epilogue) taking alternate tiles, warps 10-13
+// dK/dV reduction (thread = head_dim lane).
 // TMEM (512 columns): S[2] dP[2] (64 each, double buffered) | dQ 128 | dV^T 64 | dK^T 64.
 // Shared memory: Q, dO (32 KB each), K ring (3 x 16 KB; a K tile is held until its dQ GEMM),
 // V ring (2 x 16 KB; a V tile is free once dP is issued), P and dS double buffered (4 x 16 KB), so
@@ -37,7 +38,8 @@ namespace hga {
 
 using namespace sm100;
 
-constexpr int kBwdThreads = 320;
+constexpr int kBwdThreads = 512;                // 16 warps: 128 registers per thread
+constexpr int kBwdProducers = 3;                // warps 0, 14, 15 issue the K/V copies
 constexpr int kBwdKStages = 3;
 constexpr int kBwdVStages = 2;
 constexpr int kBwdD = 128;
@@ -110,8 +112,8 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < kBwdKStages; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
-    for (int s = 0; s < kBwdVStages; ++s) { mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1); }
+    for (int s = 0; s < kBwdKStages; ++s) { mbar_init(&sm.k_full[s], kBwdProducers); mbar_init(&sm.k_empty[s], 1); }
+    for (int s = 0; s < kBwdVStages; ++s) { mbar_init(&sm.v_full[s], kBwdProducers); mbar_init(&sm.v_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sm.sdp_full[s], 1); mbar_init(&sm.sdp_free[s], 128);
       mbar_init(&sm.pds_full[s], 128); mbar_init(&sm.pds_free[s], 1);
@@ -157,7 +159,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   // Row threads: LSE and delta = rowsum(dO o O) of the thread's own row (delta comes from a
   // coalesced pre-pass, k_bwd_delta_sm100).  Loaded here so the latency hides behind the set-up.
   float delta = 0.f, row_lse = 0.f;
-  if (warp >= 2 && warp < 6) {
+  if (warp >= 2 && warp < 10) {
     const int r = mt * 128 + (warp & 3) * 32 + lane;
     const int64_t row = ((int64_t)b * dm.Hq + h * dm.G + r / dm.Bq) * dm.S + qb * dm.Bq + r % dm.Bq;
     delta = delta_ws[row];
@@ -177,33 +179,46 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   HGA_TRACE_POINT(1);
   // step s (processing order) handles tile j = n_tiles - 1 - s (ascending key order)
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ producer
+  if (warp == 0 || warp >= 14) {
+    // ------------------------------------------------------------------ producers
+    // Issuing one TMA box costs the issuing warp on the order of a hundred cycles, so the sixteen
+    // octet boxes of a step are spread over three warps: producer p takes octets p, p+3, p+6 of
+    // the K tile (lanes 0-2) and of the V tile (lanes 8-10).  Every producer arrives on the full
+    // barriers with the byte count of its own boxes.
+    const int pi = warp == 0 ? 0 : warp - 13;
+    const int sub = lane & 7;
+    const int oct_in_tile = pi + kBwdProducers * sub;          // < 8 for the lanes that copy
+    const bool k_lane = lane < 8 && oct_in_tile < 8, v_lane = lane >= 8 && lane < 16 && oct_in_tile < 8;
+    const uint32_t my_bytes = (uint32_t)((8 - pi + kBwdProducers - 1) / kBwdProducers) * kOct;
     bool ok = true;
     int issued = 0;
     for (int s = 0; s < n_tiles; ++s) {
       const int j = n_tiles - 1 - s;
       const int ks = s % kBwdKStages, vs = s % kBwdVStages;
-      const int o = 8 * j + (lane & 7);
+      const int o = 8 * j + oct_in_tile;
       const int row = o < n_oct ? sm.oct_row[o] : dm.L;    // past the list: zeros
       if (lane == 0 && s >= kBwdKStages) ok = bwd_wait(&sm.k_empty[ks], (s / kBwdKStages - 1) & 1, abort);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
-      if (lane == 0) mbar_arrive_expect_tx(&sm.k_full[ks], kKvTile);
+      HGA_TRACE_POINT(21);
+      if (lane == 0) mbar_arrive_expect_tx(&sm.k_full[ks], my_bytes);
       __syncwarp();
-      if (lane < 8) tma_load_5d(sm.k[ks] + lane * kOct, &map_k, &sm.k_full[ks], 0, row, 0, h, b);
+      if (k_lane) tma_load_5d(sm.k[ks] + oct_in_tile * kOct, &map_k, &sm.k_full[ks], 0, row, 0, h, b);
+      HGA_TRACE_POINT(22);
       if (lane == 0 && s >= kBwdVStages) ok = bwd_wait(&sm.v_empty[vs], (s / kBwdVStages - 1) & 1, abort);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
-      if (lane == 0) mbar_arrive_expect_tx(&sm.v_full[vs], kKvTile);
+      HGA_TRACE_POINT(23);
+      if (lane == 0) mbar_arrive_expect_tx(&sm.v_full[vs], my_bytes);
       __syncwarp();
-      if (lane >= 8 && lane < 16) tma_load_5d(sm.v[vs] + (lane - 8) * kOct, &map_v, &sm.v_full[vs], 0, row, 0, h, b);
+      if (v_lane) tma_load_5d(sm.v[vs] + oct_in_tile * kOct, &map_v, &sm.v_full[vs], 0, row, 0, h, b);
       issued = s + 1;
       HGA_TRACE_POINT(2);
     }
     if (*abort && lane == 0) {
-      // giving up: let the copies still in flight land before shared memory is released
-      mbar_wait(&sm.q_full, 0);
+      // giving up: let the copies still in flight land before shared memory is released (bounded:
+      // a full barrier also needs the other producers, which may have stopped earlier)
+      if (pi == 0) mbar_wait(&sm.q_full, 0);
       for (int s = issued > kBwdKStages ? issued - kBwdKStages : 0; s < issued; ++s)
         mbar_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1);
       for (int s = issued > kBwdVStages ? issued - kBwdVStages : 0; s < issued; ++s)
@@ -253,6 +268,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (s + 1 < n_tiles) {
           ok = bwd_wait(&sm.k_full[(s + 1) % kBwdKStages], ((s + 1) / kBwdKStages) & 1, abort) &&
                bwd_wait(&sm.v_full[(s + 1) % kBwdVStages], ((s + 1) / kBwdVStages) & 1, abort);
+          HGA_TRACE_POINT(24);
           // TMEM buffer (s+1)&1 held step s-1: its rows have been read once sdp_free completed
           if (ok && s >= 1) ok = bwd_wait(&sm.sdp_free[(s + 1) & 1], ((s - 1) >> 1) & 1, abort);
           if (!ok) break;
@@ -294,8 +310,12 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       if (ok) mma_commit(&sm.dq_done);
     }
-  } else if (warp < 6) {
+  } else if (warp < 10) {
     // ------------------------------------------------------------------ one thread per query row
+    // Two warpgroups take alternate steps (warps 2-5 the even ones, 6-9 the odd ones), each with
+    // its own S/dP buffer in TMEM and its own P/dS buffer in shared memory, so the exp2 / dS work
+    // of step s+1 overlaps that of step s and the loop is paced by the tensor pipe.
+    const int wg = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int row_in_tile = quarter * 32 + lane;
     const int r = mt * 128 + row_in_tile;
@@ -310,78 +330,77 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // this row's 128-byte line inside the P / dS buffers, and its swizzle key
     const uint32_t line = (uint32_t)(row_in_tile >> 3) * 1024 + (uint32_t)(row_in_tile & 7) * 128;
     const uint32_t key = (uint32_t)(row_in_tile & 7);
+    const uint32_t p_line = smem_u32(sm.p[wg]) + line, ds_line = smem_u32(sm.ds[wg]) + line;
+    const uint32_t sdp_addr = lane_base + kColSdP + wg * 128;
     bool ok = true;
-    for (int s = 0; s < n_tiles; ++s) {
-      const int j = n_tiles - 1 - s, buf = s & 1;
-      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[buf], (s >> 1) & 1, abort));
+    for (int s = wg; s < n_tiles; s += 2) {          // buffer index s & 1 == wg
+      const int j = n_tiles - 1 - s;
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[wg], (s >> 1) & 1, abort));
       if (!ok) break;
       tc_fence_after_sync();
       HGA_TRACE_POINT(11);
-      const int vis = limit - kKT * j;
-      uint32_t pk[32], dk[32];
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t sv[32], dp[32];
-        tmem_ld32(lane_base + kColSdP + buf * 128 + half * 32, sv);
-        tmem_ld32(lane_base + kColSdP + buf * 128 + 64 + half * 32, dp);
-        tmem_wait_ld();
-        if (half == 1) {
-          // both halves are in registers: the MMA warp may overwrite this S/dP buffer
-          tc_fence_before_sync();
-          mbar_arrive(&sm.sdp_free[buf]);
-        }
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), sl2, neg_lse2));
-          float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), sl2, neg_lse2));
-          if (vis < kKT) {                    // diagonal / ragged tile only
-            if (half * 32 + 2 * i >= vis) p0 = 0.f;
-            if (half * 32 + 2 * i + 1 >= vis) p1 = 0.f;
-          }
-          const float d0 = p0 * fmaf(__uint_as_float(dp[2 * i]), dm.scale, neg_delta_s);
-          const float d1 = p1 * fmaf(__uint_as_float(dp[2 * i + 1]), dm.scale, neg_delta_s);
-          pk[half * 16 + i] = pack_bf16(p0, p1);
-          dk[half * 16 + i] = pack_bf16(d0, d1);
-        }
-      }
-      HGA_TRACE_POINT(12);
       if (s >= 2) {     // the GEMMs that read this P/dS buffer two steps ago must have finished
-        ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_free[buf], ((s - 2) >> 1) & 1, abort));
+        ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_free[wg], ((s - 2) >> 1) & 1, abort));
         if (!ok) break;
       }
       HGA_TRACE_POINT(13);
-      const uint32_t p_line = smem_u32(sm.p[buf]) + line, ds_line = smem_u32(sm.ds[buf]) + line;
+      const int vis = limit - kKT * j;
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {    // 8 chunks of 16 bytes (8 keys) per row, XOR-swizzled
-        const uint32_t off = ((uint32_t)c ^ key) * 16;
-        st_shared_v4(p_line + off, pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-        st_shared_v4(ds_line + off, dk[4 * c], dk[4 * c + 1], dk[4 * c + 2], dk[4 * c + 3]);
+      for (int q4 = 0; q4 < 4; ++q4) {               // 16 columns (keys) at a time: 128-register budget
+        uint32_t sv[16], dp[16];
+        tmem_ld16(sdp_addr + q4 * 16, sv);
+        tmem_ld16(sdp_addr + 64 + q4 * 16, dp);
+        tmem_wait_ld();
+        if (q4 == 3) {
+          // the whole S/dP tile is in registers: the MMA warp may overwrite this buffer
+          tc_fence_before_sync();
+          mbar_arrive(&sm.sdp_free[wg]);
+        }
+        uint32_t pk[8], dk[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), sl2, neg_lse2));
+          float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), sl2, neg_lse2));
+          if (vis < kKT) {                    // diagonal / ragged tile only
+            if (q4 * 16 + 2 * i >= vis) p0 = 0.f;
+            if (q4 * 16 + 2 * i + 1 >= vis) p1 = 0.f;
+          }
+          const float d0 = p0 * fmaf(__uint_as_float(dp[2 * i]), dm.scale, neg_delta_s);
+          const float d1 = p1 * fmaf(__uint_as_float(dp[2 * i + 1]), dm.scale, neg_delta_s);
+          pk[i] = pack_bf16(p0, p1);
+          dk[i] = pack_bf16(d0, d1);
+        }
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {      // two 16-byte chunks (8 keys each), XOR-swizzled
+          const uint32_t off = ((uint32_t)(2 * q4 + cc) ^ key) * 16;
+          if (s < n_active)                     // P feeds only the dV GEMM of active-key tiles
+            st_shared_v4(p_line + off, pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+          st_shared_v4(ds_line + off, dk[4 * cc], dk[4 * cc + 1], dk[4 * cc + 2], dk[4 * cc + 3]);
+        }
       }
       fence_proxy_async_smem();
-      mbar_arrive(&sm.pds_full[buf]);
+      mbar_arrive(&sm.pds_full[wg]);
       HGA_TRACE_POINT(14);
     }
     if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.dq_done, 0, abort));
     HGA_TRACE_POINT(20);
     if (ok) {
+      // dQ epilogue: each warpgroup writes half of the row (64 columns)
       tc_fence_after_sync();
-      uint16_t* qrow = dQ + b * dm.qs[0] + hq * dm.qs[1] + (int64_t)srow * dm.qs[2];
+      uint16_t* qrow = dQ + b * dm.qs[0] + hq * dm.qs[1] + (int64_t)srow * dm.qs[2] + wg * 64;
+      uint32_t x[2][32];
+      tmem_ld32(lane_base + kColDQ + wg * 64, x[0]);
+      tmem_ld32(lane_base + kColDQ + wg * 64 + 32, x[1]);
+      tmem_wait_ld();
 #pragma unroll
-      for (int c2 = 0; c2 < D / 64; ++c2) {
-        uint32_t x[2][32];
-        tmem_ld32(lane_base + kColDQ + c2 * 64, x[0]);
-        tmem_ld32(lane_base + kColDQ + c2 * 64 + 32, x[1]);
-        tmem_wait_ld();
+      for (int c = 0; c < 2; ++c) {
+        uint4* dst = reinterpret_cast<uint4*>(qrow + c * 32);
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint4* dst = reinterpret_cast<uint4*>(qrow + c2 * 64 + c * 32);
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            dst[i] = make_uint4(pack_bf16(__uint_as_float(x[c][8 * i]), __uint_as_float(x[c][8 * i + 1])),
-                                pack_bf16(__uint_as_float(x[c][8 * i + 2]), __uint_as_float(x[c][8 * i + 3])),
-                                pack_bf16(__uint_as_float(x[c][8 * i + 4]), __uint_as_float(x[c][8 * i + 5])),
-                                pack_bf16(__uint_as_float(x[c][8 * i + 6]), __uint_as_float(x[c][8 * i + 7])));
-        }
+        for (int i = 0; i < 4; ++i)
+          dst[i] = make_uint4(pack_bf16(__uint_as_float(x[c][8 * i]), __uint_as_float(x[c][8 * i + 1])),
+                              pack_bf16(__uint_as_float(x[c][8 * i + 2]), __uint_as_float(x[c][8 * i + 3])),
+                              pack_bf16(__uint_as_float(x[c][8 * i + 4]), __uint_as_float(x[c][8 * i + 5])),
+                              pack_bf16(__uint_as_float(x[c][8 * i + 6]), __uint_as_float(x[c][8 * i + 7])));
       }
     }
   } else {
