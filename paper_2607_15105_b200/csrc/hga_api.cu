@@ -179,17 +179,19 @@ int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* 
   if (!workspace || workspace_bytes < bwd_workspace_bytes(dm)) return HGA_ERR_WORKSPACE;
   if (!aligned16(workspace)) return HGA_ERR_ALIGN;
   cudaStream_t st = (cudaStream_t)stream;
-  if (!(dm.flags & HGA_FLAG_BWD_ACCUMULATE)) {
+  const bool zero_grads = !(dm.flags & HGA_FLAG_BWD_ACCUMULATE);
+  if (attn_bwd_sm100_supported(dm)) {
+    // zero-fills dK/dV itself where its kernels need it; UNSUPPORTED is returned before any launch
+    rc = launch_attn_bwd_sm100(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV, (float*)workspace,
+                               zero_grads, status_word, st);
+    if (rc != HGA_ERR_UNSUPPORTED) return rc;
+  }
+  if (zero_grads) {
     size_t bytes = (size_t)dm.B * dm.Hkv * dm.S * dm.d * sizeof(float);
     rc = record_cuda(cudaMemsetAsync(dK, 0, bytes, st));
     if (rc) return rc;
     rc = record_cuda(cudaMemsetAsync(dV, 0, bytes, st));
     if (rc) return rc;
-  }
-  if (attn_bwd_sm100_supported(dm)) {
-    rc = launch_attn_bwd_sm100(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV, (float*)workspace,
-                               status_word, st);
-    if (rc != HGA_ERR_UNSUPPORTED) return rc;
   }
   return launch_attn_bwd_generic(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV,
                                  (float*)workspace, status_word, st);

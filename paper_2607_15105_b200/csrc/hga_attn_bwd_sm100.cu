@@ -23,16 +23,11 @@
 // Shared memory: Q, dO (32 KB each), K ring (3 x 16 KB; a K tile is held until its dQ GEMM),
 // V ring (2 x 16 KB; a V tile is free once dP is issued), P and dS double buffered (4 x 16 KB), so
 // the row threads of tile s+1 never wait for the GEMMs that read P/dS of tile s.
+#include "hga_bwd_sm100.cuh"
 #include "hga_common.cuh"
 #include "hga_octets.cuh"
 #include "hga_sm100.cuh"
 
-// Optional phase timers: a profiling harness defines these three macros; otherwise no-ops.
-#ifndef HGA_TRACE_POINT
-#define HGA_TRACE_DECL
-#define HGA_TRACE_POINT(tag)
-#define HGA_TRACE_DUMP
-#endif
 
 namespace hga {
 
@@ -40,8 +35,8 @@ using namespace sm100;
 
 constexpr int kBwdThreads = 512;                // 16 warps: 128 registers per thread
 constexpr int kBwdProducers = 3;                // warps 0, 14, 15 issue the K/V copies
-constexpr int kBwdKStages = 3;
-constexpr int kBwdVStages = 2;
+constexpr int kBwdKStages = 4;
+constexpr int kBwdVStages = 3;
 constexpr int kBwdD = 128;
 constexpr int kKT = 64;                         // keys per tile
 constexpr int kOct = 8 * kBwdD * 2;             // bytes of one octet of K/V/Q/dO rows (2 panels)
@@ -53,33 +48,15 @@ struct BwdSmem {
   alignas(1024) uint8_t dO[128 * kBwdD * 2];
   alignas(1024) uint8_t k[kBwdKStages][kKvTile];
   alignas(1024) uint8_t v[kBwdVStages][kKvTile];
-  alignas(1024) uint8_t p[2][kPdsTile];         // [16 row octets][8 rows][128 B], 128-byte swizzle
-  alignas(1024) uint8_t ds[2][kPdsTile];
+  alignas(1024) uint8_t p[kPdsTile];            // [16 row octets][8 rows][128 B], 128-byte swizzle
+  alignas(1024) uint8_t ds[kPdsTile];           // (P and dS pass through shared memory only for dK/dV tiles)
   uint64_t q_full, k_full[kBwdKStages], k_empty[kBwdKStages], v_full[kBwdVStages], v_empty[kBwdVStages];
-  uint64_t sdp_full[2], sdp_free[2], pds_full[2], pds_free[2], dkv_full, dkv_free, dq_done;
+  uint64_t sdp_full[2], pds_full[2], dkv_full, dkv_free, dq_done, qdo_tmem;
   uint32_t tmem_base;
-  int n_oct, first_active;
+  int n_oct, dkv_lo, n_dkv;    // tiles [dkv_lo, dkv_lo + n_dkv) hold keys whose dK/dV this kernel adds
   volatile int abort;
   int oct_row[1];
 };
-
-__device__ __forceinline__ bool bwd_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
-  for (uint32_t i = 0; i < (1u << 20); ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && *abort) return false;
-  }
-  *abort = 1;
-  return false;
-}
-
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&h);
-}
 
 __device__ __forceinline__ float dot4_bf16(uint2 x, uint2 y) {
   float s = __uint_as_float(x.x << 16) * __uint_as_float(y.x << 16);
@@ -94,10 +71,11 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                  const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                  const float* __restrict__ delta_ws, const float* __restrict__ LSE, const int32_t* __restrict__ group_idx,
                  const int32_t* __restrict__ n_groups, Dims dm, uint16_t* __restrict__ dQ,
-                 float* __restrict__ dK, float* __restrict__ dV, int32_t* status_word) {
+                 float* __restrict__ dK, float* __restrict__ dV, int band_done, int32_t* status_word) {
   constexpr int D = kBwdD;
-  constexpr uint32_t kColSdP = 0;       // S[b] at 128*b, dP[b] at 128*b + 64
-  constexpr uint32_t kColDQ = 256, kColDV = 384, kColDK = 448;
+  constexpr uint32_t kColSdP = 0;       // S[b] at 128*b, dP[b] at 128*b + 64 (bf16 dS overwrites S[b])
+  constexpr uint32_t kColDV = 128, kColDK = 192;   // alias buffer 1, which the dK/dV steps leave idle
+  constexpr uint32_t kColDQ = 256, kColQ = 384, kColDO = 448;
   extern __shared__ uint8_t smem_raw[];
   BwdSmem& sm = *reinterpret_cast<BwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
@@ -115,11 +93,11 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     for (int s = 0; s < kBwdKStages; ++s) { mbar_init(&sm.k_full[s], kBwdProducers); mbar_init(&sm.k_empty[s], 1); }
     for (int s = 0; s < kBwdVStages; ++s) { mbar_init(&sm.v_full[s], kBwdProducers); mbar_init(&sm.v_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.sdp_full[s], 1); mbar_init(&sm.sdp_free[s], 128);
-      mbar_init(&sm.pds_full[s], 128); mbar_init(&sm.pds_free[s], 1);
+      mbar_init(&sm.sdp_full[s], 1);
+      mbar_init(&sm.pds_full[s], 128);
     }
     mbar_init(&sm.dkv_full, 1); mbar_init(&sm.dkv_free, 128);
-    mbar_init(&sm.dq_done, 1);
+    mbar_init(&sm.dq_done, 1); mbar_init(&sm.qdo_tmem, 256);
     sm.abort = 0;
     fence_barrier_init();
   }
@@ -144,16 +122,26 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     bool bad;   // invalid entries are skipped exactly as in the forward kernel (which reports them)
     const int n_oct = build_octet_table(dm, w, group_idx + (int64_t)item * dm.width, n_groups + item, sm.oct_row, &bad);
+    // Keys that receive dK/dV from this kernel: positions in [H, hi), where hi is the start of the
+    // local band when the key-major band kernel has already written that part, else no limit.
+    // Rows ascend, so these octets are a contiguous range [oa, ob) of the list.
+    const int hi = band_done ? w.ls : 0x7fffffff;
+    int below_h = 0, below_hi = 0;
+    for (int o = lane; o < n_oct; o += 32) {
+      const int row = sm.oct_row[o];
+      below_h += row + 8 <= dm.H;
+      below_hi += row < hi;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      below_h += __shfl_xor_sync(0xffffffffu, below_h, off);
+      below_hi += __shfl_xor_sync(0xffffffffu, below_hi, off);
+    }
     if (lane == 0) {
       sm.n_oct = n_oct;
-      // rows ascend, so the tiles holding active keys (position >= H) are a suffix
-      const int n_tiles = (n_oct + 7) / 8;
-      int fa = n_tiles;
-      for (int j = n_tiles - 1; j >= 0; --j) {
-        const int last = 8 * j + 7 < n_oct ? 8 * j + 7 : n_oct - 1;
-        if (sm.oct_row[last] + 8 > dm.H) fa = j; else break;
-      }
-      sm.first_active = fa;
+      const int oa = below_h, ob = below_hi;
+      sm.dkv_lo = oa / 8;
+      sm.n_dkv = ob > oa ? (ob + 7) / 8 - oa / 8 : 0;
     }
   }
   // Row threads: LSE and delta = rowsum(dO o O) of the thread's own row (delta comes from a
@@ -174,10 +162,18 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const int n_oct = sm.n_oct;
   const int n_keys = n_oct * 8;
   const int n_tiles = (n_oct + 7) / 8;
-  const int n_active = n_tiles - sm.first_active;   // steps 0 .. n_active-1 hold active-segment keys
+  const int n_active = sm.n_dkv;                    // steps 0 .. n_active-1 produce dK/dV
+  const int dkv_hi = sm.dkv_lo + n_active;
+  const int red_hi = band_done ? w.ls : 0x7fffffff;
+  // Step order: the dK/dV tiles first (descending), so their atomics drain while the rest is
+  // computed; then every other tile, descending.
+  auto tile_of_step = [&](int s) {
+    if (s < n_active) return dkv_hi - 1 - s;
+    const int j = n_tiles - 1 - (s - n_active);
+    return j >= dkv_hi ? j : j - n_active;
+  };
   volatile int* abort = &sm.abort;
   HGA_TRACE_POINT(1);
-  // step s (processing order) handles tile j = n_tiles - 1 - s (ascending key order)
 
   if (warp == 0 || warp >= 14) {
     // ------------------------------------------------------------------ producers
@@ -193,7 +189,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     bool ok = true;
     int issued = 0;
     for (int s = 0; s < n_tiles; ++s) {
-      const int j = n_tiles - 1 - s;
+      const int j = tile_of_step(s);
       const int ks = s % kBwdKStages, vs = s % kBwdVStages;
       const int o = 8 * j + oct_in_tile;
       const int row = o < n_oct ? sm.oct_row[o] : dm.L;    // past the list: zeros
@@ -231,90 +227,128 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);      // dS K-major, K tile MN-major
       constexpr uint32_t idesc_dkv = idesc_bf16_f32(D, kKT, 1, 1);     // both MN-major
       // Descriptors are built once; inside the loops an MMA costs two integer adds.
-      const uint64_t q_k = smem_desc_sw128(smem_u32(sm.q), 16, kOct);        // Q  as K-major A   (S)
-      const uint64_t do_k = smem_desc_sw128(smem_u32(sm.dO), 16, kOct);      // dO as K-major A   (dP)
+      const uint64_t q_k = smem_desc_sw128(smem_u32(sm.q), 16, kOct);        // Q  as K-major A   (S, dK/dV steps)
+      const uint64_t do_k = smem_desc_sw128(smem_u32(sm.dO), 16, kOct);      // dO as K-major A   (dP, dK/dV steps)
       const uint64_t q_mn = smem_desc_sw128(smem_u32(sm.q), 1024, kOct);     // Q^T  as MN-major A (dK^T)
       const uint64_t do_mn = smem_desc_sw128(smem_u32(sm.dO), 1024, kOct);   // dO^T as MN-major A (dV^T)
       const uint64_t k_k0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, kOct);    // K tile, K-major B  (S)
       const uint64_t v_k0 = smem_desc_sw128(smem_u32(sm.v[0]), 16, kOct);    // V tile, K-major B  (dP)
       const uint64_t k_mn0 = smem_desc_sw128(smem_u32(sm.k[0]), 1024, kOct); // K tile, MN-major B (dQ)
-      const uint64_t ds0 = smem_desc_sw128(smem_u32(sm.ds[0]), 16, 1024);    // dS: K-major A (dQ) and MN-major B (dK^T)
-      const uint64_t p0 = smem_desc_sw128(smem_u32(sm.p[0]), 16, 1024);      // P : MN-major B (dV^T)
-      auto issue_sdp = [&](int s) {
+      const uint64_t dsd = smem_desc_sw128(smem_u32(sm.ds), 16, 1024);       // dS: K-major A (dQ) and MN-major B (dK^T)
+      const uint64_t pd = smem_desc_sw128(smem_u32(sm.p), 16, 1024);         // P : MN-major B (dV^T)
+      // S and dP of step s into TMEM buffer `buf`; A from shared memory (dK/dV steps) or from the
+      // TMEM copies of Q and dO (all other steps: a third of the shared-memory operand traffic)
+      auto issue_sdp = [&](int s, uint32_t buf, bool a_in_tmem) {
         const uint64_t kd = desc_advance(k_k0, (uint32_t)(s % kBwdKStages) * kKvTile);
         const uint64_t vd = desc_advance(v_k0, (uint32_t)(s % kBwdVStages) * kKvTile);
-        const uint32_t s_acc = tmem + kColSdP + (s & 1) * 128;
+        const uint32_t s_acc = tmem + kColSdP + buf * 128;
+        if (a_in_tmem) {
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-          mma_ss(s_acc, desc_advance(q_k, off), desc_advance(kd, off), idesc_sdp, kk > 0);
-        }
+          for (int kk = 0; kk < D / 16; ++kk)
+            mma_ts(s_acc, tmem + kColQ + 8 * kk, desc_advance(kd, (kk >> 2) * 1024 + (kk & 3) * 32), idesc_sdp, kk > 0);
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-          mma_ss(s_acc + 64, desc_advance(do_k, off), desc_advance(vd, off), idesc_sdp, kk > 0);
+          for (int kk = 0; kk < D / 16; ++kk)
+            mma_ts(s_acc + 64, tmem + kColDO + 8 * kk, desc_advance(vd, (kk >> 2) * 1024 + (kk & 3) * 32), idesc_sdp, kk > 0);
+        } else {
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
+            mma_ss(s_acc, desc_advance(q_k, off), desc_advance(kd, off), idesc_sdp, kk > 0);
+          }
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
+            mma_ss(s_acc + 64, desc_advance(do_k, off), desc_advance(vd, off), idesc_sdp, kk > 0);
+          }
         }
-        mma_commit(&sm.sdp_full[s & 1]);
+        mma_commit(&sm.sdp_full[buf]);
         mma_commit(&sm.v_empty[s % kBwdVStages]);      // the V tile is only needed for dP
       };
-      bool ok = bwd_wait(&sm.q_full, 0, abort) && bwd_wait(&sm.k_full[0], 0, abort) &&
-                bwd_wait(&sm.v_full[0], 0, abort);
-      if (ok) {
+      auto wait_kv = [&](int s) {
+        return bwd_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1, abort) &&
+               bwd_wait(&sm.v_full[s % kBwdVStages], (s / kBwdVStages) & 1, abort);
+      };
+      bool ok = bwd_wait(&sm.q_full, 0, abort);
+      bool dq_started = false;
+      // ---- dK/dV steps: one at a time, buffer 0 only, every operand from shared memory.  The
+      // tensor pipe runs in issue order and a commit covers everything issued before it, so
+      // sdp_full of step s+1 also tells the row threads that the GEMMs reading P/dS of step s are done.
+      for (int s = 0; s < n_active && ok; ++s) {
+        ok = wait_kv(s);
+        if (!ok) break;
         tc_fence_after_sync();
-        issue_sdp(0);
+        issue_sdp(s, 0, false);
+        ok = bwd_wait(&sm.pds_full[0], s & 1, abort);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint64_t kmn = desc_advance(k_mn0, (uint32_t)(s % kBwdKStages) * kKvTile);
+#pragma unroll
+        for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per step
+          mma_ss(tmem + kColDQ, desc_advance(dsd, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
+                 (dq_started || kk > 0));
+        dq_started = true;
+        if (s > 0) {
+          ok = bwd_wait(&sm.dkv_free, (s - 1) & 1, abort);
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
+#pragma unroll
+        for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per step (2 row octets)
+          mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2 * kOct), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
+#pragma unroll
+        for (int kk = 0; kk < 128 / 16; ++kk)
+          mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2 * kOct), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
+        mma_commit(&sm.dkv_full);
+        mma_commit(&sm.k_empty[s % kBwdKStages]);
+        HGA_TRACE_POINT(4);
       }
-      HGA_TRACE_POINT(3);
-      for (int s = 0; s < n_tiles && ok; ++s) {
-        if (s + 1 < n_tiles) {
-          ok = bwd_wait(&sm.k_full[(s + 1) % kBwdKStages], ((s + 1) / kBwdKStages) & 1, abort) &&
-               bwd_wait(&sm.v_full[(s + 1) % kBwdVStages], ((s + 1) / kBwdVStages) & 1, abort);
-          HGA_TRACE_POINT(24);
-          // TMEM buffer (s+1)&1 held step s-1: its rows have been read once sdp_free completed
-          if (ok && s >= 1) ok = bwd_wait(&sm.sdp_free[(s + 1) & 1], ((s - 1) >> 1) & 1, abort);
+      // ---- all other steps: S/dP of step s+1 are issued before dQ of step s, into the other
+      // buffer; A operands come from TMEM (Q, dO copies; bf16 dS written over S by the row threads).
+      // Buffer i&1 is reused by step i+2 without a barrier: the row threads have finished with it
+      // before pds_full(i), and S/dP(i+2) follow dQ(i) in the in-order tensor pipe.
+      const int n_rest = n_tiles - n_active;
+      if (ok && n_rest > 0) {
+        ok = bwd_wait(&sm.qdo_tmem, 0, abort) && wait_kv(n_active);
+        if (ok) {
+          tc_fence_after_sync();
+          issue_sdp(n_active, 0, true);
+        }
+        HGA_TRACE_POINT(3);
+      }
+      for (int i = 0; i < n_rest && ok; ++i) {
+        const int s = n_active + i;
+        const uint32_t buf = (uint32_t)(i & 1);
+        if (i + 1 < n_rest) {
+          ok = wait_kv(s + 1);
+          // buffer 1 aliases the dK^T/dV^T accumulators: the reduction warps must have read the last ones
+          if (ok && i == 0 && n_active > 0) ok = bwd_wait(&sm.dkv_free, (n_active - 1) & 1, abort);
           if (!ok) break;
           tc_fence_after_sync();
           HGA_TRACE_POINT(6);
-          issue_sdp(s + 1);
+          issue_sdp(s + 1, buf ^ 1, true);
           HGA_TRACE_POINT(8);
         }
-        ok = bwd_wait(&sm.pds_full[s & 1], (s >> 1) & 1, abort);
+        // buffer 0 was also used by every dK/dV step
+        ok = bwd_wait(&sm.pds_full[buf], ((buf == 0 ? n_active : 0) + (i >> 1)) & 1, abort);
         if (!ok) break;
         tc_fence_after_sync();
         HGA_TRACE_POINT(5);
         const uint64_t kmn = desc_advance(k_mn0, (uint32_t)(s % kBwdKStages) * kKvTile);
-        const uint64_t dsd = desc_advance(ds0, (uint32_t)(s & 1) * kPdsTile);
 #pragma unroll
-        for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per step
-          mma_ss(tmem + kColDQ, desc_advance(dsd, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
-                 (s > 0 || kk > 0));
-        HGA_TRACE_POINT(7);
-        if (s < n_active) {
-          if (s > 0) {
-            ok = bwd_wait(&sm.dkv_free, (s - 1) & 1, abort);
-            if (!ok) break;
-            tc_fence_after_sync();
-          }
-          HGA_TRACE_POINT(9);
-          const uint64_t pd = desc_advance(p0, (uint32_t)(s & 1) * kPdsTile);
-#pragma unroll
-          for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per step (2 row octets)
-            mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2 * kOct), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
-#pragma unroll
-          for (int kk = 0; kk < 128 / 16; ++kk)
-            mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2 * kOct), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
-          mma_commit(&sm.dkv_full);
-          HGA_TRACE_POINT(4);
-        }
-        mma_commit(&sm.pds_free[s & 1]);
+        for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : dS (bf16) from TMEM, 8 columns per 16 keys
+          mma_ts(tmem + kColDQ, tmem + kColSdP + buf * 128 + 8 * kk, desc_advance(kmn, kk * 2 * kOct), idesc_dq,
+                 (dq_started || kk > 0));
+        dq_started = true;
         mma_commit(&sm.k_empty[s % kBwdKStages]);
+        HGA_TRACE_POINT(7);
       }
       if (ok) mma_commit(&sm.dq_done);
     }
   } else if (warp < 10) {
     // ------------------------------------------------------------------ one thread per query row
-    // Two warpgroups take alternate steps (warps 2-5 the even ones, 6-9 the odd ones), each with
-    // its own S/dP buffer in TMEM and its own P/dS buffer in shared memory, so the exp2 / dS work
-    // of step s+1 overlaps that of step s and the loop is paced by the tensor pipe.
+    // Warpgroup 0 (warps 2-5) takes the dK/dV steps and then the even ones of the remaining steps,
+    // warpgroup 1 (warps 6-9) the odd ones, each with its own S/dP buffer in TMEM, so the exp2 / dS
+    // work of one step overlaps the GEMMs of the next.
     const int wg = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int row_in_tile = quarter * 32 + lane;
@@ -330,20 +364,36 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // this row's 128-byte line inside the P / dS buffers, and its swizzle key
     const uint32_t line = (uint32_t)(row_in_tile >> 3) * 1024 + (uint32_t)(row_in_tile & 7) * 128;
     const uint32_t key = (uint32_t)(row_in_tile & 7);
-    const uint32_t p_line = smem_u32(sm.p[wg]) + line, ds_line = smem_u32(sm.ds[wg]) + line;
+    const uint32_t p_line = smem_u32(sm.p) + line, ds_line = smem_u32(sm.ds) + line;
     const uint32_t sdp_addr = lane_base + kColSdP + wg * 128;
-    bool ok = true;
-    for (int s = wg; s < n_tiles; s += 2) {          // buffer index s & 1 == wg
-      const int j = n_tiles - 1 - s;
-      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[wg], (s >> 1) & 1, abort));
+    bool ok = bwd_wait_warp(&sm.q_full, 0, abort);
+    if (ok) {
+      // TMEM copy of this row of Q (warpgroup 0) or dO (warpgroup 1): the A operand of S and dP.
+      // Row r = 8o + i lives at [octet o][panel][row i][128 B] with the 16-byte chunks XOR-swizzled by i.
+      const uint32_t src = smem_u32(wg == 0 ? sm.q : sm.dO) + (uint32_t)(row_in_tile >> 3) * kOct + key * 128;
+#pragma unroll
+      for (int pnl = 0; pnl < 2; ++pnl) {
+        uint32_t x[32];
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          ld_shared_v4(src + pnl * 1024 + (((uint32_t)c ^ key) * 16), x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]);
+        tmem_st32(lane_base + (wg == 0 ? kColQ : kColDO) + pnl * 32, x);
+      }
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(&sm.qdo_tmem);
+    }
+    uint32_t use = 0;                                 // completed phases of sdp_full[wg]
+    const int n_rest = n_tiles - n_active;
+    const int n_mine = wg == 0 ? n_active + (n_rest + 1) / 2 : n_rest / 2;
+    for (int u = 0; u < n_mine && ok; ++u) {
+      const bool dkv_step = wg == 0 && u < n_active;
+      const int s = dkv_step ? u : n_active + 2 * (u - (wg == 0 ? n_active : 0)) + wg;
+      const int j = tile_of_step(s);
+      ok = bwd_wait_warp(&sm.sdp_full[wg], use++ & 1, abort);
       if (!ok) break;
       tc_fence_after_sync();
       HGA_TRACE_POINT(11);
-      if (s >= 2) {     // the GEMMs that read this P/dS buffer two steps ago must have finished
-        ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_free[wg], ((s - 2) >> 1) & 1, abort));
-        if (!ok) break;
-      }
-      HGA_TRACE_POINT(13);
       const int vis = limit - kKT * j;
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {               // 16 columns (keys) at a time: 128-register budget
@@ -351,11 +401,6 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tmem_ld16(sdp_addr + q4 * 16, sv);
         tmem_ld16(sdp_addr + 64 + q4 * 16, dp);
         tmem_wait_ld();
-        if (q4 == 3) {
-          // the whole S/dP tile is in registers: the MMA warp may overwrite this buffer
-          tc_fence_before_sync();
-          mbar_arrive(&sm.sdp_free[wg]);
-        }
         uint32_t pk[8], dk[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -370,19 +415,29 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           pk[i] = pack_bf16(p0, p1);
           dk[i] = pack_bf16(d0, d1);
         }
+        if (dkv_step) {
+          // P and dS feed the dV^T / dK^T GEMMs as shared-memory operands
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {      // two 16-byte chunks (8 keys each), XOR-swizzled
-          const uint32_t off = ((uint32_t)(2 * q4 + cc) ^ key) * 16;
-          if (s < n_active)                     // P feeds only the dV GEMM of active-key tiles
+          for (int cc = 0; cc < 2; ++cc) {    // two 16-byte chunks (8 keys each), XOR-swizzled
+            const uint32_t off = ((uint32_t)(2 * q4 + cc) ^ key) * 16;
             st_shared_v4(p_line + off, pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-          st_shared_v4(ds_line + off, dk[4 * cc], dk[4 * cc + 1], dk[4 * cc + 2], dk[4 * cc + 3]);
+            st_shared_v4(ds_line + off, dk[4 * cc], dk[4 * cc + 1], dk[4 * cc + 2], dk[4 * cc + 3]);
+          }
+        } else {
+          // bf16 dS over the S columns already read (8 columns per 16 keys): the A operand of dQ
+          tmem_st8(sdp_addr + q4 * 8, dk);
         }
       }
-      fence_proxy_async_smem();
+      if (dkv_step) {
+        fence_proxy_async_smem();
+      } else {
+        tmem_wait_st();
+        tc_fence_before_sync();
+      }
       mbar_arrive(&sm.pds_full[wg]);
       HGA_TRACE_POINT(14);
     }
-    if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.dq_done, 0, abort));
+    if (ok) ok = bwd_wait_warp(&sm.dq_done, 0, abort);
     HGA_TRACE_POINT(20);
     if (ok) {
       // dQ epilogue: each warpgroup writes half of the row (64 columns)
@@ -412,8 +467,8 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     float* dVb = dV + ((int64_t)(b * dm.Hkv + h) * dm.S) * D + e;
     bool ok = true;
     for (int s = 0; s < n_active; ++s) {
-      const int j = n_tiles - 1 - s;
-      ok = __all_sync(0xffffffffu, bwd_wait(&sm.dkv_full, s & 1, abort));
+      const int j = tile_of_step(s);
+      ok = bwd_wait_warp(&sm.dkv_full, s & 1, abort);
       if (!ok) break;
       tc_fence_after_sync();
       HGA_TRACE_POINT(16);
@@ -432,7 +487,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const int o = 8 * j + half * 4 + (i >> 3);
           if (o < n_oct) {
             const int pos = sm.oct_row[o] + (i & 7);
-            if (pos >= dm.H) {            // warp-uniform: active-segment key
+            if (pos >= dm.H && pos < red_hi) {   // warp-uniform: a key this kernel owes dK/dV
               atomicAdd(dVb + (int64_t)(pos - dm.H) * D, __uint_as_float(gv[i]));
               atomicAdd(dKb + (int64_t)(pos - dm.H) * D, __uint_as_float(gk[i]));
             }
@@ -498,7 +553,7 @@ bool attn_bwd_sm100_supported(const Dims& dm) {
 int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
                           const float* LSE, const void* dO, const int32_t* group_idx,
                           const int32_t* n_groups, void* dQ, float* dK, float* dV, float* delta_ws,
-                          int32_t* status_word, cudaStream_t st) {
+                          bool zero_grads, int32_t* status_word, cudaStream_t st) {
   CUtensorMap mq, mdo, mk, mv;
   const uint32_t box[5] = {64, 8, 2, 1, 1};
   const uint64_t dq[5] = {64, (uint64_t)dm.S, 2, (uint64_t)dm.Hq, (uint64_t)dm.B};
@@ -523,9 +578,23 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
   k_bwd_delta_sm100<<<delta_blocks, 256, 0, st>>>((const uint16_t*)O, (const uint16_t*)dO, dm, delta_ws);
   e = cudaGetLastError();
   if (e != cudaSuccess) return record_cuda(e);
+  // dK/dV of the local band: written once per key tile by the key-major kernel (plain stores that
+  // cover every row of the active segment), which also makes zero-filling unnecessary.  Where that
+  // kernel does not apply, this kernel adds every contribution atomically onto zeroed buffers.
+  int band_done = 0;
+  if (attn_bwd_band_sm100_supported(dm)) {
+    const int rc = launch_attn_bwd_band_sm100(dm, Q, K, V, LSE, dO, dK, dV, delta_ws, status_word, st);
+    if (rc == HGA_OK) band_done = 1;
+    else if (rc != HGA_ERR_UNSUPPORTED) return rc;
+  }
+  if (!band_done && zero_grads) {
+    const size_t bytes = (size_t)dm.B * dm.Hkv * dm.S * dm.d * sizeof(float);
+    if ((e = cudaMemsetAsync(dK, 0, bytes, st)) != cudaSuccess) return record_cuda(e);
+    if ((e = cudaMemsetAsync(dV, 0, bytes, st)) != cudaSuccess) return record_cuda(e);
+  }
   const int units = dm.B * dm.Hkv * dm.NQB * (dm.rows / 128);
   k_attn_bwd_sm100<<<units, kBwdThreads, smem, st>>>(mq, mdo, mk, mv, delta_ws, LSE, group_idx, n_groups, dm,
-                                                    (uint16_t*)dQ, dK, dV, status_word);
+                                                    (uint16_t*)dQ, dK, dV, band_done, status_word);
   count_launch(2);
   return record_cuda(cudaGetLastError());
 }

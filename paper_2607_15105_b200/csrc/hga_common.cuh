@@ -83,7 +83,12 @@ bool attn_bwd_sm100_supported(const Dims& dm);
 int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
                           const float* LSE, const void* dO, const int32_t* group_idx,
                           const int32_t* n_groups, void* dQ, float* dK, float* dV, float* delta_ws,
-                          int32_t* status_word, cudaStream_t st);
+                          bool zero_grads, int32_t* status_word, cudaStream_t st);
+// Key-major dK/dV of the local band (plain stores covering every active-segment row).
+bool attn_bwd_band_sm100_supported(const Dims& dm);
+int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const float* LSE,
+                               const void* dO, float* dK, float* dV, const float* delta_ws, int32_t* status_word,
+                               cudaStream_t st);
 
 // Validates an hga_params block and fills the resolved description (hga_api.cu).
 int resolve_params(const hga_params* p, Dims& dm);
