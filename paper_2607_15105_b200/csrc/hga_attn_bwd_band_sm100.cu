@@ -235,12 +235,12 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
       const float neg_delta_s = -dl * dm.scale;
       const int vis_m = vis;
       if (m + 2 < n_steps) row_of(m + 2, lse, dl, vis);      // prefetch the next M-tile's row data
-      ok = bwd_wait_warp(&sm.sdp_full[wg], (m >> 1) & 1, abort);
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[wg], (m >> 1) & 1, abort));
       if (!ok) break;
       tc_fence_after_sync();
       HGA_TRACE_POINT(11);
       if (m >= 2) {     // the GEMMs that read this P/dS buffer two steps ago must have finished
-        ok = bwd_wait_warp(&sm.pds_free[wg], ((m >> 1) - 1) & 1, abort);
+        ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_free[wg], ((m >> 1) - 1) & 1, abort));
         if (!ok) break;
       }
 #pragma unroll
@@ -278,7 +278,7 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
       mbar_arrive(&sm.pds_full[wg]);
       HGA_TRACE_POINT(14);
     }
-    if (ok) ok = bwd_wait_warp(&sm.acc_done, 0, abort);
+    if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.acc_done, 0, abort));
     HGA_TRACE_POINT(20);
     if (ok) {
       // epilogue: thread = head_dim element (TMEM lane); a warp's store covers 128 contiguous bytes

@@ -3,40 +3,41 @@
 //
 // Work unit (one CTA): one 128-row M-tile of one item, swept over the item's routed keys in
 // 64-key tiles (8 octets, gathered by TMA exactly as in the forward kernel).  Per tile:
-//   S  = Q K^T          (smem x smem)  -> TMEM          dP = dO V^T     (smem x smem) -> TMEM
+//   S  = Q K^T, dP = dO V^T   (smem x smem)  -> one of three S/dP buffers in TMEM
 //   P  = 2^(S*c - LSE*log2e),  dS = scale * P o (dP - delta)            (one thread per row)
-//   dQ += dS K          (dS K-major from smem, K tile MN-major)          -> TMEM, kept for all tiles
-//   and, only for tiles that hold keys of the active segment (position >= H):
-//   dV^T = dO^T P,  dK^T = Q^T dS   (M = head_dim, N = 64 keys, K = 128 rows) -> TMEM
+//   dQ += dS K                (dS as bf16 in TMEM over the S columns, K tile MN-major from smem)
+// and, only for tiles holding keys whose dK/dV this kernel must add (keys of the active segment
+// selected through routing; the local band is written by k_attn_bwd_band_sm100; without that
+// kernel, every active key), P and dS also pass through shared memory for
+//   dV^T = dO^T P,  dK^T = Q^T dS   (M = head_dim, N = 64 keys, K = 128 rows) -> TMEM.
 // dK^T/dV^T are produced transposed so that a reduction warp's 32 lanes hold 32 consecutive
-// elements of one key row: its red.global.add.f32 is one coalesced 128-byte request.  History
-// tiles skip two of the five GEMMs and all atomics.
+// elements of one key row: its red.global.add.f32 is one coalesced 128-byte request.
 //
-// Tiles are processed in DESCENDING key order.  The keys of the active segment are a suffix of the
-// ascending key list, so their tiles come first and their atomics drain while the history tiles
-// are still being computed, instead of forming a tail at the end of the CTA.
+// The dK/dV tiles are processed first (their atomics drain while the rest is computed), then all
+// other tiles in descending key order.
 //
-// Warp roles (448 threads): warp 0 producer (TMA), warp 1 MMA issuer, warps 2-5 and 6-9 two
-// warpgroups of one thread per query row (P, dS, dQ epilogue) taking alternate tiles, warps 10-13
-// dK/dV reduction (thread = head_dim lane).
-// TMEM (512 columns): S[2] dP[2] (64 each, double buffered) | dQ 128 | dV^T 64 | dK^T 64.
-// Shared memory: Q, dO (32 KB each), K ring (3 x 16 KB; a K tile is held until its dQ GEMM),
-// V ring (2 x 16 KB; a V tile is free once dP is issued), P and dS double buffered (4 x 16 KB), so
-// the row threads of tile s+1 never wait for the GEMMs that read P/dS of tile s.
+// Warp roles (512 threads): warps 0 and 14 producers (TMA), warp 1 issues S/dP, warp 15 issues
+// dQ and dK^T/dV^T (two issuing threads, so neither hand-off stalls the other's GEMMs), warps 2-5
+// and 6-9 two warpgroups of one thread per query row taking alternate tiles (P, dS, dQ epilogue),
+// warps 10-13 dK/dV reduction (thread = head_dim lane).
+// TMEM (512 columns): S/dP buffer 0 | buffer 1 (aliased by dV^T, dK^T while dK/dV tiles run) |
+// dQ | buffer 2.  Shared memory: Q, dO (32 KB each), K ring (5 x 16 KB; a K tile is held until
+// its dQ GEMM), V ring (3 x 16 KB; a V tile is free once dP is done), P and dS (16 KB each).
 #include "hga_bwd_sm100.cuh"
 #include "hga_common.cuh"
 #include "hga_octets.cuh"
 #include "hga_sm100.cuh"
 
+#include <cstddef>
 
 namespace hga {
 
 using namespace sm100;
 
 constexpr int kBwdThreads = 512;                // 16 warps: 128 registers per thread
-constexpr int kBwdProducers = 3;                // warps 0, 14, 15 issue the K/V copies
-constexpr int kBwdKStages = 4;
-constexpr int kBwdVStages = 3;
+constexpr int kBwdProducers = 2;                // warps 0 and 14 issue the K/V copies
+constexpr int kBwdKStages = 5;                  // a K tile is held until its dQ GEMM is done
+constexpr int kBwdVStages = 3;                  // a V tile is free once dP is done
 constexpr int kBwdD = 128;
 constexpr int kKT = 64;                         // keys per tile
 constexpr int kOct = 8 * kBwdD * 2;             // bytes of one octet of K/V/Q/dO rows (2 panels)
@@ -51,7 +52,7 @@ struct BwdSmem {
   alignas(1024) uint8_t p[kPdsTile];            // [16 row octets][8 rows][128 B], 128-byte swizzle
   alignas(1024) uint8_t ds[kPdsTile];           // (P and dS pass through shared memory only for dK/dV tiles)
   uint64_t q_full, k_full[kBwdKStages], k_empty[kBwdKStages], v_full[kBwdVStages], v_empty[kBwdVStages];
-  uint64_t sdp_full[2], pds_full[2], dkv_full, dkv_free, dq_done, qdo_tmem;
+  uint64_t sdp_full[3], pds_full[3], buf_free[3], dkv_full, dkv_free, dq_done;
   uint32_t tmem_base;
   int n_oct, dkv_lo, n_dkv;    // tiles [dkv_lo, dkv_lo + n_dkv) hold keys whose dK/dV this kernel adds
   volatile int abort;
@@ -73,9 +74,10 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                  const int32_t* __restrict__ n_groups, Dims dm, uint16_t* __restrict__ dQ,
                  float* __restrict__ dK, float* __restrict__ dV, int band_done, int32_t* status_word) {
   constexpr int D = kBwdD;
-  constexpr uint32_t kColSdP = 0;       // S[b] at 128*b, dP[b] at 128*b + 64 (bf16 dS overwrites S[b])
+  // three S/dP buffers of 128 columns (S at +0, dP at +64; bf16 dS later overwrites S): 0, 128, 384
+  auto buf_col = [](uint32_t bf) -> uint32_t { return bf == 2 ? 384u : bf * 128u; };
   constexpr uint32_t kColDV = 128, kColDK = 192;   // alias buffer 1, which the dK/dV steps leave idle
-  constexpr uint32_t kColDQ = 256, kColQ = 384, kColDO = 448;
+  constexpr uint32_t kColDQ = 256;
   extern __shared__ uint8_t smem_raw[];
   BwdSmem& sm = *reinterpret_cast<BwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
@@ -92,12 +94,12 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     mbar_init(&sm.q_full, 1);
     for (int s = 0; s < kBwdKStages; ++s) { mbar_init(&sm.k_full[s], kBwdProducers); mbar_init(&sm.k_empty[s], 1); }
     for (int s = 0; s < kBwdVStages; ++s) { mbar_init(&sm.v_full[s], kBwdProducers); mbar_init(&sm.v_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.sdp_full[s], 1);
+    for (int s = 0; s < 3; ++s) {
+      mbar_init(&sm.sdp_full[s], 1); mbar_init(&sm.buf_free[s], 1);
       mbar_init(&sm.pds_full[s], 128);
     }
     mbar_init(&sm.dkv_full, 1); mbar_init(&sm.dkv_free, 128);
-    mbar_init(&sm.dq_done, 1); mbar_init(&sm.qdo_tmem, 256);
+    mbar_init(&sm.dq_done, 1);
     sm.abort = 0;
     fence_barrier_init();
   }
@@ -175,13 +177,13 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   volatile int* abort = &sm.abort;
   HGA_TRACE_POINT(1);
 
-  if (warp == 0 || warp >= 14) {
+  if (warp == 0 || warp == 14) {
     // ------------------------------------------------------------------ producers
     // Issuing one TMA box costs the issuing warp on the order of a hundred cycles, so the sixteen
-    // octet boxes of a step are spread over three warps: producer p takes octets p, p+3, p+6 of
-    // the K tile (lanes 0-2) and of the V tile (lanes 8-10).  Every producer arrives on the full
+    // octet boxes of a step are spread over two warps: producer p takes octets p, p+2, p+4, p+6 of
+    // the K tile (lanes 0-3) and of the V tile (lanes 8-11).  Every producer arrives on the full
     // barriers with the byte count of its own boxes.
-    const int pi = warp == 0 ? 0 : warp - 13;
+    const int pi = warp == 0 ? 0 : 1;
     const int sub = lane & 7;
     const int oct_in_tile = pi + kBwdProducers * sub;          // < 8 for the lanes that copy
     const bool k_lane = lane < 8 && oct_in_tile < 8, v_lane = lane >= 8 && lane < 16 && oct_in_tile < 8;
@@ -224,122 +226,103 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_sdp = idesc_bf16_f32(128, kKT, 0, 0);   // rows x keys, both K-major
-      constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);      // dS K-major, K tile MN-major
-      constexpr uint32_t idesc_dkv = idesc_bf16_f32(D, kKT, 1, 1);     // both MN-major
       // Descriptors are built once; inside the loops an MMA costs two integer adds.
       const uint64_t q_k = smem_desc_sw128(smem_u32(sm.q), 16, kOct);        // Q  as K-major A   (S, dK/dV steps)
       const uint64_t do_k = smem_desc_sw128(smem_u32(sm.dO), 16, kOct);      // dO as K-major A   (dP, dK/dV steps)
-      const uint64_t q_mn = smem_desc_sw128(smem_u32(sm.q), 1024, kOct);     // Q^T  as MN-major A (dK^T)
-      const uint64_t do_mn = smem_desc_sw128(smem_u32(sm.dO), 1024, kOct);   // dO^T as MN-major A (dV^T)
       const uint64_t k_k0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, kOct);    // K tile, K-major B  (S)
       const uint64_t v_k0 = smem_desc_sw128(smem_u32(sm.v[0]), 16, kOct);    // V tile, K-major B  (dP)
-      const uint64_t k_mn0 = smem_desc_sw128(smem_u32(sm.k[0]), 1024, kOct); // K tile, MN-major B (dQ)
-      const uint64_t dsd = smem_desc_sw128(smem_u32(sm.ds), 16, 1024);       // dS: K-major A (dQ) and MN-major B (dK^T)
-      const uint64_t pd = smem_desc_sw128(smem_u32(sm.p), 16, 1024);         // P : MN-major B (dV^T)
-      // S and dP of step s into TMEM buffer `buf`; A from shared memory (dK/dV steps) or from the
-      // TMEM copies of Q and dO (all other steps: a third of the shared-memory operand traffic)
-      auto issue_sdp = [&](int s, uint32_t buf, bool a_in_tmem) {
+      // Two threads feed the tensor pipe.  This one (warp 1) issues S and dP of every step and
+      // runs ahead as far as the three TMEM buffers allow; the other (warp 15) issues the GEMMs
+      // that consume the row threads' output (dQ, and dV^T/dK^T on dK/dV steps).  Neither waits
+      // for barriers that only concern the other.
+      // Step s uses buffer 0 while it is a dK/dV step, then buffers 0,1,2,0,... .
+      auto buf_of = [&](int s) -> uint32_t { return s < n_active ? 0u : (uint32_t)((s - n_active) % 3); };
+      auto use_of = [&](int s) {              // earlier uses of the buffer of step s
+        const int i = s - n_active;
+        return s < n_active ? s : (i % 3 == 0 ? n_active : 0) + i / 3;
+      };
+      auto wait_k = [&](int s) { return bwd_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1, abort); };
+      auto wait_v = [&](int s) { return bwd_wait(&sm.v_full[s % kBwdVStages], (s / kBwdVStages) & 1, abort); };
+      auto wait_buf = [&](int s) {
+        bool good = true;
+        // the GEMMs that read the previous contents of this buffer (dS, or P/dS in shared memory) are done
+        const int use = use_of(s);
+        if (use > 0) good = bwd_wait(&sm.buf_free[buf_of(s)], (use - 1) & 1, abort);
+        // buffer 1 aliases the dK^T/dV^T accumulators: the reduction warps must have read the last ones
+        if (good && n_active > 0 && s == n_active + 1) good = bwd_wait(&sm.dkv_free, (n_active - 1) & 1, abort);
+        return good;
+      };
+      bool ok = bwd_wait(&sm.q_full, 0, abort);
+      for (int s = 0; s < n_tiles && ok; ++s) {
+        const uint32_t buf = buf_of(s);
+        ok = wait_k(s) && wait_v(s) && wait_buf(s);
+        if (!ok) break;
+        tc_fence_after_sync();
+        HGA_TRACE_POINT(6);
         const uint64_t kd = desc_advance(k_k0, (uint32_t)(s % kBwdKStages) * kKvTile);
         const uint64_t vd = desc_advance(v_k0, (uint32_t)(s % kBwdVStages) * kKvTile);
-        const uint32_t s_acc = tmem + kColSdP + buf * 128;
-        if (a_in_tmem) {
+        const uint32_t s_acc = tmem + buf_col(buf);
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk)
-            mma_ts(s_acc, tmem + kColQ + 8 * kk, desc_advance(kd, (kk >> 2) * 1024 + (kk & 3) * 32), idesc_sdp, kk > 0);
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
+          mma_ss(s_acc, desc_advance(q_k, off), desc_advance(kd, off), idesc_sdp, kk > 0);
+        }
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk)
-            mma_ts(s_acc + 64, tmem + kColDO + 8 * kk, desc_advance(vd, (kk >> 2) * 1024 + (kk & 3) * 32), idesc_sdp, kk > 0);
-        } else {
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-            mma_ss(s_acc, desc_advance(q_k, off), desc_advance(kd, off), idesc_sdp, kk > 0);
-          }
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-            mma_ss(s_acc + 64, desc_advance(do_k, off), desc_advance(vd, off), idesc_sdp, kk > 0);
-          }
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
+          mma_ss(s_acc + 64, desc_advance(do_k, off), desc_advance(vd, off), idesc_sdp, kk > 0);
         }
         mma_commit(&sm.sdp_full[buf]);
         mma_commit(&sm.v_empty[s % kBwdVStages]);      // the V tile is only needed for dP
-      };
-      auto wait_kv = [&](int s) {
-        return bwd_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1, abort) &&
-               bwd_wait(&sm.v_full[s % kBwdVStages], (s / kBwdVStages) & 1, abort);
-      };
-      bool ok = bwd_wait(&sm.q_full, 0, abort);
-      bool dq_started = false;
-      // ---- dK/dV steps: one at a time, buffer 0 only, every operand from shared memory.  The
-      // tensor pipe runs in issue order and a commit covers everything issued before it, so
-      // sdp_full of step s+1 also tells the row threads that the GEMMs reading P/dS of step s are done.
-      for (int s = 0; s < n_active && ok; ++s) {
-        ok = wait_kv(s);
-        if (!ok) break;
-        tc_fence_after_sync();
-        issue_sdp(s, 0, false);
-        ok = bwd_wait(&sm.pds_full[0], s & 1, abort);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint64_t kmn = desc_advance(k_mn0, (uint32_t)(s % kBwdKStages) * kKvTile);
-#pragma unroll
-        for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per step
-          mma_ss(tmem + kColDQ, desc_advance(dsd, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
-                 (dq_started || kk > 0));
-        dq_started = true;
-        if (s > 0) {
-          ok = bwd_wait(&sm.dkv_free, (s - 1) & 1, abort);
-          if (!ok) break;
-          tc_fence_after_sync();
-        }
-#pragma unroll
-        for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per step (2 row octets)
-          mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2 * kOct), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
-#pragma unroll
-        for (int kk = 0; kk < 128 / 16; ++kk)
-          mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2 * kOct), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
-        mma_commit(&sm.dkv_full);
-        mma_commit(&sm.k_empty[s % kBwdKStages]);
-        HGA_TRACE_POINT(4);
+        HGA_TRACE_POINT(8);
       }
-      // ---- all other steps: S/dP of step s+1 are issued before dQ of step s, into the other
-      // buffer; A operands come from TMEM (Q, dO copies; bf16 dS written over S by the row threads).
-      // Buffer i&1 is reused by step i+2 without a barrier: the row threads have finished with it
-      // before pds_full(i), and S/dP(i+2) follow dQ(i) in the in-order tensor pipe.
-      const int n_rest = n_tiles - n_active;
-      if (ok && n_rest > 0) {
-        ok = bwd_wait(&sm.qdo_tmem, 0, abort) && wait_kv(n_active);
-        if (ok) {
-          tc_fence_after_sync();
-          issue_sdp(n_active, 0, true);
-        }
-        HGA_TRACE_POINT(3);
-      }
-      for (int i = 0; i < n_rest && ok; ++i) {
-        const int s = n_active + i;
-        const uint32_t buf = (uint32_t)(i & 1);
-        if (i + 1 < n_rest) {
-          ok = wait_kv(s + 1);
-          // buffer 1 aliases the dK^T/dV^T accumulators: the reduction warps must have read the last ones
-          if (ok && i == 0 && n_active > 0) ok = bwd_wait(&sm.dkv_free, (n_active - 1) & 1, abort);
-          if (!ok) break;
-          tc_fence_after_sync();
-          HGA_TRACE_POINT(6);
-          issue_sdp(s + 1, buf ^ 1, true);
-          HGA_TRACE_POINT(8);
-        }
-        // buffer 0 was also used by every dK/dV step
-        ok = bwd_wait(&sm.pds_full[buf], ((buf == 0 ? n_active : 0) + (i >> 1)) & 1, abort);
+    }
+  } else if (warp == 15) {
+    // ------------------------------------------------------------------ second MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);      // dS K-major, K tile MN-major
+      constexpr uint32_t idesc_dkv = idesc_bf16_f32(D, kKT, 1, 1);     // both MN-major
+      const uint64_t q_mn = smem_desc_sw128(smem_u32(sm.q), 1024, kOct);     // Q^T  as MN-major A (dK^T)
+      const uint64_t do_mn = smem_desc_sw128(smem_u32(sm.dO), 1024, kOct);   // dO^T as MN-major A (dV^T)
+      const uint64_t k_mn0 = smem_desc_sw128(smem_u32(sm.k[0]), 1024, kOct); // K tile, MN-major B (dQ)
+      const uint64_t dsd = smem_desc_sw128(smem_u32(sm.ds), 16, 1024);       // dS: K-major A (dQ) and MN-major B (dK^T)
+      const uint64_t pd = smem_desc_sw128(smem_u32(sm.p), 16, 1024);         // P : MN-major B (dV^T)
+      bool ok = true;
+      for (int s = 0; s < n_tiles && ok; ++s) {
+        const bool dkv_step = s < n_active;
+        const int i = s - n_active;
+        const uint32_t buf = dkv_step ? 0u : (uint32_t)(i % 3);
+        const int use = dkv_step ? s : (buf == 0 ? n_active : 0) + i / 3;
+        ok = bwd_wait(&sm.pds_full[buf], use & 1, abort);
         if (!ok) break;
         tc_fence_after_sync();
         HGA_TRACE_POINT(5);
         const uint64_t kmn = desc_advance(k_mn0, (uint32_t)(s % kBwdKStages) * kKvTile);
+        if (dkv_step) {
 #pragma unroll
-        for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : dS (bf16) from TMEM, 8 columns per 16 keys
-          mma_ts(tmem + kColDQ, tmem + kColSdP + buf * 128 + 8 * kk, desc_advance(kmn, kk * 2 * kOct), idesc_dq,
-                 (dq_started || kk > 0));
-        dq_started = true;
+          for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per MMA, dS from shared memory
+            mma_ss(tmem + kColDQ, desc_advance(dsd, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
+                   (s > 0 || kk > 0));
+          if (s > 0) {
+            ok = bwd_wait(&sm.dkv_free, (s - 1) & 1, abort);
+            if (!ok) break;
+            tc_fence_after_sync();
+          }
+#pragma unroll
+          for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per MMA (2 row octets)
+            mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2 * kOct), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
+#pragma unroll
+          for (int kk = 0; kk < 128 / 16; ++kk)
+            mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2 * kOct), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
+          mma_commit(&sm.dkv_full);
+        } else {
+#pragma unroll
+          for (int kk = 0; kk < kKT / 16; ++kk)   // dS (bf16) from TMEM, 8 columns per 16 keys
+            mma_ts(tmem + kColDQ, tmem + buf_col(buf) + 8 * kk, desc_advance(kmn, kk * 2 * kOct), idesc_dq,
+                   (s > 0 || kk > 0));
+        }
         mma_commit(&sm.k_empty[s % kBwdKStages]);
+        mma_commit(&sm.buf_free[buf]);
         HGA_TRACE_POINT(7);
       }
       if (ok) mma_commit(&sm.dq_done);
@@ -365,32 +348,18 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t line = (uint32_t)(row_in_tile >> 3) * 1024 + (uint32_t)(row_in_tile & 7) * 128;
     const uint32_t key = (uint32_t)(row_in_tile & 7);
     const uint32_t p_line = smem_u32(sm.p) + line, ds_line = smem_u32(sm.ds) + line;
-    const uint32_t sdp_addr = lane_base + kColSdP + wg * 128;
-    bool ok = bwd_wait_warp(&sm.q_full, 0, abort);
-    if (ok) {
-      // TMEM copy of this row of Q (warpgroup 0) or dO (warpgroup 1): the A operand of S and dP.
-      // Row r = 8o + i lives at [octet o][panel][row i][128 B] with the 16-byte chunks XOR-swizzled by i.
-      const uint32_t src = smem_u32(wg == 0 ? sm.q : sm.dO) + (uint32_t)(row_in_tile >> 3) * kOct + key * 128;
-#pragma unroll
-      for (int pnl = 0; pnl < 2; ++pnl) {
-        uint32_t x[32];
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-          ld_shared_v4(src + pnl * 1024 + (((uint32_t)c ^ key) * 16), x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]);
-        tmem_st32(lane_base + (wg == 0 ? kColQ : kColDO) + pnl * 32, x);
-      }
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(&sm.qdo_tmem);
-    }
-    uint32_t use = 0;                                 // completed phases of sdp_full[wg]
+    bool ok = true;
     const int n_rest = n_tiles - n_active;
     const int n_mine = wg == 0 ? n_active + (n_rest + 1) / 2 : n_rest / 2;
     for (int u = 0; u < n_mine && ok; ++u) {
       const bool dkv_step = wg == 0 && u < n_active;
       const int s = dkv_step ? u : n_active + 2 * (u - (wg == 0 ? n_active : 0)) + wg;
+      const int i = s - n_active;
+      const uint32_t buf = dkv_step ? 0u : (uint32_t)(i % 3);
+      const int use = dkv_step ? s : (buf == 0 ? n_active : 0) + i / 3;     // earlier uses of buf
+      const uint32_t sdp_addr = lane_base + buf_col(buf);
       const int j = tile_of_step(s);
-      ok = bwd_wait_warp(&sm.sdp_full[wg], use++ & 1, abort);
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[buf], use & 1, abort));
       if (!ok) break;
       tc_fence_after_sync();
       HGA_TRACE_POINT(11);
@@ -434,10 +403,10 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tmem_wait_st();
         tc_fence_before_sync();
       }
-      mbar_arrive(&sm.pds_full[wg]);
+      mbar_arrive(&sm.pds_full[buf]);
       HGA_TRACE_POINT(14);
     }
-    if (ok) ok = bwd_wait_warp(&sm.dq_done, 0, abort);
+    if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.dq_done, 0, abort));
     HGA_TRACE_POINT(20);
     if (ok) {
       // dQ epilogue: each warpgroup writes half of the row (64 columns)
@@ -468,7 +437,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     bool ok = true;
     for (int s = 0; s < n_active; ++s) {
       const int j = tile_of_step(s);
-      ok = bwd_wait_warp(&sm.dkv_full, s & 1, abort);
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.dkv_full, s & 1, abort));
       if (!ok) break;
       tc_fence_after_sync();
       HGA_TRACE_POINT(16);
@@ -567,7 +536,8 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
       encode_tensor_map_bf16(&mk, K, 5, dk, sk, box, true) ||
       encode_tensor_map_bf16(&mv, V, 5, dk, sv, box, true))
     return HGA_ERR_UNSUPPORTED;
-  const size_t smem = sizeof(BwdSmem) + sizeof(int) * (max_routed_tokens(dm) / 8 + 8) + 1024;
+  // the octet table starts inside the struct's tail padding; 1024 bytes of slack for the manual alignment
+  const size_t smem = offsetof(BwdSmem, oct_row) + sizeof(int) * (max_routed_tokens(dm) / 8 + 8) + 1024;
   if (smem > 227 * 1024) return HGA_ERR_UNSUPPORTED;
   cudaError_t e = cudaFuncSetAttribute(k_attn_bwd_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return record_cuda(e);

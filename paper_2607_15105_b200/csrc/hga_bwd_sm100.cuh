@@ -26,15 +26,6 @@ __device__ __forceinline__ bool bwd_wait(uint64_t* bar, uint32_t parity, volatil
   return false;
 }
 
-// Whole-warp wait: one lane polls, the result is broadcast (the shuffle also reconverges the warp).
-// Polling from all 32 lanes multiplies the barrier traffic in shared memory, which slows every
-// other barrier operation of the CTA.
-__device__ __forceinline__ bool bwd_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort) {
-  int ok = 1;
-  if ((threadIdx.x & 31) == 0) ok = bwd_wait(bar, parity, abort);
-  return __shfl_sync(0xffffffffu, ok, 0) != 0;
-}
-
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
