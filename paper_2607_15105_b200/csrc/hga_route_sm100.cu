@@ -4,8 +4,7 @@
 // Scores are max over the item's G*Bq query rows of q . summary.  The GEMM puts 128 summaries
 // on the MMA M dimension (= TMEM lanes) and up to 256 query rows on N (= TMEM columns), so the
 // maximum over rows is an in-thread reduction over the columns a thread reads back with
-// tcgen05.ld: thread = summary.  Two accumulators of 256 columns alternate, so reading one
-// overlaps the MMAs of the next.
+// tcgen05.ld: thread = summary.
 //   phase 1  candidate chunk summaries, 128 per tile, streamed by TMA (octets of 8 rows)
 //   select   k_c rounds of block arg-max on packed (orderable score, ~index) keys: highest score,
 //            ties to the lowest index; the winners are then ordered ascending
@@ -22,12 +21,18 @@ namespace hga {
 using namespace sm100;
 
 constexpr int kRtThreads = 320;     // warp 0 producer, warp 1 MMA, warps 2-5 readers, 6-9 help in select
+// One summary-tile stage and one accumulator per CTA: an item has only a few tiles, so there is
+// little to pipeline inside a CTA; the smaller footprint (under half of the shared memory and of
+// TMEM) lets two CTAs share an SM, and the serial phases of one item overlap the GEMMs of another.
+constexpr int kRtStages = 1;
+constexpr int kRtAccs = 1;
+constexpr int kRtTmemCols = 256 * kRtAccs;
 
 template <int D>
 struct RouteSmem {
   static constexpr int kTile = 128 * D * 2;
-  alignas(1024) uint8_t a[2][kTile];           // summary tiles (A operand), 2 stages
-  uint64_t q_full, a_full[2], a_empty[2], acc_full[2], acc_free[2];
+  alignas(1024) uint8_t a[kRtStages][kTile];   // summary tiles (A operand)
+  uint64_t q_full, a_full[kRtStages], a_empty[kRtStages], acc_full[kRtAccs], acc_free[kRtAccs];
   uint32_t tmem_base;
   volatile int abort;
   int n_sel;
@@ -52,7 +57,7 @@ __device__ __forceinline__ uint32_t rt_orderable(float f) {
 }
 
 template <int D>
-__global__ void __launch_bounds__(kRtThreads, 1)
+__global__ void __launch_bounds__(kRtThreads, 2)
 k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_cs,
               const __grid_constant__ CUtensorMap map_gs, Dims dm, int32_t* __restrict__ chunk_idx,
               int32_t* __restrict__ group_idx, int32_t* __restrict__ n_groups,
@@ -81,16 +86,14 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.a_full[s], 1); mbar_init(&sm.a_empty[s], 1);
-      mbar_init(&sm.acc_full[s], 1); mbar_init(&sm.acc_free[s], 128);
-    }
+    for (int s = 0; s < kRtStages; ++s) { mbar_init(&sm.a_full[s], 1); mbar_init(&sm.a_empty[s], 1); }
+    for (int s = 0; s < kRtAccs; ++s) { mbar_init(&sm.acc_full[s], 1); mbar_init(&sm.acc_free[s], 128); }
     sm.abort = 0;
     sm.n_sel = 0;
     fence_barrier_init();
   }
   if (warp == 1) {
-    tmem_alloc(&sm.tmem_base, 512);
+    tmem_alloc(&sm.tmem_base, kRtTmemCols);
     tmem_relinquish();
   }
   if (warp == 0 && lane == 0) {
@@ -117,7 +120,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       }
       bool ok = true;
       for (int t = 0; t < n_tiles; ++t) {
-        const int tg = t_begin + t, s = tg & 1, use = tg >> 1;
+        const int tg = t_begin + t, s = tg % kRtStages, use = tg / kRtStages;
         if (lane == 0 && use > 0) ok = rt_wait(&sm.a_empty[s], (use - 1) & 1, abort);
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
@@ -141,10 +144,10 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const uint32_t idesc = idesc_bf16_f32(128, rows_half, 0, 0);
         bool ok = phase2 ? true : rt_wait(&sm.q_full, 0, abort);
         for (int t = 0; t < n_tiles && ok; ++t) {
-          const int tg = t_begin + t, s = tg & 1;
-          ok = rt_wait(&sm.a_full[s], (tg >> 1) & 1, abort);
+          const int tg = t_begin + t, s = tg % kRtStages;
+          ok = rt_wait(&sm.a_full[s], (tg / kRtStages) & 1, abort);
           for (int hf = 0; hf < n_halves && ok; ++hf) {
-            const int step = tg * n_halves + hf, buf = step & 1, use = step >> 1;
+            const int step = tg * n_halves + hf, buf = step % kRtAccs, use = step / kRtAccs;
             if (use > 0) ok = rt_wait(&sm.acc_free[buf], (use - 1) & 1, abort);
             if (!ok) break;
             tc_fence_after_sync();
@@ -171,8 +174,8 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const int tg = t_begin + t;
         float best = -FLT_MAX;
         for (int hf = 0; hf < n_halves; ++hf) {
-          const int step = tg * n_halves + hf, buf = step & 1;
-          ok = __all_sync(0xffffffffu, rt_wait(&sm.acc_full[buf], (step >> 1) & 1, abort));
+          const int step = tg * n_halves + hf, buf = step % kRtAccs;
+          ok = __all_sync(0xffffffffu, rt_wait(&sm.acc_full[buf], (step / kRtAccs) & 1, abort));
           if (!ok) break;
           tc_fence_after_sync();
           for (int c = 0; c < rows_half; c += 32) {
@@ -211,32 +214,57 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 
   // ---------------------------------------------------------------------- chunk top-k
   if (!sm.abort) {
-    for (int r = 0; r < k_sel; ++r) {
-      unsigned long long best = 0;
-      for (int i = tid; i < n_cand; i += kRtThreads) best = keys[i] > best ? keys[i] : best;
+    if (n_cand <= 2 * kRtThreads) {
+      // Few candidates: rank every key by counting the larger ones (keys are distinct, the index
+      // is part of the key), no rounds and no block-wide arg-max.  A candidate is selected when
+      // fewer than k_sel keys beat it; its place in the ascending output is the number of selected
+      // candidates with a lower index.
+      unsigned long long* flags = reinterpret_cast<unsigned long long*>(sm.sel);   // bit i: candidate i selected
+      for (int i = tid; i < (n_cand + 63) / 64; i += kRtThreads) flags[i] = 0;
+      __syncthreads();
+      for (int i = tid; i < n_cand; i += kRtThreads) {
+        const unsigned long long mine = keys[i];
+        int beat = 0;
+        for (int q = 0; q < n_cand; ++q) beat += keys[q] > mine;
+        if (beat < k_sel) atomicOr(&flags[i >> 6], 1ull << (i & 63));
+      }
+      __syncthreads();
+      for (int i = tid; i < n_cand; i += kRtThreads) {
+        if ((flags[i >> 6] >> (i & 63)) & 1ull) {
+          int pos = __popcll(flags[i >> 6] & ((1ull << (i & 63)) - 1));
+          for (int q = 0; q < (i >> 6); ++q) pos += __popcll(flags[q]);
+          sm.sorted[pos] = j0 + i;
+        }
+      }
+      __syncthreads();
+    } else {
+      for (int r = 0; r < k_sel; ++r) {
+        unsigned long long best = 0;
+        for (int i = tid; i < n_cand; i += kRtThreads) best = keys[i] > best ? keys[i] : best;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-        best = other > best ? other : best;
+        for (int o = 16; o > 0; o >>= 1) {
+          const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+          best = other > best ? other : best;
+        }
+        if (lane == 0) sm.warp_best[warp] = best;
+        __syncthreads();
+        if (tid == 0) {
+          for (int q = 1; q < kRtThreads / 32; ++q) best = sm.warp_best[q] > best ? sm.warp_best[q] : best;
+          const int j = 0x7fffffff - (int)(uint32_t)(best & 0xffffffffu);
+          sm.sel[r] = j;
+          keys[j - j0] = 0;                                  // taken
+        }
+        __syncthreads();
       }
-      if (lane == 0) sm.warp_best[warp] = best;
-      __syncthreads();
-      if (tid == 0) {
-        for (int q = 1; q < kRtThreads / 32; ++q) best = sm.warp_best[q] > best ? sm.warp_best[q] : best;
-        const int j = 0x7fffffff - (int)(uint32_t)(best & 0xffffffffu);
-        sm.sel[r] = j;
-        keys[j - j0] = 0;                                  // taken
+      // ascending order by counting ranks (indices are distinct)
+      for (int i = tid; i < k_sel; i += kRtThreads) {
+        const int v = sm.sel[i];
+        int rank = 0;
+        for (int q = 0; q < k_sel; ++q) rank += sm.sel[q] < v;
+        sm.sorted[rank] = v;
       }
       __syncthreads();
     }
-    // ascending order by counting ranks (indices are distinct)
-    for (int i = tid; i < k_sel; i += kRtThreads) {
-      const int v = sm.sel[i];
-      int rank = 0;
-      for (int q = 0; q < k_sel; ++q) rank += sm.sel[q] < v;
-      sm.sorted[rank] = v;
-    }
-    __syncthreads();
     for (int i = tid; i < dm.kc; i += kRtThreads)
       chunk_idx[(int64_t)item * dm.kc + i] = i < k_sel ? sm.sorted[i] : -1;
   }
@@ -275,7 +303,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   __syncthreads();
   if (warp == 1) {
     __syncwarp();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(tmem, kRtTmemCols);
   }
 }
 
@@ -319,6 +347,9 @@ static int launch_route(const Dims& dm, const void* Q, const void* chunk_sum, co
   const int max_cand = route_max_cand(dm);
   const size_t smem = route_sm100_smem(dm, max_cand);
   cudaError_t e = cudaFuncSetAttribute(k_route_sm100<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return record_cuda(e);
+  // two CTAs per SM need the largest shared-memory carve-out
+  e = cudaFuncSetAttribute(k_route_sm100<D>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
   if (e != cudaSuccess) return record_cuda(e);
   const int items = dm.B * dm.Hkv * dm.NQB;
   k_route_sm100<D><<<items, kRtThreads, smem, st>>>(mq, mc, mg, dm, chunk_idx, group_idx, n_groups, chunk_scores,
