@@ -82,9 +82,10 @@ def active_group_pairs(cfg, group_idx, n_groups):
     return n * cfg.group * cfg.gqa * cfg.q_block
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the call's main kernel, from the ncu
-# captures summarised under profiles/ (k_attn_fwd_sm100_cfg3_16k.md, k_attn_bwd_sm100_cfg3_16k.md).
-NCU_TRAFFIC_BYTES = {3: {"hga_attn_fwd": 63.56e6, "hga_attn_bwd": 104.89e6}}
+# dram__bytes_read.sum + dram__bytes_write.sum per call, summed over the call's kernels, from the
+# ncu captures summarised under profiles/ (forward: k_attn_fwd_sm100; backward: k_bwd_delta_sm100
+# 33.58 MB + k_attn_bwd_band_sm100 42.94 MB + k_attn_bwd_sm100 88.62 MB).
+NCU_TRAFFIC_BYTES = {3: {"hga_attn_fwd": 64.08e6, "hga_attn_bwd": 165.14e6}}
 
 
 def roofline_entry(name, flops, nbytes, seconds, peaks, sustained=False):
