@@ -1,28 +1,41 @@
 // hga_attn_bwd for sm_100a (head_dim 128): backward of routed exact-token attention with the
 // routing frozen (Section 2.1, last paragraph) and history K/V detached (Section 2.2).
 //
-// Work unit (one CTA): one 128-row M-tile of one item, swept over the item's routed keys in
-// 64-key tiles (8 octets, gathered by TMA exactly as in the forward kernel).  Per tile:
-//   S  = Q K^T, dP = dO V^T   (smem x smem)  -> one of three S/dP buffers in TMEM
-//   P  = 2^(S*c - LSE*log2e),  dS = scale * P o (dP - delta)            (one thread per row)
-//   dQ += dS K                (dS as bf16 in TMEM over the S columns, K tile MN-major from smem)
-// and, only for tiles holding keys whose dK/dV this kernel must add (keys of the active segment
-// selected through routing; the local band is written by k_attn_bwd_band_sm100; without that
-// kernel, every active key), P and dS also pass through shared memory for
-//   dV^T = dO^T P,  dK^T = Q^T dS   (M = head_dim, N = 64 keys, K = 128 rows) -> TMEM.
-// dK^T/dV^T are produced transposed so that a reduction warp's 32 lanes hold 32 consecutive
-// elements of one key row: its red.global.add.f32 is one coalesced 128-byte request.
+// Work unit (one CTA): one 128-row M-tile of one item, swept over the item's routed keys, which
+// TMA gathers in 64-key tiles (8 octets) exactly as in the forward kernel.  Two kinds of steps:
 //
-// The dK/dV tiles are processed first (their atomics drain while the rest is computed), then all
-// other tiles in descending key order.
+//  * dK/dV steps (one 64-key tile each): tiles that hold keys whose dK/dV this kernel must add,
+//    i.e. keys of the active segment that were selected through routing (the local band is written
+//    by the key-major kernel k_attn_bwd_band_sm100; without it, every active key).  They come first:
+//      S = Q K^T, dP = dO V^T -> TMEM;  P, dS by one thread per row -> shared memory;
+//      dQ += dS K;  dV^T = dO^T P, dK^T = Q^T dS (M = head_dim, N = 64 keys, K = 128 rows) -> TMEM,
+//    then four reduction warps add the transposed tiles to global memory (a warp's 32 lanes hold 32
+//    consecutive elements of one key row: one coalesced 128-byte red.global.add.f32 request).
 //
-// Warp roles (512 threads): warps 0 and 14 producers (TMA), warp 1 issues S/dP, warp 15 issues
-// dQ and dK^T/dV^T (two issuing threads, so neither hand-off stalls the other's GEMMs), warps 2-5
-// and 6-9 two warpgroups of one thread per query row taking alternate tiles (P, dS, dQ epilogue),
-// warps 10-13 dK/dV reduction (thread = head_dim lane).
-// TMEM (512 columns): S/dP buffer 0 | buffer 1 (aliased by dV^T, dK^T while dK/dV tiles run) |
-// dQ | buffer 2.  Shared memory: Q, dO (32 KB each), K ring (5 x 16 KB; a K tile is held until
-// its dQ GEMM), V ring (3 x 16 KB; a V tile is free once dP is done), P and dS (16 KB each).
+//  * all other steps run on PAIRS of tiles (128 keys), because a tcgen05.mma with N = 64 runs at
+//    little more than half the rate of one with N = 128:
+//      S(u)  = Q K^T   (N = 128: two adjacent ring stages are one B operand)  -> TMEM region
+//      dP(u) = dO V^T                                                          -> TMEM region
+//      phase 1 of the row threads: P = 2^(S*c - LSE*log2e), kept as packed bf16 in registers;
+//      phase 2: dS = scale * P o (dP - delta), written as bf16 over the dP columns already read;
+//      dQ += dS K      (A = dS from TMEM, B = the two K stages, MN-major).
+//    Three 128-column TMEM regions rotate: S(u+1) is issued while the row threads still work on
+//    step u, dP(u+1) goes into S(u)'s region as soon as they are done with it, and dQ(u) follows; so
+//    the exp2 of step u+1 overlaps the dP GEMM of step u+1, and the tensor pipe never waits for the
+//    row threads except for that one hand-off.  The in-order tensor pipe makes the other hazards
+//    (dQ(u) reads dS before S(u+2) overwrites it) free of barriers.
+//
+// Warp roles (512 threads): warp 0 copies K tiles and runs up to three pairs ahead, warps 14 and 15
+// copy V tiles (half of each tile; V has room for one pair only, refilled as soon as the dP GEMM of
+// the previous pair is done, so their issue time matters), warp 1 MMA issuer, warps 2-5 and 6-9
+// one thread per query row (warpgroup 0: first tile of a pair and all dK/dV steps; warpgroup 1:
+// second tile of a pair; both write the dQ epilogue), warps 10-13 dK/dV reduction.
+// Every barrier hand-off costs the MMA thread a few hundred cycles and every tcgen05.commit about a
+// hundred, so a paired step has one full barrier per operand and pair, and the dP commit doubles as
+// the V stages' release.
+// TMEM (512 columns): region 0 | region 2 (aliased by dV^T, dK^T during the dK/dV steps) | dQ |
+// region 1.  Shared memory: Q, dO (32 KB each), K ring of six 16 KB stages, V ring of two, P and dS
+// (16 KB each, used by the dK/dV steps only).
 #include "hga_bwd_sm100.cuh"
 #include "hga_common.cuh"
 #include "hga_octets.cuh"
@@ -35,9 +48,8 @@ namespace hga {
 using namespace sm100;
 
 constexpr int kBwdThreads = 512;                // 16 warps: 128 registers per thread
-constexpr int kBwdProducers = 2;                // warps 0 and 14 issue the K/V copies
-constexpr int kBwdKStages = 5;                  // a K tile is held until its dQ GEMM is done
-constexpr int kBwdVStages = 3;                  // a V tile is free once dP is done
+constexpr int kBwdKStages = 6;                  // K ring: three pairs (a K tile is held until its dQ GEMM)
+constexpr int kBwdVStages = 2;                  // V ring: one pair (a V tile is free once dP is done)
 constexpr int kBwdD = 128;
 constexpr int kKT = 64;                         // keys per tile
 constexpr int kOct = 8 * kBwdD * 2;             // bytes of one octet of K/V/Q/dO rows (2 panels)
@@ -52,9 +64,15 @@ struct BwdSmem {
   alignas(1024) uint8_t p[kPdsTile];            // [16 row octets][8 rows][128 B], 128-byte swizzle
   alignas(1024) uint8_t ds[kPdsTile];           // (P and dS pass through shared memory only for dK/dV tiles)
   uint64_t q_full, k_full[kBwdKStages], k_empty[kBwdKStages], v_full[kBwdVStages], v_empty[kBwdVStages];
-  uint64_t sdp_full[3], pds_full[3], buf_free[3], dkv_full, dkv_free, dq_done;
+  uint64_t sdp_full, pds_full, dkv_full, dkv_free;      // dK/dV steps
+  uint64_t s_full[2], dp_full[4], ds_full;              // paired steps (S(u+1) is committed before step u is over: two barriers;
+                                                        // dP: four, so that a copy item taken ahead of time cannot mistake an older phase)
+  uint64_t phase_a_done;                                // every GEMM of the dK/dV steps is complete
+  uint64_t kp_full[kBwdKStages / 2], kp_empty[kBwdKStages], vp_full;       // paired steps: one barrier per pair of stages
+                                                        // (kp_empty: indexed by pair number mod 6, see dp_full)
+  uint64_t dq_done;
   uint32_t tmem_base;
-  int n_oct, dkv_lo, n_dkv;    // tiles [dkv_lo, dkv_lo + n_dkv) hold keys whose dK/dV this kernel adds
+  int n_oct, dkv_lo, n_dkv;    // tiles [dkv_lo, dkv_lo + n_dkv) are processed as dK/dV steps
   volatile int abort;
   int oct_row[1];
 };
@@ -74,10 +92,12 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                  const int32_t* __restrict__ n_groups, Dims dm, uint16_t* __restrict__ dQ,
                  float* __restrict__ dK, float* __restrict__ dV, int band_done, int32_t* status_word) {
   constexpr int D = kBwdD;
-  // three S/dP buffers of 128 columns (S at +0, dP at +64; bf16 dS later overwrites S): 0, 128, 384
-  auto buf_col = [](uint32_t bf) -> uint32_t { return bf == 2 ? 384u : bf * 128u; };
-  constexpr uint32_t kColDV = 128, kColDK = 192;   // alias buffer 1, which the dK/dV steps leave idle
+  // TMEM columns.  Regions 0, 1, 2 rotate through the roles S / dP+dS of the paired steps; a dK/dV
+  // step keeps S (64 columns) and dP (64) in region 0 and dV^T, dK^T in region 1.
   constexpr uint32_t kColDQ = 256;
+  constexpr uint32_t kColDV = 128, kColDK = 192;
+  // (region 2 is the one that aliases dV^T/dK^T: the paired steps reach it last)
+  auto region = [](int r) -> uint32_t { return r == 0 ? 0u : (r == 1 ? 384u : 128u); };
   extern __shared__ uint8_t smem_raw[];
   BwdSmem& sm = *reinterpret_cast<BwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
@@ -92,13 +112,16 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < kBwdKStages; ++s) { mbar_init(&sm.k_full[s], kBwdProducers); mbar_init(&sm.k_empty[s], 1); }
-    for (int s = 0; s < kBwdVStages; ++s) { mbar_init(&sm.v_full[s], kBwdProducers); mbar_init(&sm.v_empty[s], 1); }
-    for (int s = 0; s < 3; ++s) {
-      mbar_init(&sm.sdp_full[s], 1); mbar_init(&sm.buf_free[s], 1);
-      mbar_init(&sm.pds_full[s], 128);
-    }
+    for (int s = 0; s < kBwdKStages; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
+    for (int s = 0; s < kBwdVStages; ++s) { mbar_init(&sm.v_full[s], 2); mbar_init(&sm.v_empty[s], 1); }   // two V producers
+    mbar_init(&sm.sdp_full, 1); mbar_init(&sm.pds_full, 128);
     mbar_init(&sm.dkv_full, 1); mbar_init(&sm.dkv_free, 128);
+    mbar_init(&sm.s_full[0], 1); mbar_init(&sm.s_full[1], 1); mbar_init(&sm.ds_full, 256);
+    for (int s = 0; s < 4; ++s) mbar_init(&sm.dp_full[s], 1);
+    mbar_init(&sm.phase_a_done, 1);
+    for (int s = 0; s < kBwdKStages / 2; ++s) mbar_init(&sm.kp_full[s], 1);
+    for (int s = 0; s < kBwdKStages; ++s) mbar_init(&sm.kp_empty[s], 1);
+    mbar_init(&sm.vp_full, 2);
     mbar_init(&sm.dq_done, 1);
     sm.abort = 0;
     fence_barrier_init();
@@ -164,174 +187,243 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const int n_oct = sm.n_oct;
   const int n_keys = n_oct * 8;
   const int n_tiles = (n_oct + 7) / 8;
-  const int n_active = sm.n_dkv;                    // steps 0 .. n_active-1 produce dK/dV
-  const int dkv_hi = sm.dkv_lo + n_active;
+  const int n_act = sm.n_dkv;                       // steps 0 .. n_act-1 are dK/dV steps
+  const int dkv_hi = sm.dkv_lo + n_act;
+  const int n_pairs = (n_tiles - n_act + 1) / 2;    // paired steps; the last may hold one tile only
+  // Ring slots: dK/dV step s uses slot s; the paired steps start on an even slot (a pair of stages is
+  // one contiguous operand), so after an odd number of dK/dV steps one slot passes unused: the
+  // producers complete its full barriers without a copy, the MMA thread releases it at once.
+  const int n_act_even = n_pairs > 0 ? (n_act + 1) & ~1 : n_act;
   const int red_hi = band_done ? w.ls : 0x7fffffff;
   // Step order: the dK/dV tiles first (descending), so their atomics drain while the rest is
   // computed; then every other tile, descending.
   auto tile_of_step = [&](int s) {
-    if (s < n_active) return dkv_hi - 1 - s;
-    const int j = n_tiles - 1 - (s - n_active);
-    return j >= dkv_hi ? j : j - n_active;
+    if (s < n_act) return dkv_hi - 1 - s;
+    const int j = n_tiles - 1 - (s - n_act);
+    return j >= dkv_hi ? j : j - n_act;
   };
   volatile int* abort = &sm.abort;
   HGA_TRACE_POINT(1);
 
-  if (warp == 0 || warp == 14) {
+  if (warp == 0 || warp >= 14) {
     // ------------------------------------------------------------------ producers
-    // Issuing one TMA box costs the issuing warp on the order of a hundred cycles, so the sixteen
-    // octet boxes of a step are spread over two warps: producer p takes octets p, p+2, p+4, p+6 of
-    // the K tile (lanes 0-3) and of the V tile (lanes 8-11).  Every producer arrives on the full
-    // barriers with the byte count of its own boxes.
-    const int pi = warp == 0 ? 0 : 1;
-    const int sub = lane & 7;
-    const int oct_in_tile = pi + kBwdProducers * sub;          // < 8 for the lanes that copy
-    const bool k_lane = lane < 8 && oct_in_tile < 8, v_lane = lane >= 8 && lane < 16 && oct_in_tile < 8;
-    const uint32_t my_bytes = (uint32_t)((8 - pi + kBwdProducers - 1) / kBwdProducers) * kOct;
+    // K and V advance independently (their rings differ in depth, and a V tile is released long
+    // before the K tile of the same step): warp 0 copies the K tiles (eight octet boxes, one per
+    // lane) and runs several steps ahead; warps 14 and 15 copy the V tiles (four boxes each), whose
+    // short ring is refilled only after the dP GEMM of the previous pair, so their issue time is on
+    // the critical path.  Issuing a box costs the issuing warp on the order of a hundred cycles;
+    // different warps issue in parallel.
+    const bool is_v = warp != 0;
+    const int n_stages = is_v ? kBwdVStages : kBwdKStages;
+    const CUtensorMap* map = is_v ? &map_v : &map_k;
     bool ok = true;
-    int issued = 0;
-    for (int s = 0; s < n_tiles; ++s) {
-      const int j = tile_of_step(s);
-      const int ks = s % kBwdKStages, vs = s % kBwdVStages;
-      const int o = 8 * j + oct_in_tile;
-      const int row = o < n_oct ? sm.oct_row[o] : dm.L;    // past the list: zeros
-      if (lane == 0 && s >= kBwdKStages) ok = bwd_wait(&sm.k_empty[ks], (s / kBwdKStages - 1) & 1, abort);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      HGA_TRACE_POINT(21);
-      if (lane == 0) mbar_arrive_expect_tx(&sm.k_full[ks], my_bytes);
-      __syncwarp();
-      if (k_lane) tma_load_5d(sm.k[ks] + oct_in_tile * kOct, &map_k, &sm.k_full[ks], 0, row, 0, h, b);
-      HGA_TRACE_POINT(22);
-      if (lane == 0 && s >= kBwdVStages) ok = bwd_wait(&sm.v_empty[vs], (s / kBwdVStages - 1) & 1, abort);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      HGA_TRACE_POINT(23);
-      if (lane == 0) mbar_arrive_expect_tx(&sm.v_full[vs], my_bytes);
-      __syncwarp();
-      if (v_lane) tma_load_5d(sm.v[vs] + oct_in_tile * kOct, &map_v, &sm.v_full[vs], 0, row, 0, h, b);
-      issued = s + 1;
-      HGA_TRACE_POINT(2);
+    // ---- slots of the dK/dV steps: one tile per slot, one full/empty barrier pair per stage
+    {
+      const int oct_in_tile = is_v ? (warp == 14 ? lane : 4 + lane) : lane;
+      const bool copy_lane = is_v ? lane < 4 : lane < 8;
+      const uint32_t my_bytes = (uint32_t)(is_v ? 4 : 8) * kOct;
+      for (int slot = 0; slot < n_act_even && ok; ++slot) {
+        const int st = slot % n_stages;
+        uint64_t* full = is_v ? &sm.v_full[st] : &sm.k_full[st];
+        uint64_t* empty = is_v ? &sm.v_empty[st] : &sm.k_empty[st];
+        uint8_t* dst = is_v ? sm.v[st] : sm.k[st];
+        const bool skipped = slot >= n_act;
+        int row = dm.L;                                      // past the list: zeros
+        if (!skipped) {
+          const int o = 8 * tile_of_step(slot) + oct_in_tile;
+          if (o < n_oct) row = sm.oct_row[o];
+        }
+        if (lane == 0 && slot >= n_stages) ok = bwd_wait(empty, (uint32_t)(slot / n_stages - 1) & 1, abort);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        if (lane == 0) { if (skipped) mbar_arrive(full); else mbar_arrive_expect_tx(full, my_bytes); }
+        __syncwarp();
+        if (copy_lane && !skipped) tma_load_5d(dst + oct_in_tile * kOct, map, full, 0, row, 0, h, b);
+        HGA_TRACE_POINT(2);
+      }
+    }
+    // ---- paired steps: pair p fills stages 2*ps, 2*ps+1 (ps continues the slot numbering) and
+    // completes ONE barrier per operand, so the MMA thread observes one barrier per operand and
+    // pair.  Lanes 0-7 (K) / 0-3 (V): first tile, lanes 8-15 / 4-7: second tile.
+    {
+      const int n_ps = n_stages / 2;
+      const int which = is_v ? lane >> 2 : lane >> 3;                     // tile of the pair
+      const int oct_in_tile = is_v ? (warp == 14 ? 0 : 4) + (lane & 3) : lane & 7;
+      const bool copy_lane = is_v ? lane < 8 : lane < 16;
+      for (int p = 0; p < n_pairs && ok; ++p) {
+        const int ps = (n_act_even / 2 + p) % n_ps;
+        uint64_t* full = is_v ? &sm.vp_full : &sm.kp_full[ps];
+        const int s = n_act + 2 * p + which;                              // step (tile order)
+        int row = dm.L;
+        if (s < n_tiles) {
+          const int o = 8 * tile_of_step(s) + oct_in_tile;
+          if (o < n_oct) row = sm.oct_row[o];
+        }
+        if (lane == 0) {
+          if (p < n_ps) {
+            // first paired use of these stages: if a dK/dV step used them, those steps must be over
+            if (2 * ps < n_act_even) ok = bwd_wait(&sm.phase_a_done, 0, abort);
+          } else if (is_v) {
+            ok = bwd_wait(&sm.dp_full[(p - 1) & 3], (uint32_t)((p - 1) >> 2) & 1, abort);   // dP of the previous pair has read the V stages
+          } else {
+            ok = bwd_wait(&sm.kp_empty[(n_act_even / 2 + p - 3) % kBwdKStages], (uint32_t)((p - 3) / kBwdKStages) & 1, abort);   // dQ of pair p-3 is done
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)(is_v ? 8 : 16) * kOct);
+        __syncwarp();
+        if (copy_lane)
+          tma_load_5d((is_v ? sm.v[2 * ps + which] : sm.k[2 * ps + which]) + oct_in_tile * kOct, map, full, 0, row, 0, h, b);
+        HGA_TRACE_POINT(2);
+      }
     }
     if (*abort && lane == 0) {
-      // giving up: let the copies still in flight land before shared memory is released (bounded:
-      // a full barrier also needs the other producers, which may have stopped earlier)
-      if (pi == 0) mbar_wait(&sm.q_full, 0);
-      for (int s = issued > kBwdKStages ? issued - kBwdKStages : 0; s < issued; ++s)
-        mbar_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1);
-      for (int s = issued > kBwdVStages ? issued - kBwdVStages : 0; s < issued; ++s)
-        mbar_wait(&sm.v_full[s % kBwdVStages], (s / kBwdVStages) & 1);
+      // giving up: give the copies still in flight time to land before shared memory is released
+      // (the full barriers may never complete once another role has stopped, hence a bounded sleep)
+      if (warp == 0) mbar_wait(&sm.q_full, 0);
+      for (int it = 0; it < 64; ++it) __nanosleep(1000);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc_sdp = idesc_bf16_f32(128, kKT, 0, 0);   // rows x keys, both K-major
+      constexpr uint32_t idesc_sdp = idesc_bf16_f32(128, kKT, 0, 0);       // rows x 64 keys, both K-major
+      constexpr uint32_t idesc_sdp2 = idesc_bf16_f32(128, 2 * kKT, 0, 0);  // rows x 128 keys
+      constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);          // dS K-major, K tile MN-major
+      constexpr uint32_t idesc_dkv = idesc_bf16_f32(D, kKT, 1, 1);         // both MN-major
       // Descriptors are built once; inside the loops an MMA costs two integer adds.
-      const uint64_t q_k = smem_desc_sw128(smem_u32(sm.q), 16, kOct);        // Q  as K-major A   (S, dK/dV steps)
-      const uint64_t do_k = smem_desc_sw128(smem_u32(sm.dO), 16, kOct);      // dO as K-major A   (dP, dK/dV steps)
-      const uint64_t k_k0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, kOct);    // K tile, K-major B  (S)
-      const uint64_t v_k0 = smem_desc_sw128(smem_u32(sm.v[0]), 16, kOct);    // V tile, K-major B  (dP)
-      // Two threads feed the tensor pipe.  This one (warp 1) issues S and dP of every step and
-      // runs ahead as far as the three TMEM buffers allow; the other (warp 15) issues the GEMMs
-      // that consume the row threads' output (dQ, and dV^T/dK^T on dK/dV steps).  Neither waits
-      // for barriers that only concern the other.
-      // Step s uses buffer 0 while it is a dK/dV step, then buffers 0,1,2,0,... .
-      auto buf_of = [&](int s) -> uint32_t { return s < n_active ? 0u : (uint32_t)((s - n_active) % 3); };
-      auto use_of = [&](int s) {              // earlier uses of the buffer of step s
-        const int i = s - n_active;
-        return s < n_active ? s : (i % 3 == 0 ? n_active : 0) + i / 3;
-      };
-      auto wait_k = [&](int s) { return bwd_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1, abort); };
-      auto wait_v = [&](int s) { return bwd_wait(&sm.v_full[s % kBwdVStages], (s / kBwdVStages) & 1, abort); };
-      auto wait_buf = [&](int s) {
-        bool good = true;
-        // the GEMMs that read the previous contents of this buffer (dS, or P/dS in shared memory) are done
-        const int use = use_of(s);
-        if (use > 0) good = bwd_wait(&sm.buf_free[buf_of(s)], (use - 1) & 1, abort);
-        // buffer 1 aliases the dK^T/dV^T accumulators: the reduction warps must have read the last ones
-        if (good && n_active > 0 && s == n_active + 1) good = bwd_wait(&sm.dkv_free, (n_active - 1) & 1, abort);
-        return good;
-      };
-      bool ok = bwd_wait(&sm.q_full, 0, abort);
-      for (int s = 0; s < n_tiles && ok; ++s) {
-        const uint32_t buf = buf_of(s);
-        ok = wait_k(s) && wait_v(s) && wait_buf(s);
-        if (!ok) break;
-        tc_fence_after_sync();
-        HGA_TRACE_POINT(6);
-        const uint64_t kd = desc_advance(k_k0, (uint32_t)(s % kBwdKStages) * kKvTile);
-        const uint64_t vd = desc_advance(v_k0, (uint32_t)(s % kBwdVStages) * kKvTile);
-        const uint32_t s_acc = tmem + buf_col(buf);
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-          mma_ss(s_acc, desc_advance(q_k, off), desc_advance(kd, off), idesc_sdp, kk > 0);
-        }
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-          mma_ss(s_acc + 64, desc_advance(do_k, off), desc_advance(vd, off), idesc_sdp, kk > 0);
-        }
-        mma_commit(&sm.sdp_full[buf]);
-        mma_commit(&sm.v_empty[s % kBwdVStages]);      // the V tile is only needed for dP
-        HGA_TRACE_POINT(8);
-      }
-    }
-  } else if (warp == 15) {
-    // ------------------------------------------------------------------ second MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);      // dS K-major, K tile MN-major
-      constexpr uint32_t idesc_dkv = idesc_bf16_f32(D, kKT, 1, 1);     // both MN-major
+      const uint64_t q_k = smem_desc_sw128(smem_u32(sm.q), 16, kOct);        // Q  as K-major A   (S)
+      const uint64_t do_k = smem_desc_sw128(smem_u32(sm.dO), 16, kOct);      // dO as K-major A   (dP)
       const uint64_t q_mn = smem_desc_sw128(smem_u32(sm.q), 1024, kOct);     // Q^T  as MN-major A (dK^T)
       const uint64_t do_mn = smem_desc_sw128(smem_u32(sm.dO), 1024, kOct);   // dO^T as MN-major A (dV^T)
-      const uint64_t k_mn0 = smem_desc_sw128(smem_u32(sm.k[0]), 1024, kOct); // K tile, MN-major B (dQ)
+      const uint64_t k_k0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, kOct);    // K tile(s), K-major B  (S)
+      const uint64_t v_k0 = smem_desc_sw128(smem_u32(sm.v[0]), 16, kOct);    // V tile(s), K-major B  (dP)
+      const uint64_t k_mn0 = smem_desc_sw128(smem_u32(sm.k[0]), 1024, kOct); // K tile(s), MN-major B (dQ)
       const uint64_t dsd = smem_desc_sw128(smem_u32(sm.ds), 16, 1024);       // dS: K-major A (dQ) and MN-major B (dK^T)
       const uint64_t pd = smem_desc_sw128(smem_u32(sm.p), 16, 1024);         // P : MN-major B (dV^T)
-      bool ok = true;
-      for (int s = 0; s < n_tiles && ok; ++s) {
-        const bool dkv_step = s < n_active;
-        const int i = s - n_active;
-        const uint32_t buf = dkv_step ? 0u : (uint32_t)(i % 3);
-        const int use = dkv_step ? s : (buf == 0 ? n_active : 0) + i / 3;
-        ok = bwd_wait(&sm.pds_full[buf], use & 1, abort);
+      // (arguments are ring slots)
+      auto wait_k = [&](int s) { return bwd_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1, abort); };
+      auto wait_v = [&](int s) { return bwd_wait(&sm.v_full[s % kBwdVStages], (s / kBwdVStages) & 1, abort); };
+      // acc (128 rows x N keys) = a (Q or dO, K-major) x b^T (key tiles at ring stage st, K-major)
+      auto issue_qk = [&](uint32_t acc, uint64_t a, uint64_t b0, int st, uint32_t idesc) {   // st: ring stage
+        const uint64_t bd = desc_advance(b0, (uint32_t)st * kKvTile);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
+          mma_ss(acc, desc_advance(a, off), desc_advance(bd, off), idesc, kk > 0);
+        }
+      };
+      bool ok = bwd_wait(&sm.q_full, 0, abort);
+      bool dq_started = false;
+      // ---- dK/dV steps: one at a time, every operand from shared memory.  The tensor pipe runs in
+      // issue order and a commit covers everything issued before it, so sdp_full of step s+1 also
+      // tells the row threads that the GEMMs reading P/dS of step s are done.
+      for (int s = 0; s < n_act && ok; ++s) {
+        const int st = s % kBwdKStages, vst = s % kBwdVStages;
+        ok = wait_k(s) && wait_v(s);
+        if (!ok) break;
+        tc_fence_after_sync();
+        issue_qk(tmem + region(0), q_k, k_k0, st, idesc_sdp);
+        issue_qk(tmem + region(0) + 64, do_k, v_k0, vst, idesc_sdp);
+        mma_commit(&sm.sdp_full);
+        mma_commit(&sm.v_empty[vst]);
+        ok = bwd_wait(&sm.pds_full, s & 1, abort);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint64_t kmn = desc_advance(k_mn0, (uint32_t)st * kKvTile);
+#pragma unroll
+        for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per MMA
+          mma_ss(tmem + kColDQ, desc_advance(dsd, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
+                 (dq_started || kk > 0));
+        dq_started = true;
+        if (s > 0) {
+          ok = bwd_wait(&sm.dkv_free, (s - 1) & 1, abort);
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
+#pragma unroll
+        for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per MMA (2 row octets)
+          mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2 * kOct), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
+#pragma unroll
+        for (int kk = 0; kk < 128 / 16; ++kk)
+          mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2 * kOct), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
+        mma_commit(&sm.dkv_full);
+        mma_commit(&sm.k_empty[st]);
+        HGA_TRACE_POINT(4);
+      }
+      // ---- paired steps.  Step u covers ring stages st, st+1 (contiguous); S(u) lives in region
+      // (2u)%3, dP(u) and later dS(u) in region (2u+1)%3.
+      if (ok && n_pairs > 0) {
+        if (n_act_even > n_act) {
+          // the unused slot: observe its (copy-less) full barriers and release it
+          ok = wait_k(n_act) && wait_v(n_act);
+          if (ok) {
+            mma_commit(&sm.k_empty[n_act % kBwdKStages]);
+            mma_commit(&sm.v_empty[n_act % kBwdVStages]);
+          }
+        }
+        if (ok && n_act_even > 0) mma_commit(&sm.phase_a_done);
+        const int ps0 = (n_act_even / 2) % (kBwdKStages / 2);
+        if (ok) ok = bwd_wait(&sm.kp_full[ps0], 0, abort);
+        if (ok) {
+          tc_fence_after_sync();
+          issue_qk(tmem + region(0), q_k, k_k0, 2 * ps0, idesc_sdp2);
+          mma_commit(&sm.s_full[0]);
+        }
+        if (ok) ok = bwd_wait(&sm.vp_full, 0, abort);
+        if (ok) {
+          tc_fence_after_sync();
+          issue_qk(tmem + region(1), do_k, v_k0, 0, idesc_sdp2);
+          mma_commit(&sm.dp_full[0]);    // also tells the V producers that the V stages are free
+        }
+        HGA_TRACE_POINT(3);
+      }
+      int rs = 0;                                     // region of S(u)
+      for (int u = 0; u < n_pairs && ok; ++u) {
+        constexpr int kPs = kBwdKStages / 2;
+        const int ps = (n_act_even / 2 + u) % kPs, ps_n = (ps + 1) % kPs;     // pair stages of steps u, u+1
+        const int rp = rs == 2 ? 0 : rs + 1;          // region of dP(u), dS(u)
+        const int rs_n = rp == 2 ? 0 : rp + 1;        // region of S(u+1): two steps ago it held dP(u-1)
+        if (u + 1 < n_pairs) {
+          ok = bwd_wait(&sm.kp_full[ps_n], (uint32_t)((u + 1) / kPs) & 1, abort);
+          // S(1) is the first to use the region that aliases the dK^T/dV^T accumulators: the
+          // reduction warps must have read the last ones
+          if (ok && u == 0 && n_act > 0) ok = bwd_wait(&sm.dkv_free, (n_act - 1) & 1, abort);
+          if (!ok) break;
+          tc_fence_after_sync();
+          issue_qk(tmem + region(rs_n), q_k, k_k0, 2 * ps_n, idesc_sdp2);
+          mma_commit(&sm.s_full[(u + 1) & 1]);
+          HGA_TRACE_POINT(6);
+        }
+        ok = bwd_wait(&sm.ds_full, u & 1, abort);     // the row threads are done with S(u) and dP(u)
         if (!ok) break;
         tc_fence_after_sync();
         HGA_TRACE_POINT(5);
-        const uint64_t kmn = desc_advance(k_mn0, (uint32_t)(s % kBwdKStages) * kKvTile);
-        if (dkv_step) {
-#pragma unroll
-          for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per MMA, dS from shared memory
-            mma_ss(tmem + kColDQ, desc_advance(dsd, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
-                   (s > 0 || kk > 0));
-          if (s > 0) {
-            ok = bwd_wait(&sm.dkv_free, (s - 1) & 1, abort);
-            if (!ok) break;
-            tc_fence_after_sync();
-          }
-#pragma unroll
-          for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per MMA (2 row octets)
-            mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2 * kOct), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
-#pragma unroll
-          for (int kk = 0; kk < 128 / 16; ++kk)
-            mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2 * kOct), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
-          mma_commit(&sm.dkv_full);
-        } else {
-#pragma unroll
-          for (int kk = 0; kk < kKT / 16; ++kk)   // dS (bf16) from TMEM, 8 columns per 16 keys
-            mma_ts(tmem + kColDQ, tmem + buf_col(buf) + 8 * kk, desc_advance(kmn, kk * 2 * kOct), idesc_dq,
-                   (s > 0 || kk > 0));
+        if (u + 1 < n_pairs) {
+          ok = bwd_wait(&sm.vp_full, (uint32_t)(u + 1) & 1, abort);
+          if (!ok) break;
+          tc_fence_after_sync();
+          issue_qk(tmem + region(rs), do_k, v_k0, 0, idesc_sdp2);       // dP(u+1) into the region of S(u)
+          mma_commit(&sm.dp_full[(u + 1) & 3]);
+          HGA_TRACE_POINT(8);
         }
-        mma_commit(&sm.k_empty[s % kBwdKStages]);
-        mma_commit(&sm.buf_free[buf]);
+        // dQ += dS K over 128 keys: bf16 dS from TMEM (first tile at columns 0-31 of its region,
+        // second tile at 64-95), the two K stages as one MN-major B operand
+        const uint64_t kmn = desc_advance(k_mn0, (uint32_t)(2 * ps) * kKvTile);
+        const uint32_t ds_base = tmem + region(rp);
+#pragma unroll
+        for (int kk = 0; kk < 2 * kKT / 16; ++kk)
+          mma_ts(tmem + kColDQ, ds_base + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), desc_advance(kmn, kk * 2 * kOct),
+                 idesc_dq, (dq_started || kk > 0));
+        dq_started = true;
+        mma_commit(&sm.kp_empty[(n_act_even / 2 + u) % kBwdKStages]);
         HGA_TRACE_POINT(7);
+        rs = rs_n;
       }
       if (ok) mma_commit(&sm.dq_done);
     }
   } else if (warp < 10) {
     // ------------------------------------------------------------------ one thread per query row
-    // Warpgroup 0 (warps 2-5) takes the dK/dV steps and then the even ones of the remaining steps,
-    // warpgroup 1 (warps 6-9) the odd ones, each with its own S/dP buffer in TMEM, so the exp2 / dS
-    // work of one step overlaps the GEMMs of the next.
     const int wg = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int row_in_tile = quarter * 32 + lane;
@@ -344,67 +436,105 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const float neg_lse2 = -row_lse * 1.4426950408889634f;
     const float neg_delta_s = -delta * dm.scale;
     HGA_TRACE_POINT(10);
-    // this row's 128-byte line inside the P / dS buffers, and its swizzle key
-    const uint32_t line = (uint32_t)(row_in_tile >> 3) * 1024 + (uint32_t)(row_in_tile & 7) * 128;
-    const uint32_t key = (uint32_t)(row_in_tile & 7);
-    const uint32_t p_line = smem_u32(sm.p) + line, ds_line = smem_u32(sm.ds) + line;
     bool ok = true;
-    const int n_rest = n_tiles - n_active;
-    const int n_mine = wg == 0 ? n_active + (n_rest + 1) / 2 : n_rest / 2;
-    for (int u = 0; u < n_mine && ok; ++u) {
-      const bool dkv_step = wg == 0 && u < n_active;
-      const int s = dkv_step ? u : n_active + 2 * (u - (wg == 0 ? n_active : 0)) + wg;
-      const int i = s - n_active;
-      const uint32_t buf = dkv_step ? 0u : (uint32_t)(i % 3);
-      const int use = dkv_step ? s : (buf == 0 ? n_active : 0) + i / 3;     // earlier uses of buf
-      const uint32_t sdp_addr = lane_base + buf_col(buf);
-      const int j = tile_of_step(s);
-      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[buf], use & 1, abort));
-      if (!ok) break;
-      tc_fence_after_sync();
-      HGA_TRACE_POINT(11);
-      const int vis = limit - kKT * j;
+    if (wg == 0) {
+      // ---- dK/dV steps (warpgroup 0): P and dS go to shared memory as operands of dV^T / dK^T / dQ
+      // this row's 128-byte line inside the P / dS buffers, and its swizzle key
+      const uint32_t line = (uint32_t)(row_in_tile >> 3) * 1024 + (uint32_t)(row_in_tile & 7) * 128;
+      const uint32_t key = (uint32_t)(row_in_tile & 7);
+      const uint32_t p_line = smem_u32(sm.p) + line, ds_line = smem_u32(sm.ds) + line;
+      const uint32_t sdp_addr = lane_base + region(0);
+      for (int s = 0; s < n_act && ok; ++s) {
+        ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full, s & 1, abort));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const int vis = limit - kKT * tile_of_step(s);
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {               // 16 columns (keys) at a time: 128-register budget
-        uint32_t sv[16], dp[16];
-        tmem_ld16(sdp_addr + q4 * 16, sv);
-        tmem_ld16(sdp_addr + 64 + q4 * 16, dp);
-        tmem_wait_ld();
-        uint32_t pk[8], dk[8];
+        for (int q4 = 0; q4 < 4; ++q4) {             // 16 columns (keys) at a time
+          uint32_t sv[16], dp[16];
+          tmem_ld16(sdp_addr + q4 * 16, sv);
+          tmem_ld16(sdp_addr + 64 + q4 * 16, dp);
+          tmem_wait_ld();
+          uint32_t pk[8], dk[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), sl2, neg_lse2));
-          float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), sl2, neg_lse2));
-          if (vis < kKT) {                    // diagonal / ragged tile only
-            if (q4 * 16 + 2 * i >= vis) p0 = 0.f;
-            if (q4 * 16 + 2 * i + 1 >= vis) p1 = 0.f;
+          for (int i = 0; i < 8; ++i) {
+            float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), sl2, neg_lse2));
+            float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), sl2, neg_lse2));
+            if (vis < kKT) {                  // diagonal / ragged tile only
+              if (q4 * 16 + 2 * i >= vis) p0 = 0.f;
+              if (q4 * 16 + 2 * i + 1 >= vis) p1 = 0.f;
+            }
+            const float d0 = p0 * fmaf(__uint_as_float(dp[2 * i]), dm.scale, neg_delta_s);
+            const float d1 = p1 * fmaf(__uint_as_float(dp[2 * i + 1]), dm.scale, neg_delta_s);
+            pk[i] = pack_bf16(p0, p1);
+            dk[i] = pack_bf16(d0, d1);
           }
-          const float d0 = p0 * fmaf(__uint_as_float(dp[2 * i]), dm.scale, neg_delta_s);
-          const float d1 = p1 * fmaf(__uint_as_float(dp[2 * i + 1]), dm.scale, neg_delta_s);
-          pk[i] = pack_bf16(p0, p1);
-          dk[i] = pack_bf16(d0, d1);
-        }
-        if (dkv_step) {
-          // P and dS feed the dV^T / dK^T GEMMs as shared-memory operands
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {    // two 16-byte chunks (8 keys each), XOR-swizzled
             const uint32_t off = ((uint32_t)(2 * q4 + cc) ^ key) * 16;
             st_shared_v4(p_line + off, pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
             st_shared_v4(ds_line + off, dk[4 * cc], dk[4 * cc + 1], dk[4 * cc + 2], dk[4 * cc + 3]);
           }
-        } else {
-          // bf16 dS over the S columns already read (8 columns per 16 keys): the A operand of dQ
-          tmem_st8(sdp_addr + q4 * 8, dk);
+        }
+        tc_fence_before_sync();
+        fence_proxy_async_smem();
+        mbar_arrive(&sm.pds_full);
+      }
+    }
+    // ---- paired steps: warpgroup wg owns the wg-th tile of each pair (64 of the 128 columns)
+    int rs = 0;
+    for (int u = 0; u < n_pairs && ok; ++u) {
+      const int rp = rs == 2 ? 0 : rs + 1;
+      const int s = n_act + 2 * u + wg;
+      const int vis = s < n_tiles ? limit - kKT * tile_of_step(s) : 0;     // a missing tile is fully masked
+      const uint32_t s_addr = lane_base + region(rs) + wg * 64;
+      const uint32_t dp_addr = lane_base + region(rp) + wg * 64;
+      uint32_t pk[32];                                // P of this row, 64 keys, packed bf16
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.s_full[u & 1], (u >> 1) & 1, abort));
+      if (!ok) break;
+      tc_fence_after_sync();
+      HGA_TRACE_POINT(11);
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        uint32_t sv[16];
+        tmem_ld16(s_addr + q4 * 16, sv);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), sl2, neg_lse2));
+          float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), sl2, neg_lse2));
+          if (vis < kKT) {
+            if (q4 * 16 + 2 * i >= vis) p0 = 0.f;
+            if (q4 * 16 + 2 * i + 1 >= vis) p1 = 0.f;
+          }
+          pk[8 * q4 + i] = pack_bf16(p0, p1);
         }
       }
-      if (dkv_step) {
-        fence_proxy_async_smem();
-      } else {
-        tmem_wait_st();
-        tc_fence_before_sync();
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.dp_full[u & 3], (u >> 2) & 1, abort));
+      if (!ok) break;
+      tc_fence_after_sync();
+      HGA_TRACE_POINT(13);
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        uint32_t dp[16], dk[8];
+        tmem_ld16(dp_addr + q4 * 16, dp);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float p0 = __uint_as_float(pk[8 * q4 + i] << 16);
+          const float p1 = __uint_as_float(pk[8 * q4 + i] & 0xffff0000u);
+          const float d0 = p0 * fmaf(__uint_as_float(dp[2 * i]), dm.scale, neg_delta_s);
+          const float d1 = p1 * fmaf(__uint_as_float(dp[2 * i + 1]), dm.scale, neg_delta_s);
+          dk[i] = pack_bf16(d0, d1);
+        }
+        // bf16 dS over the dP columns already read (8 columns per 16 keys): the A operand of dQ
+        tmem_st8(dp_addr + q4 * 8, dk);
       }
-      mbar_arrive(&sm.pds_full[buf]);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(&sm.ds_full);
       HGA_TRACE_POINT(14);
+      rs = rp == 2 ? 0 : rp + 1;
     }
     if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.dq_done, 0, abort));
     HGA_TRACE_POINT(20);
@@ -435,7 +565,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     float* dKb = dK + ((int64_t)(b * dm.Hkv + h) * dm.S) * D + e;
     float* dVb = dV + ((int64_t)(b * dm.Hkv + h) * dm.S) * D + e;
     bool ok = true;
-    for (int s = 0; s < n_active; ++s) {
+    for (int s = 0; s < n_act; ++s) {
       const int j = tile_of_step(s);
       ok = __all_sync(0xffffffffu, bwd_wait(&sm.dkv_full, s & 1, abort));
       if (!ok) break;
