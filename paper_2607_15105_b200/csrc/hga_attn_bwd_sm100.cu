@@ -138,12 +138,14 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       mbar_arrive_expect_tx(&sm.q_full, 2 * 128 * kBwdD * 2);
     }
     __syncwarp();
-    {
-      const int o = lane & 15;
-      const int r = mt * 128 + 8 * o;
+    if (lane < 8) {
+      // four boxes of 64 rows x one 64-element panel per tensor, laid out [panel][128 rows][128 B]
+      const int half = lane & 1, panel = (lane >> 1) & 1;
+      const int r = mt * 128 + 64 * half;
       const int a = r / dm.Bq, t = r % dm.Bq;
-      if (lane < 16) tma_load_5d(sm.q + o * kOct, &map_q, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
-      else tma_load_5d(sm.dO + o * kOct, &map_do, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
+      const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
+      if (lane < 4) tma_load_5d(sm.q + off, &map_q, &sm.q_full, 0, qb * dm.Bq + t, panel, h * dm.G + a, b);
+      else tma_load_5d(sm.dO + off, &map_do, &sm.q_full, 0, qb * dm.Bq + t, panel, h * dm.G + a, b);
     }
     bool bad;   // invalid entries are skipped exactly as in the forward kernel (which reports them)
     const int n_oct = build_octet_table(dm, w, group_idx + (int64_t)item * dm.width, n_groups + item, sm.oct_row, &bad);
@@ -292,10 +294,11 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);          // dS K-major, K tile MN-major
       constexpr uint32_t idesc_dkv = idesc_bf16_f32(D, kKT, 1, 1);         // both MN-major
       // Descriptors are built once; inside the loops an MMA costs two integer adds.
-      const uint64_t q_k = smem_desc_sw128(smem_u32(sm.q), 16, kOct);        // Q  as K-major A   (S)
-      const uint64_t do_k = smem_desc_sw128(smem_u32(sm.dO), 16, kOct);      // dO as K-major A   (dP)
-      const uint64_t q_mn = smem_desc_sw128(smem_u32(sm.q), 1024, kOct);     // Q^T  as MN-major A (dK^T)
-      const uint64_t do_mn = smem_desc_sw128(smem_u32(sm.dO), 1024, kOct);   // dO^T as MN-major A (dV^T)
+      // Q, dO: [panel][128 rows][128 B] (8-row groups 1024 B apart, panels 16 KB apart)
+      const uint64_t q_k = smem_desc_sw128(smem_u32(sm.q), 16, 1024);        // Q  as K-major A   (S)
+      const uint64_t do_k = smem_desc_sw128(smem_u32(sm.dO), 16, 1024);      // dO as K-major A   (dP)
+      const uint64_t q_mn = smem_desc_sw128(smem_u32(sm.q), 16384, 1024);    // Q^T  as MN-major A (dK^T)
+      const uint64_t do_mn = smem_desc_sw128(smem_u32(sm.dO), 16384, 1024);  // dO^T as MN-major A (dV^T)
       const uint64_t k_k0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, kOct);    // K tile(s), K-major B  (S)
       const uint64_t v_k0 = smem_desc_sw128(smem_u32(sm.v[0]), 16, kOct);    // V tile(s), K-major B  (dP)
       const uint64_t k_mn0 = smem_desc_sw128(smem_u32(sm.k[0]), 1024, kOct); // K tile(s), MN-major B (dQ)
@@ -309,8 +312,8 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint64_t bd = desc_advance(b0, (uint32_t)st * kKvTile);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-          mma_ss(acc, desc_advance(a, off), desc_advance(bd, off), idesc, kk > 0);
+          const uint32_t a_off = (kk >> 2) * 16384 + (kk & 3) * 32, b_off = (kk >> 2) * 1024 + (kk & 3) * 32;
+          mma_ss(acc, desc_advance(a, a_off), desc_advance(bd, b_off), idesc, kk > 0);
         }
       };
       bool ok = bwd_wait(&sm.q_full, 0, abort);
@@ -343,10 +346,10 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
 #pragma unroll
         for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per MMA (2 row octets)
-          mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2 * kOct), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
+          mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2048), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
 #pragma unroll
         for (int kk = 0; kk < 128 / 16; ++kk)
-          mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2 * kOct), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
+          mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2048), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
         mma_commit(&sm.dkv_full);
         mma_commit(&sm.k_empty[st]);
         HGA_TRACE_POINT(4);
@@ -646,7 +649,7 @@ k_bwd_delta_sm100(const uint16_t* __restrict__ O, const uint16_t* __restrict__ d
 
 bool attn_bwd_sm100_supported(const Dims& dm) {
   if (dm.flags & HGA_FLAG_GENERIC_KERNELS) return false;
-  return dm.d == 128 && dm.rows % 128 == 0 && dm.g % 8 == 0;
+  return dm.d == 128 && dm.rows % 128 == 0 && dm.g % 8 == 0 && dm.Bq % 64 == 0;
 }
 
 int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
@@ -655,14 +658,15 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
                           bool zero_grads, int32_t* status_word, cudaStream_t st) {
   CUtensorMap mq, mdo, mk, mv;
   const uint32_t box[5] = {64, 8, 2, 1, 1};
+  const uint32_t box_q[5] = {64, 64, 1, 1, 1};
   const uint64_t dq[5] = {64, (uint64_t)dm.S, 2, (uint64_t)dm.Hq, (uint64_t)dm.B};
   const uint64_t dk[5] = {64, (uint64_t)dm.L, 2, (uint64_t)dm.Hkv, (uint64_t)dm.B};
   const uint64_t sq[4] = {(uint64_t)dm.qs[2] * 2, 128, (uint64_t)dm.qs[1] * 2, (uint64_t)dm.qs[0] * 2};
   const uint64_t so[4] = {(uint64_t)dm.os[2] * 2, 128, (uint64_t)dm.os[1] * 2, (uint64_t)dm.os[0] * 2};
   const uint64_t sk[4] = {(uint64_t)dm.ks[2] * 2, 128, (uint64_t)dm.ks[1] * 2, (uint64_t)dm.ks[0] * 2};
   const uint64_t sv[4] = {(uint64_t)dm.vs[2] * 2, 128, (uint64_t)dm.vs[1] * 2, (uint64_t)dm.vs[0] * 2};
-  if (encode_tensor_map_bf16(&mq, Q, 5, dq, sq, box, true) ||
-      encode_tensor_map_bf16(&mdo, dO, 5, dq, so, box, true) ||
+  if (encode_tensor_map_bf16(&mq, Q, 5, dq, sq, box_q, true) ||
+      encode_tensor_map_bf16(&mdo, dO, 5, dq, so, box_q, true) ||
       encode_tensor_map_bf16(&mk, K, 5, dk, sk, box, true) ||
       encode_tensor_map_bf16(&mv, V, 5, dk, sv, box, true))
     return HGA_ERR_UNSUPPORTED;
