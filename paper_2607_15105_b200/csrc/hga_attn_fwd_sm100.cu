@@ -52,7 +52,7 @@ struct FwdSmem {
   alignas(1024) uint8_t k[kStages][kTileBytes];
   alignas(1024) uint8_t v[kStages][kTileBytes];
   uint64_t q_full;
-  uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+  uint64_t k_full[kStages], v_full[kStages], v_empty[kStages];
   uint64_t s_full[2], p_full[2], tail_done, o_done;
   uint32_t tmem_base;
   int n_oct;
@@ -96,7 +96,7 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1);
+      mbar_init(&sm.k_full[s], 1);
       mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
     }
     for (int u = 0; u < 2; ++u) { mbar_init(&sm.s_full[u], 1); mbar_init(&sm.p_full[u], 128); }
@@ -144,7 +144,10 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // ------------------------------------------------------------------ producers: warp 0 K, warp 6 V
     const bool is_k = warp == 0;
     uint64_t* full = is_k ? sm.k_full : sm.v_full;
-    uint64_t* empty = is_k ? sm.k_empty : sm.v_empty;
+    // a K stage is free as soon as S of its tile is complete: that is s_full of the same index (the K
+    // ring and the S buffers both have two slots), which saves the MMA thread one commit per tile
+    static_assert(kStages == 2, "K ring and S buffers are indexed alike");
+    uint64_t* empty = is_k ? sm.s_full : sm.v_empty;
     uint8_t* ring = is_k ? sm.k[0] : sm.v[0];
     const CUtensorMap* map = is_k ? &map_k : &map_v;
     bool ok = true;
@@ -190,8 +193,7 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;   // panel, then 32-byte K step
           mma_ss(d_addr, desc_advance(q_desc, off), desc_advance(kd, off), idesc_s, kk > 0);
         }
-        mma_commit(&sm.s_full[j & 1]);
-        mma_commit(&sm.k_empty[j % kStages]);
+        mma_commit(&sm.s_full[j & 1]);           // also releases the K stage (see the K producer)
       };
       bool ok = wait_or_abort(&sm.q_full, 0, abort);
       for (int j = 0; j < 2 && j < n_tiles && ok; ++j) {      // prologue: S two tiles ahead
