@@ -165,8 +165,12 @@ HGA_API int hga_workspace_bytes(const hga_params* p, size_t* route_bytes, size_t
  * resident device K/V (device [B,Hkv,L,d] dense, history already in place), runs
  * build_summaries(active range) -> route -> attn_fwd -> attn_bwd, and copies O (bf16),
  * dQ (bf16), dK, dV (fp32) back to the host buffers.  dO_host == NULL runs the forward half
- * only.  All work is queued on `stream`; the host buffers are valid after the caller
- * synchronises the stream.  arena: device scratch of hga_step_arena_bytes() bytes.
+ * only.  The step runs as a pipeline over the (batch, kv head) pairs, which are independent
+ * problems: one pair's kernels overlap the next pair's host->device copies and the previous
+ * pair's device->host copies.  The copies run on two streams the library creates once per
+ * device (on the first call there); they start after the work already queued on `stream`,
+ * and `stream` waits for the last of them, so the host buffers are valid after the caller
+ * synchronises `stream`.  arena: device scratch of hga_step_arena_bytes() bytes.
  * chunk_sum / group_sum: resident device summaries (history part already built). */
 HGA_API int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host,
                   const void* Vseg_host, const void* dO_host, void* K_dev, void* V_dev,

@@ -2,6 +2,9 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
+#include <map>
+#include <mutex>
+#include <vector>
 
 #include "hga_common.cuh"
 
@@ -79,6 +82,42 @@ size_t route_workspace_bytes(const Dims& dm) {
 size_t bwd_workspace_bytes(const Dims& dm) {
   // delta = rowsum(dO * O), fp32 [B, Hq, S]
   return (size_t)dm.B * dm.Hq * dm.S * sizeof(float) + 16;
+}
+
+// Copy streams and events of hga_step_host, created once per device and kept until exit.
+struct StepPipe {
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  std::vector<cudaEvent_t> in_done, comp_done;
+};
+
+static StepPipe* step_pipe(int n_pairs) {
+  static std::mutex mu;
+  static std::map<int, StepPipe> pipes;
+  std::lock_guard<std::mutex> lock(mu);
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+  StepPipe& sp = pipes[dev];
+  if (!sp.in) {
+    if (cudaStreamCreateWithFlags(&sp.in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&sp.out, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&sp.fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&sp.join, cudaEventDisableTiming) != cudaSuccess) {
+      record_cuda(cudaGetLastError());
+      return nullptr;
+    }
+  }
+  while ((int)sp.in_done.size() < n_pairs) {
+    cudaEvent_t a = nullptr, b = nullptr;
+    if (cudaEventCreateWithFlags(&a, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&b, cudaEventDisableTiming) != cudaSuccess) {
+      record_cuda(cudaGetLastError());
+      return nullptr;
+    }
+    sp.in_done.push_back(a);
+    sp.comp_done.push_back(b);
+  }
+  return &sp;
 }
 
 }  // namespace hga
@@ -245,9 +284,9 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   size_t kv32 = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 4;
   size_t kvseg = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 2;
   size_t items = (size_t)dm.B * dm.Hkv * dm.NQB;
-  void* dQin = take(qb); void* ddO = take(qb); void* dOut = take(qb); void* ddQ = take(qb);
-  float* ddK = (float*)take(kv32); float* ddV = (float*)take(kv32);
-  void* kseg = take(kvseg); void* vseg = take(kvseg);
+  char* dQin = (char*)take(qb); char* ddO = (char*)take(qb); char* dOut = (char*)take(qb); char* ddQ = (char*)take(qb);
+  char* ddK = (char*)take(kv32); char* ddV = (char*)take(kv32);
+  take(kvseg); take(kvseg);                          // (reserved: earlier versions staged the K/V rows here)
   int32_t* cidx = (int32_t*)take(items * (dm.kc + dm.width + 1) * 4 + 64);
   int32_t* gidx = cidx + items * dm.kc;
   int32_t* ng = gidx + items * dm.width;
@@ -255,45 +294,68 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   void* rws = take(route_workspace_bytes(dm));
   void* bws = take(bwd_workspace_bytes(dm));
 
-  // host -> device: Q, (dO), and the active segment's K/V rows appended behind the history
-  rc = record_cuda(cudaMemcpyAsync(dQin, Q_host, qb, cudaMemcpyHostToDevice, st));
-  if (rc) return rc;
-  if (bwd) {
-    rc = record_cuda(cudaMemcpyAsync(ddO, dO_host, qb, cudaMemcpyHostToDevice, st));
-    if (rc) return rc;
-  }
-  rc = record_cuda(cudaMemcpyAsync(kseg, Kseg_host, kvseg, cudaMemcpyHostToDevice, st));
-  if (rc) return rc;
-  rc = record_cuda(cudaMemcpyAsync(vseg, Vseg_host, kvseg, cudaMemcpyHostToDevice, st));
-  if (rc) return rc;
-  const size_t row = (size_t)dm.d * 2;
-  rc = record_cuda(cudaMemcpy2DAsync((char*)K_dev + (size_t)dm.H * row, (size_t)dm.L * row, kseg,
-                                     (size_t)dm.S * row, (size_t)dm.S * row,
-                                     (size_t)dm.B * dm.Hkv, cudaMemcpyDeviceToDevice, st));
-  if (rc) return rc;
-  rc = record_cuda(cudaMemcpy2DAsync((char*)V_dev + (size_t)dm.H * row, (size_t)dm.L * row, vseg,
-                                     (size_t)dm.S * row, (size_t)dm.S * row,
-                                     (size_t)dm.B * dm.Hkv, cudaMemcpyDeviceToDevice, st));
-  if (rc) return rc;
+  // The (batch, kv head) pairs are independent problems (routing, attention and dK/dV never cross kv
+  // heads), so the step runs as a pipeline over them: while one pair's kernels run, the next pair's
+  // inputs arrive on a copy stream and the previous pair's results leave on another (the two copy
+  // directions overlap as well).  Everything is ordered after the work already queued on `stream`,
+  // and `stream` ends up waiting for the last copy, so the caller sees one stream as before.
+  StepPipe* pipe = step_pipe(dm.B * dm.Hkv);
+  if (!pipe) return HGA_ERR_CUDA;
+  hga_params pc = *p;                                // one (batch, kv head): B = 1, Hkv = 1, Hq = G, dense
+  pc.batch = 1;
+  pc.n_q_heads = dm.G;
+  pc.n_kv_heads = 1;
+  const size_t q_c = (size_t)dm.G * dm.S * dm.d * 2;           // bytes of one pair's Q / dO / O / dQ rows
+  const size_t kvseg_c = (size_t)dm.S * dm.d * 2, kv32_c = (size_t)dm.S * dm.d * 4;
+  const size_t kv_c = (size_t)dm.L * dm.d * 2;                 // one (batch, kv head) of the resident K / V
+  const size_t hist = (size_t)dm.H * dm.d * 2;
+  const size_t cs_c = (size_t)dm.Nc * dm.d * 2, gs_c = (size_t)dm.Ng * dm.d * 2;
+#define HGA_TRY(x) do { rc = (x); if (rc) return rc; } while (0)
+  HGA_TRY(record_cuda(cudaEventRecord(pipe->fork, st)));
+  HGA_TRY(record_cuda(cudaStreamWaitEvent(pipe->in, pipe->fork, 0)));
+  HGA_TRY(record_cuda(cudaStreamWaitEvent(pipe->out, pipe->fork, 0)));
+  const int n_pairs = dm.B * dm.Hkv;
+  for (int c = 0; c < n_pairs; ++c) {
+    // host -> device: this pair's Q, (dO), and its active-segment K/V rows straight behind the history
+    HGA_TRY(record_cuda(cudaMemcpyAsync(dQin + c * q_c, (const char*)Q_host + c * q_c, q_c, cudaMemcpyHostToDevice, pipe->in)));
+    if (bwd)
+      HGA_TRY(record_cuda(cudaMemcpyAsync(ddO + c * q_c, (const char*)dO_host + c * q_c, q_c, cudaMemcpyHostToDevice, pipe->in)));
+    HGA_TRY(record_cuda(cudaMemcpyAsync((char*)K_dev + c * kv_c + hist, (const char*)Kseg_host + c * kvseg_c, kvseg_c,
+                                        cudaMemcpyHostToDevice, pipe->in)));
+    HGA_TRY(record_cuda(cudaMemcpyAsync((char*)V_dev + c * kv_c + hist, (const char*)Vseg_host + c * kvseg_c, kvseg_c,
+                                        cudaMemcpyHostToDevice, pipe->in)));
+    HGA_TRY(record_cuda(cudaEventRecord(pipe->in_done[c], pipe->in)));
+    HGA_TRY(record_cuda(cudaStreamWaitEvent(st, pipe->in_done[c], 0)));
 
-  rc = hga_build_summaries(p, K_dev, dm.H, dm.L, chunk_sum, group_sum, stream);
-  if (rc) return rc;
-  rc = hga_route(p, dQin, chunk_sum, group_sum, cidx, gidx, ng, nullptr, nullptr, rws,
-                 route_workspace_bytes(dm), stream);
-  if (rc) return rc;
-  rc = hga_attn_fwd(p, dQin, K_dev, V_dev, gidx, ng, dOut, lse, status_word, stream);
-  if (rc) return rc;
-  rc = record_cuda(cudaMemcpyAsync(O_host, dOut, qb, cudaMemcpyDeviceToHost, st));
-  if (rc) return rc;
-  if (!bwd) return HGA_OK;
-  rc = hga_attn_bwd(p, dQin, K_dev, V_dev, dOut, lse, ddO, gidx, ng, ddQ, ddK, ddV, bws,
-                    bwd_workspace_bytes(dm), status_word, stream);
-  if (rc) return rc;
-  rc = record_cuda(cudaMemcpyAsync(dQ_host, ddQ, qb, cudaMemcpyDeviceToHost, st));
-  if (rc) return rc;
-  rc = record_cuda(cudaMemcpyAsync(dK_host, ddK, kv32, cudaMemcpyDeviceToHost, st));
-  if (rc) return rc;
-  return record_cuda(cudaMemcpyAsync(dV_host, ddV, kv32, cudaMemcpyDeviceToHost, st));
+    const char* Kc = (const char*)K_dev + c * kv_c;
+    const char* Vc = (const char*)V_dev + c * kv_c;
+    char* csc = (char*)chunk_sum + c * cs_c;
+    char* gsc = (char*)group_sum + c * gs_c;
+    int32_t* gic = gidx + (size_t)c * dm.NQB * dm.width;
+    int32_t* ngc = ng + (size_t)c * dm.NQB;
+    float* lsec = lse + (size_t)c * dm.G * dm.S;
+    HGA_TRY(hga_build_summaries(&pc, Kc, dm.H, dm.L, csc, gsc, stream));
+    HGA_TRY(hga_route(&pc, dQin + c * q_c, csc, gsc, cidx + (size_t)c * dm.NQB * dm.kc, gic, ngc, nullptr, nullptr, rws,
+                      route_workspace_bytes(dm), stream));
+    HGA_TRY(hga_attn_fwd(&pc, dQin + c * q_c, Kc, Vc, gic, ngc, dOut + c * q_c, lsec, status_word, stream));
+    if (bwd)
+      HGA_TRY(hga_attn_bwd(&pc, dQin + c * q_c, Kc, Vc, dOut + c * q_c, lsec, ddO + c * q_c, gic, ngc, ddQ + c * q_c,
+                           (float*)(ddK + c * kv32_c), (float*)(ddV + c * kv32_c), bws, bwd_workspace_bytes(dm),
+                           status_word, stream));
+    HGA_TRY(record_cuda(cudaEventRecord(pipe->comp_done[c], st)));
+    HGA_TRY(record_cuda(cudaStreamWaitEvent(pipe->out, pipe->comp_done[c], 0)));
+    // device -> host: this pair's results
+    HGA_TRY(record_cuda(cudaMemcpyAsync((char*)O_host + c * q_c, dOut + c * q_c, q_c, cudaMemcpyDeviceToHost, pipe->out)));
+    if (bwd) {
+      HGA_TRY(record_cuda(cudaMemcpyAsync((char*)dQ_host + c * q_c, ddQ + c * q_c, q_c, cudaMemcpyDeviceToHost, pipe->out)));
+      HGA_TRY(record_cuda(cudaMemcpyAsync((char*)dK_host + c * kv32_c, ddK + c * kv32_c, kv32_c, cudaMemcpyDeviceToHost, pipe->out)));
+      HGA_TRY(record_cuda(cudaMemcpyAsync((char*)dV_host + c * kv32_c, ddV + c * kv32_c, kv32_c, cudaMemcpyDeviceToHost, pipe->out)));
+    }
+  }
+  HGA_TRY(record_cuda(cudaEventRecord(pipe->join, pipe->out)));
+  HGA_TRY(record_cuda(cudaStreamWaitEvent(st, pipe->join, 0)));
+#undef HGA_TRY
+  return HGA_OK;
 }
 
 }  // extern "C"
