@@ -228,6 +228,54 @@ def config_dict(cfg, args):
             "l2": "flushed between timed steps (512 MiB write)", "parallelism": "dp%d" % args.gpus}
 
 
+def time_tbptt_walk(cfg, args, stream):
+    """hga_tbptt_walk over a fresh synthetic sequence of cfg.total_len tokens in segments of
+    cfg.seg_len (same generator, every token a query); tokens/s counts every token once."""
+    import torch
+    from paper_2607_15105_b200 import binding
+    from paper_2607_15105_b200.workloads import make_inputs
+    L, S = cfg.total_len, cfg.seg_len
+    n_seg = L // S
+    y = make_inputs(cfg.scaled(seg_len=L, seed=cfg.seed + 77))
+    dev = "cuda"
+    as_bf16 = lambda a: torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+    Q, K, V, dO = as_bf16(y["Q"]), as_bf16(y["K"]), as_bf16(y["V"]), as_bf16(y["dO"])
+    del y
+    B, Hq, Hkv, d = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    nqb, kc, kge = S // cfg.q_block, cfg.topk_chunks, min(cfg.topk_groups, cfg.chunk // cfg.group)
+    p = binding.make_params(cfg)
+    cs = torch.zeros(B, Hkv, L // cfg.chunk, d, dtype=torch.bfloat16, device=dev)
+    gs = torch.zeros(B, Hkv, L // cfg.group, d, dtype=torch.bfloat16, device=dev)
+    ci = torch.zeros(n_seg, B, Hkv, nqb, max(kc, 1), dtype=torch.int32, device=dev)
+    gi = torch.zeros(n_seg, B, Hkv, nqb, max(kc * kge, 1), dtype=torch.int32, device=dev)
+    ng = torch.zeros(n_seg, B, Hkv, nqb, dtype=torch.int32, device=dev)
+    O, dQ = torch.zeros_like(Q), torch.zeros_like(Q)
+    LSE = torch.zeros(n_seg, B, Hq, S, dtype=torch.float32, device=dev)
+    dK = torch.zeros(n_seg, B, Hkv, S, d, dtype=torch.float32, device=dev)
+    dV = torch.zeros_like(dK)
+    rb, bb = binding.hga_workspace_bytes(p)
+    ws = torch.empty(rb + bb + 512, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def run():
+        binding.hga_tbptt_walk(p, Q, K, V, dO, cs, gs, ci, gi, ng, O, LSE, dQ, dK, dV, ws, status)
+
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize()
+    reps = max(3, min(args.steps, 10))
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in ev:
+        a.record(stream)
+        run()
+        b.record(stream)
+    torch.cuda.synchronize()
+    ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+    return {"tokens_per_s": round(B * L / (ms * 1e-3), 1), "ms_per_sequence": round(ms, 4), "segments": n_seg,
+            "tokens": B * L, "launch": "eager", "device_status_word": int(status.item()),
+            "note": "one layer, forward+backward of every segment (history 0 .. L-S); inputs larger than L2"}
+
+
 # ----------------------------------------------------------------------------- main arm
 
 def main():
@@ -240,6 +288,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA-graph replay")
     ap.add_argument("--flags", type=int, default=0, help="hga_params.flags (debugging)")
+    ap.add_argument("--no-walk", action="store_true",
+                    help="skip the whole-sequence TBPTT walk (every segment of the sequence, one layer)")
     args = ap.parse_args()
     cfg = CONFIGS[args.config]
     if args.impl == "reference":
@@ -382,6 +432,10 @@ def main():
         b.record(stream)
     barrier()
     e2e_ms = np.array([a.elapsed_time(b) for a, b in e2e_ev])
+    # whole-sequence walk (Section 2.2): every segment of a total_len sequence through the path, one layer
+    walk = None
+    if rank == 0 and world == 1 and cfg.backward and not args.no_walk and cfg.history > 0:
+        walk = time_tbptt_walk(cfg, args, stream)
     clocks = sampler.stop() if rank == 0 else None      # sampled across all timed loops above
     status = int(buf.status.item())
 
@@ -436,6 +490,8 @@ def main():
             "paper_context": "217.75 (HGA) / 207.02 (dense) tokens/s: whole-model QLoRA step at 2K on a "
                              "Quadro RTX 5000 (Table 2); another machine and scope, not the target",
         }
+        if walk is not None:
+            line["tbptt_walk"] = walk
         if not args.no_cpu_baseline and world == 1:
             tps, threads, what, _ = oracle_throughput(cfg, x)
             line["cpu_baseline"] = {"value": round(tps, 3), "unit": "tokens/s", "cores": threads,

@@ -83,6 +83,11 @@ typedef struct hga_params {
   int32_t sink, local;                             /* tokens, multiples of c                     */
   float   softmax_scale;                           /* <= 0 selects 1/sqrt(head_dim)              */
   int32_t flags;                                   /* HGA_FLAG_*                                 */
+  int32_t summary_len;                             /* token length the summary buffers are laid
+                                                      out for (>= total_len, multiple of chunk);
+                                                      0 means total_len.  Lets one pair of buffers
+                                                      [B,Hkv,summary_len/c,d], [B,Hkv,summary_len/g,d]
+                                                      serve a sequence walked segment by segment */
   /* element strides of the (batch, head, token) axes; all-zero means dense.  q_stride
    * also describes dQ; o_stride describes O and dO; k_stride / v_stride describe K / V. */
   int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];
@@ -178,6 +183,26 @@ HGA_API int hga_step_host(const hga_params* p, const void* Q_host, const void* K
                   float* dV_host, void* arena, size_t arena_bytes, int32_t* status_word,
                   void* stream);
 HGA_API int hga_step_arena_bytes(const hga_params* p, size_t* bytes);
+
+/* Section 2.2 (training walks a long sequence in fixed-size segments; the K/V of earlier
+ * segments are kept as detached history, gradients never cross a segment boundary): one layer's
+ * forward and backward over a WHOLE sequence, segment by segment, on device buffers.
+ * `p` describes the sequence: total_len = its length L, seg_len = the segment length S
+ * (L % S == 0); strides, where given, are those of the full-length tensors.  Segment s
+ * (s = 0 .. L/S - 1) has history s*S and runs build_summaries([s*S, (s+1)*S)) -> route ->
+ * attn_fwd -> attn_bwd exactly as the four calls above would with total_len = (s+1)*S.
+ *   Q, dO (in), O, dQ (out)  bf16 [B,Hq,L,d]      K, V  bf16 [B,Hkv,L,d]
+ *   chunk_sum, group_sum     bf16 [B,Hkv,L/c,d], [B,Hkv,L/g,d]: written segment by segment
+ *   chunk_idx [L/S,B,Hkv,S/Bq,k_c], group_idx [L/S,B,Hkv,S/Bq,k_c*kg_eff], n_groups [L/S,B,Hkv,S/Bq]
+ *   LSE fp32 [L/S,B,Hq,S]    dK, dV fp32 [L/S,B,Hkv,S,d] (segment s holds the rows of its own tokens)
+ * dO == NULL runs the forward half only (dQ, dK, dV may then be NULL).  p->summary_len is
+ * ignored (the summary buffers are laid out for L).  workspace: device scratch of at least
+ * route_bytes + bwd_bytes as hga_workspace_bytes(p) reports them.  All work is queued on
+ * `stream` in order. */
+HGA_API int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void* V, const void* dO,
+                   void* chunk_sum, void* group_sum, int32_t* chunk_idx, int32_t* group_idx,
+                   int32_t* n_groups, void* O, float* LSE, void* dQ, float* dK, float* dV,
+                   void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
 
 HGA_API const char* hga_status_string(int status);
 HGA_API int hga_version(void);

@@ -22,7 +22,7 @@ HGA_STATUS_WAIT_TIMEOUT = 2
 HGA_ROUTE_STATIC_SCRATCH_BYTES = 4 << 20
 
 EXPORTS = ("hga_build_summaries", "hga_route", "hga_route_static", "hga_attn_fwd", "hga_attn_bwd",
-           "hga_workspace_bytes", "hga_step_host", "hga_step_arena_bytes", "hga_status_string",
+           "hga_workspace_bytes", "hga_step_host", "hga_step_arena_bytes", "hga_tbptt_walk", "hga_status_string",
            "hga_version", "hga_last_cuda_error", "hga_kernel_launch_count")
 
 
@@ -30,7 +30,7 @@ class HgaParams(C.Structure):
     _fields_ = ([(n, C.c_int32) for n in (
         "batch", "n_q_heads", "n_kv_heads", "head_dim", "total_len", "seg_len", "chunk", "group",
         "q_block", "topk_chunks", "topk_groups", "sink", "local")]
-        + [("softmax_scale", C.c_float), ("flags", C.c_int32)]
+        + [("softmax_scale", C.c_float), ("flags", C.c_int32), ("summary_len", C.c_int32)]
         + [(n, C.c_int64 * 3) for n in ("q_stride", "k_stride", "v_stride", "o_stride")])
 
 
@@ -68,16 +68,17 @@ def lib():
         L.hga_workspace_bytes.argtypes = [pp, C.POINTER(sz), C.POINTER(sz)]
         L.hga_step_arena_bytes.argtypes = [pp, C.POINTER(sz)]
         L.hga_step_host.argtypes = [pp] + [vp] * 13 + [sz, vp, vp]
+        L.hga_tbptt_walk.argtypes = [pp] + [vp] * 15 + [sz, vp, vp]
         _lib = L
     return _lib
 
 
 def make_params(cfg, softmax_scale: float = 0.0, flags: int = 0, q_stride=None, k_stride=None,
-                v_stride=None, o_stride=None) -> HgaParams:
+                v_stride=None, o_stride=None, summary_len: int = 0) -> HgaParams:
     """hga_params from any object with the HGA shape fields (e.g. workloads.HgaConfig)."""
     p = HgaParams(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.total_len,
                   cfg.seg_len, cfg.chunk, cfg.group, cfg.q_block, cfg.topk_chunks,
-                  cfg.topk_groups, cfg.sink, cfg.local, softmax_scale, flags)
+                  cfg.topk_groups, cfg.sink, cfg.local, softmax_scale, flags, summary_len)
     for name, s in (("q_stride", q_stride), ("k_stride", k_stride), ("v_stride", v_stride),
                     ("o_stride", o_stride)):
         if s is not None:
@@ -184,6 +185,16 @@ def hga_step_host(p, Q_host, Kseg_host, Vseg_host, dO_host, K_dev, V_dev, chunk_
         C.byref(p), _ptr(Q_host), _ptr(Kseg_host), _ptr(Vseg_host), _ptr(dO_host), _ptr(K_dev),
         _ptr(V_dev), _ptr(chunk_sum), _ptr(group_sum), _ptr(O_host), _ptr(dQ_host), _ptr(dK_host),
         _ptr(dV_host), _ptr(arena), nbytes, _ptr(status_word), _stream(stream)))
+
+
+def hga_tbptt_walk(p, Q, K, V, dO, chunk_sum, group_sum, chunk_idx, group_idx, n_groups, O, LSE, dQ,
+                   dK, dV, workspace, status_word=None, stream=None):
+    """One layer over a whole sequence, segment by segment (all tensors CUDA; see hga.h)."""
+    nbytes = workspace.numel() * workspace.element_size()
+    _check("hga_tbptt_walk", lib().hga_tbptt_walk(
+        C.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(chunk_sum), _ptr(group_sum),
+        _ptr(chunk_idx), _ptr(group_idx), _ptr(n_groups), _ptr(O), _ptr(LSE), _ptr(dQ), _ptr(dK),
+        _ptr(dV), _ptr(workspace), nbytes, _ptr(status_word), _stream(stream)))
 
 
 class HgaLayerBuffers:

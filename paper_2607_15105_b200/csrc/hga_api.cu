@@ -51,6 +51,9 @@ static int resolve(const hga_params* p, Dims& dm) {
   dm.kge = dm.kg < dm.per ? dm.kg : dm.per;
   dm.sink = p->sink; dm.local = p->local;
   dm.NQB = dm.S / dm.Bq; dm.Nc = dm.L / dm.c; dm.Ng = dm.L / dm.g;
+  if (p->summary_len != 0 && (p->summary_len < p->total_len || p->summary_len % p->chunk)) return HGA_ERR_SHAPE;
+  dm.NcS = (p->summary_len ? p->summary_len : dm.L) / dm.c;
+  dm.NgS = (p->summary_len ? p->summary_len : dm.L) / dm.g;
   dm.width = dm.kc * dm.kge; dm.rows = dm.G * dm.Bq;
   dm.flags = p->flags;
   dm.scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)dm.d);
@@ -309,7 +312,7 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   const size_t kvseg_c = (size_t)dm.S * dm.d * 2, kv32_c = (size_t)dm.S * dm.d * 4;
   const size_t kv_c = (size_t)dm.L * dm.d * 2;                 // one (batch, kv head) of the resident K / V
   const size_t hist = (size_t)dm.H * dm.d * 2;
-  const size_t cs_c = (size_t)dm.Nc * dm.d * 2, gs_c = (size_t)dm.Ng * dm.d * 2;
+  const size_t cs_c = (size_t)dm.NcS * dm.d * 2, gs_c = (size_t)dm.NgS * dm.d * 2;
 #define HGA_TRY(x) do { rc = (x); if (rc) return rc; } while (0)
   HGA_TRY(record_cuda(cudaEventRecord(pipe->fork, st)));
   HGA_TRY(record_cuda(cudaStreamWaitEvent(pipe->in, pipe->fork, 0)));
@@ -355,6 +358,65 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   HGA_TRY(record_cuda(cudaEventRecord(pipe->join, pipe->out)));
   HGA_TRY(record_cuda(cudaStreamWaitEvent(st, pipe->join, 0)));
 #undef HGA_TRY
+  return HGA_OK;
+}
+
+int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void* V, const void* dO,
+                   void* chunk_sum, void* group_sum, int32_t* chunk_idx, int32_t* group_idx,
+                   int32_t* n_groups, void* O, float* LSE, void* dQ, float* dK, float* dV,
+                   void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream) {
+  if (!p) return HGA_ERR_NULL;
+  if (p->seg_len < 1 || p->total_len < p->seg_len || p->total_len % p->seg_len) return HGA_ERR_SHAPE;
+  hga_params full = *p;                 // the last segment's problem: validates shapes, resolves the full-length strides
+  full.summary_len = 0;
+  Dims dmf;
+  int rc = resolve(&full, dmf);
+  if (rc) return rc;
+  if (!Q || !K || !V || !chunk_sum || !group_sum || !group_idx || !n_groups || !O || !LSE || !workspace)
+    return HGA_ERR_NULL;
+  if (dmf.kc > 0 && !chunk_idx) return HGA_ERR_NULL;
+  const bool bwd = dO != nullptr;
+  if (bwd && (!dQ || !dK || !dV)) return HGA_ERR_NULL;
+  const size_t route_ws = route_workspace_bytes(dmf), bwd_ws = bwd_workspace_bytes(dmf);
+  const size_t route_ws_up = (route_ws + 255) & ~(size_t)255;
+  if (workspace_bytes < route_ws_up + bwd_ws) return HGA_ERR_WORKSPACE;
+  const int S = p->seg_len, n_seg = p->total_len / S;
+  // full-length strides (elements): dmf's token counts are those of the last segment (S active rows,
+  // L keys), so the Q/O strides are rebuilt for L rows when the caller gave none
+  hga_params ps = *p;
+  ps.summary_len = p->total_len;
+  const int64_t zero[3] = {0, 0, 0};
+  const int64_t d = p->head_dim, L = p->total_len;
+  auto fill = [&](int64_t* s, const int64_t* given, int heads) {
+    if (memcmp(given, zero, sizeof zero) == 0) { s[2] = d; s[1] = L * d; s[0] = (int64_t)heads * L * d; }
+  };
+  fill(ps.q_stride, p->q_stride, p->n_q_heads);
+  fill(ps.o_stride, p->o_stride, p->n_q_heads);
+  fill(ps.k_stride, p->k_stride, p->n_kv_heads);
+  fill(ps.v_stride, p->v_stride, p->n_kv_heads);
+  const size_t items = (size_t)dmf.B * dmf.Hkv * dmf.NQB;
+  const size_t lse_seg = (size_t)dmf.B * dmf.Hq * S, kv_seg = (size_t)dmf.B * dmf.Hkv * S * dmf.d;
+  for (int s = 0; s < n_seg; ++s) {
+    ps.total_len = (s + 1) * S;
+    const int64_t q_off = (int64_t)s * S * ps.q_stride[2] * 2, o_off = (int64_t)s * S * ps.o_stride[2] * 2;   // bytes
+    const char* Qs = (const char*)Q + q_off;
+    char* Os = (char*)O + o_off;
+    int32_t* ci = chunk_idx ? chunk_idx + s * items * dmf.kc : nullptr;
+    int32_t* gi = group_idx + s * items * dmf.width;
+    int32_t* ng = n_groups + s * items;
+    float* lse = LSE + s * lse_seg;
+    rc = hga_build_summaries(&ps, K, s * S, (s + 1) * S, chunk_sum, group_sum, stream);
+    if (rc) return rc;
+    rc = hga_route(&ps, Qs, chunk_sum, group_sum, ci, gi, ng, nullptr, nullptr, workspace, route_ws, stream);
+    if (rc) return rc;
+    rc = hga_attn_fwd(&ps, Qs, K, V, gi, ng, Os, lse, status_word, stream);
+    if (rc) return rc;
+    if (bwd) {
+      rc = hga_attn_bwd(&ps, Qs, K, V, Os, lse, (const char*)dO + o_off, gi, ng, (char*)dQ + q_off,
+                        dK + s * kv_seg, dV + s * kv_seg, (char*)workspace + route_ws_up, bwd_ws, status_word, stream);
+      if (rc) return rc;
+    }
+  }
   return HGA_OK;
 }
 

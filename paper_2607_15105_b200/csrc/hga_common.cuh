@@ -17,6 +17,7 @@ struct Dims {
   int kc, kg, kge, per; // k_c, k_g, min(k_g, c/g), c/g
   int sink, local;
   int NQB, Nc, Ng;      // query blocks per sequence, chunks, groups
+  int NcS, NgS;         // rows per (batch, kv head) in the chunk / group summary buffers (>= Nc, Ng)
   int width;            // group_idx entries per item = kc * kge
   int rows;             // G * Bq query rows per item
   int flags;

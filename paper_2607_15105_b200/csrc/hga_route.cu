@@ -95,7 +95,7 @@ k_chunk_scores(const uint16_t* __restrict__ Q, const uint16_t* __restrict__ chun
   }
   __syncthreads();
   const uint16_t* Qitem = Q + b * dm.qs[0] + (int64_t)(h * dm.G) * dm.qs[1] + (int64_t)(qb * dm.Bq) * dm.qs[2];
-  score_tile<D>(dm, Qitem, chunk_sum + (int64_t)bh * dm.Nc * D, s_rows, s_sum, s_q, s_red, s_out);
+  score_tile<D>(dm, Qitem, chunk_sum + (int64_t)bh * dm.NcS * D, s_rows, s_sum, s_q, s_red, s_out);
   if (threadIdx.x < kScoreTile && base + threadIdx.x < n_cand)
     scores[(int64_t)item * dm.Nc + j0 + base + threadIdx.x] = s_out[threadIdx.x];
 }
@@ -207,7 +207,7 @@ k_route_groups(const uint16_t* __restrict__ Q, const uint16_t* __restrict__ grou
                         ? ci[i / dm.per] * dm.per + (i % dm.per) : -1;
     }
     __syncthreads();
-    score_tile<D>(dm, Qitem, group_sum + (int64_t)bh * dm.Ng * D, s_rows, s_sum, s_q, s_red, s_out);
+    score_tile<D>(dm, Qitem, group_sum + (int64_t)bh * dm.NgS * D, s_rows, s_sum, s_q, s_red, s_out);
     if (group_scores_out && tid < chunks_per_tile * dm.per && base + tid < total)
       group_scores_out[(int64_t)item * dm.kc * dm.per + base + tid] = s_out[tid];
     // one thread per opened chunk of this tile: top-kg_eff of its `per` groups.  Chunks are

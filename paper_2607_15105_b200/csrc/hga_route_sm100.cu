@@ -338,8 +338,8 @@ static int launch_route(const Dims& dm, const void* Q, const void* chunk_sum, co
   const uint64_t dc[5] = {64, (uint64_t)dm.Nc, (uint64_t)(D / 64), (uint64_t)dm.Hkv, (uint64_t)dm.B};
   const uint64_t dg[5] = {64, (uint64_t)dm.Ng, (uint64_t)(D / 64), (uint64_t)dm.Hkv, (uint64_t)dm.B};
   const uint64_t sq[4] = {(uint64_t)dm.qs[2] * 2, 128, (uint64_t)dm.qs[1] * 2, (uint64_t)dm.qs[0] * 2};
-  const uint64_t sc[4] = {(uint64_t)D * 2, 128, (uint64_t)dm.Nc * D * 2, (uint64_t)dm.Hkv * dm.Nc * D * 2};
-  const uint64_t sg[4] = {(uint64_t)D * 2, 128, (uint64_t)dm.Ng * D * 2, (uint64_t)dm.Hkv * dm.Ng * D * 2};
+  const uint64_t sc[4] = {(uint64_t)D * 2, 128, (uint64_t)dm.NcS * D * 2, (uint64_t)dm.Hkv * dm.NcS * D * 2};
+  const uint64_t sg[4] = {(uint64_t)D * 2, 128, (uint64_t)dm.NgS * D * 2, (uint64_t)dm.Hkv * dm.NgS * D * 2};
   if (encode_tensor_map_bf16(&mq, Q, 5, dq, sq, box, true) ||
       encode_tensor_map_bf16(&mc, chunk_sum, 5, dc, sc, box, true) ||
       encode_tensor_map_bf16(&mg, group_sum, 5, dg, sg, box, true))

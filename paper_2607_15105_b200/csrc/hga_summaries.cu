@@ -57,7 +57,7 @@ k_build_summaries(const uint16_t* __restrict__ K, Dims dm, int chunk_begin,
       csum[2 * e] += s[2 * e];
       csum[2 * e + 1] += s[2 * e + 1];
     }
-    const int64_t m = (int64_t)bh * dm.Ng + (int64_t)j * dm.per + u;
+    const int64_t m = (int64_t)bh * dm.NgS + (int64_t)j * dm.per + u;
     *reinterpret_cast<uint4*>(group_sum + m * D + v * 8) = make_uint4(o[0], o[1], o[2], o[3]);
   }
 #pragma unroll
@@ -75,7 +75,7 @@ k_build_summaries(const uint16_t* __restrict__ K, Dims dm, int chunk_begin,
       o[e] = (uint32_t)f64_to_bf16_once(a / (double)dm.c) |
              ((uint32_t)f64_to_bf16_once(c2 / (double)dm.c) << 16);
     }
-    const int64_t jj = (int64_t)bh * dm.Nc + j;
+    const int64_t jj = (int64_t)bh * dm.NcS + j;
     *reinterpret_cast<uint4*>(chunk_sum + jj * D + v * 8) = make_uint4(o[0], o[1], o[2], o[3]);
   }
 }
