@@ -73,7 +73,8 @@ class HgaConfig:
         return replace(self, **kw)
 
 
-# The five benchmark configurations (seed = 1337 + configuration number).
+# The five benchmark configurations (seed = 1337 + configuration number), plus a sixth in the
+# paper's own default routing shape: eight selected chunks opened whole (k_g = c/g), Section 3 / Table 1.
 CONFIGS = {
     1: HgaConfig("cfg1_tiny_1k", 1, 2, 1, 64, 1024, 256, 64, 8, 64, 4, 4, 64, 64,
                  topics=8, needles=0, backward=True, seed=1338),
@@ -85,6 +86,8 @@ CONFIGS = {
                  topics=1024, needles=32, backward=False, seed=1341),
     5: HgaConfig("cfg5_stress_b4_64k", 4, 32, 8, 128, 65536, 4096, 128, 16, 128, 32, 4, 128, 256,
                  topics=0, needles=0, backward=True, seed=1342),
+    6: HgaConfig("cfg6_paper_default_16k", 1, 32, 8, 128, 16384, 2048, 64, 8, 64, 8, 8, 64, 128,
+                 topics=256, needles=32, backward=True, seed=1343),
 }
 
 

@@ -1,4 +1,4 @@
-"""The five benchmark configurations at full size, in the launch configuration bench.py times:
+"""The benchmark configurations at full size, in the launch configuration bench.py times:
 the whole path runs on the GPU; the oracle recomputes sampled items (all query blocks of one
 (batch, kv head) so that its dK/dV rows are complete, plus a few scattered items)."""
 import numpy as np
@@ -26,11 +26,11 @@ def sample_items(cfg, full_head, extra, seed):
 
 
 # routed keys per item (a data-independent count) for the last query block of each config
-ROUTED_KEYS_LAST_BLOCK = {1: 320, 2: 512, 3: 768, 4: 768, 5: 2560}
+ROUTED_KEYS_LAST_BLOCK = {1: 320, 2: 512, 3: 768, 4: 768, 5: 2560, 6: 768}
 
 
 @pytest.mark.parametrize("n,full_head,extra", [(1, (0, 0), 4), (2, (0, 5), 12), (3, (0, 3), 12),
-                                               (4, (0, 6), 0), (5, (2, 5), 0)])
+                                               (4, (0, 6), 0), (5, (2, 5), 0), (6, (0, 1), 8)])
 def test_config_against_oracle(n, full_head, extra):
     cfg = CONFIGS[n]
     x = make_inputs(cfg)
