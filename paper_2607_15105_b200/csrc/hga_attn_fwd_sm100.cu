@@ -302,27 +302,33 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // rounding of a dominant weight cancel.
         HGA_TRACE_POINT(13);
         const float neg_m = -m_used;
-        float la = 0.f, lb = 0.f, ra = 0.f, rb = 0.f;
+        // two columns per step on packed fp32 pairs: one FMA for both arguments, one add each for the
+        // exact and the rounded sums (the row threads are issue-bound when two CTAs share the SM)
+        const uint64_t sl2_2 = pack_f32x2(sl2, sl2), neg_m2 = pack_f32x2(neg_m, neg_m);
+        uint64_t lsum = pack_f32x2(0.f, 0.f), rsum = pack_f32x2(0.f, 0.f);
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            float p0 = fast_exp2(fmaf(__uint_as_float(x[c][2 * i]), sl2, neg_m));
-            float p1 = fast_exp2(fmaf(__uint_as_float(x[c][2 * i + 1]), sl2, neg_m));
+            float a0, a1;
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[c][2 * i]), __uint_as_float(x[c][2 * i + 1])), sl2_2, neg_m2),
+                         a0, a1);
+            float p0 = fast_exp2(a0), p1 = fast_exp2(a1);
             if (vis < kFT) {                              // diagonal / ragged tile only
               if (32 * c + 2 * i >= vis) p0 = 0.f;
               if (32 * c + 2 * i + 1 >= vis) p1 = 0.f;
             }
-            la += p0;
-            lb += p1;
+            lsum = add_f32x2(lsum, pack_f32x2(p0, p1));
             const __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
             pk[i] = *reinterpret_cast<const uint32_t*>(&hh);
-            ra += __uint_as_float(pk[i] << 16);
-            rb += __uint_as_float(pk[i] & 0xffff0000u);
+            rsum = add_f32x2(rsum, pack_f32x2(__uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u)));
           }
           tmem_st16(s_addr + c * 16, pk);
         }
+        float la, lb, ra, rb;
+        unpack_f32x2(lsum, la, lb);
+        unpack_f32x2(rsum, ra, rb);
         l += la + lb;
         l_mma += ra + rb;
         HGA_TRACE_POINT(14);
