@@ -250,22 +250,22 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tc_fence_after_sync();
         HGA_TRACE_POINT(11);     // waiting for S
         const int vis = limit - kFT * j;                  // visible columns of this tile (may be <= 0)
-        uint32_t x[2][32];
-        tmem_ld32(s_addr, x[0]);
-        tmem_ld32(s_addr + 32, x[1]);
-        tmem_wait_ld();
+        // S is read from TMEM twice (row maximum, then exponentials), 32 columns at a time: holding
+        // all 64 values across both passes costs more registers than the budget of two CTAs per SM allows
         float mxs[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-        if (vis >= kFT) {
 #pragma unroll
-          for (int c = 0; c < 2; ++c)
+        for (int c = 0; c < 2; ++c) {
+          uint32_t x[32];
+          tmem_ld32(s_addr + 32 * c, x);
+          tmem_wait_ld();
+          if (vis >= kFT) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mxs[i & 3] = fmaxf(mxs[i & 3], __uint_as_float(x[c][i]));
-        } else {
-#pragma unroll
-          for (int c = 0; c < 2; ++c)
+            for (int i = 0; i < 32; ++i) mxs[i & 3] = fmaxf(mxs[i & 3], __uint_as_float(x[i]));
+          } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (32 * c + i < vis) mxs[i & 3] = fmaxf(mxs[i & 3], __uint_as_float(x[c][i]));
+              if (32 * c + i < vis) mxs[i & 3] = fmaxf(mxs[i & 3], __uint_as_float(x[i]));
+          }
         }
         const float mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])) * sl2;
         HGA_TRACE_POINT(12);
@@ -308,11 +308,13 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         uint64_t lsum = pack_f32x2(0.f, 0.f), rsum = pack_f32x2(0.f, 0.f);
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
-          uint32_t pk[16];
+          uint32_t x[32], pk[16];
+          tmem_ld32(s_addr + 32 * c, x);       // (P of the first half lands in columns 0-15: already consumed)
+          tmem_wait_ld();
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             float a0, a1;
-            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[c][2 * i]), __uint_as_float(x[c][2 * i + 1])), sl2_2, neg_m2),
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1])), sl2_2, neg_m2),
                          a0, a1);
             float p0 = fast_exp2(a0), p1 = fast_exp2(a1);
             if (vis < kFT) {                              // diagonal / ragged tile only
