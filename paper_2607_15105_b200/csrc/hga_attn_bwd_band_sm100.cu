@@ -233,6 +233,8 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
     for (int m = wg; m < n_steps; m += 2) {
       const float neg_lse2 = -lse * 1.4426950408889634f;
       const float neg_delta_s = -dl * dm.scale;
+      const uint64_t sl2_2 = pack_f32x2(sl2, sl2), neg_lse2_2 = pack_f32x2(neg_lse2, neg_lse2);
+      const uint64_t scale_2 = pack_f32x2(dm.scale, dm.scale), neg_delta_s_2 = pack_f32x2(neg_delta_s, neg_delta_s);
       const int vis_m = vis;
       if (m + 2 < n_steps) row_of(m + 2, lse, dl, vis);      // prefetch the next M-tile's row data
       ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[wg], (m >> 1) & 1, abort));
@@ -256,14 +258,16 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
         uint32_t pk[8], dk[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), sl2, neg_lse2));
-          float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), sl2, neg_lse2));
+          // packed fp32 pairs: one FMA-pipe instruction for two columns
+          float a0, a1, d0, d1;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), sl2_2, neg_lse2_2), a0, a1);
+          float p0 = fast_exp2(a0), p1 = fast_exp2(a1);
           if (vis_m < kKT) {                  // the tile's own query block: causal mask
             if (q4 * 16 + 2 * i >= vis_m) p0 = 0.f;
             if (q4 * 16 + 2 * i + 1 >= vis_m) p1 = 0.f;
           }
-          const float d0 = p0 * fmaf(__uint_as_float(dp[2 * i]), dm.scale, neg_delta_s);
-          const float d1 = p1 * fmaf(__uint_as_float(dp[2 * i + 1]), dm.scale, neg_delta_s);
+          const uint64_t g2 = fma_f32x2(pack_f32x2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])), scale_2, neg_delta_s_2);
+          unpack_f32x2(mul_f32x2(pack_f32x2(p0, p1), g2), d0, d1);
           pk[i] = pack_bf16(p0, p1);
           dk[i] = pack_bf16(d0, d1);
         }

@@ -485,6 +485,8 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
     }
     // ---- paired steps: warpgroup wg owns the wg-th tile of each pair (64 of the 128 columns)
+    const uint64_t sl2_2 = pack_f32x2(sl2, sl2), neg_lse2_2 = pack_f32x2(neg_lse2, neg_lse2);
+    const uint64_t scale_2 = pack_f32x2(dm.scale, dm.scale), neg_delta_s_2 = pack_f32x2(neg_delta_s, neg_delta_s);
     int rs = 0;
     for (int u = 0; u < n_pairs && ok; ++u) {
       const int rp = rs == 2 ? 0 : rs + 1;
@@ -504,8 +506,9 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tmem_wait_ld();
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), sl2, neg_lse2));
-          float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), sl2, neg_lse2));
+          float a0, a1;            // packed fp32 pairs: one FMA for the two exponent arguments
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), sl2_2, neg_lse2_2), a0, a1);
+          float p0 = fast_exp2(a0), p1 = fast_exp2(a1);
           if (vis < kKT) {
             if (q4 * 16 + 2 * i >= vis) p0 = 0.f;
             if (q4 * 16 + 2 * i + 1 >= vis) p1 = 0.f;
@@ -524,10 +527,10 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tmem_wait_ld();
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float p0 = __uint_as_float(pk[8 * q4 + i] << 16);
-          const float p1 = __uint_as_float(pk[8 * q4 + i] & 0xffff0000u);
-          const float d0 = p0 * fmaf(__uint_as_float(dp[2 * i]), dm.scale, neg_delta_s);
-          const float d1 = p1 * fmaf(__uint_as_float(dp[2 * i + 1]), dm.scale, neg_delta_s);
+          const uint64_t p2 = pack_f32x2(__uint_as_float(pk[8 * q4 + i] << 16), __uint_as_float(pk[8 * q4 + i] & 0xffff0000u));
+          const uint64_t g2 = fma_f32x2(pack_f32x2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])), scale_2, neg_delta_s_2);
+          float d0, d1;
+          unpack_f32x2(mul_f32x2(p2, g2), d0, d1);
           dk[i] = pack_bf16(d0, d1);
         }
         // bf16 dS over the dP columns already read (8 columns per 16 keys): the A operand of dQ
