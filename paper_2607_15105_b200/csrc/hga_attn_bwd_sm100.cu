@@ -70,7 +70,7 @@ struct BwdSmem {
   uint64_t phase_a_done;                                // every GEMM of the dK/dV steps is complete
   uint64_t kp_full[kBwdKStages / 2], kp_empty[kBwdKStages], vp_full;       // paired steps: one barrier per pair of stages
                                                         // (kp_empty: indexed by pair number mod 6, see dp_full)
-  uint64_t dq_done;
+  uint64_t dq_done, dq_staged;
   uint32_t tmem_base;
   int n_oct, dkv_lo, n_dkv;    // tiles [dkv_lo, dkv_lo + n_dkv) are processed as dK/dV steps
   volatile int abort;
@@ -88,8 +88,8 @@ __device__ __forceinline__ float dot4_bf16(uint2 x, uint2 y) {
 __global__ void __launch_bounds__(kBwdThreads, 1)
 k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
                  const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                 const float* __restrict__ delta_ws, const float* __restrict__ LSE, const int32_t* __restrict__ group_idx,
-                 const int32_t* __restrict__ n_groups, Dims dm, uint16_t* __restrict__ dQ,
+                 const __grid_constant__ CUtensorMap map_dq, const float* __restrict__ delta_ws, const float* __restrict__ LSE, const int32_t* __restrict__ group_idx,
+                 const int32_t* __restrict__ n_groups, Dims dm,
                  float* __restrict__ dK, float* __restrict__ dV, int band_done, int32_t* status_word) {
   constexpr int D = kBwdD;
   // TMEM columns.  Regions 0, 1, 2 rotate through the roles S / dP+dS of the paired steps; a dK/dV
@@ -122,7 +122,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     for (int s = 0; s < kBwdKStages / 2; ++s) mbar_init(&sm.kp_full[s], 1);
     for (int s = 0; s < kBwdKStages; ++s) mbar_init(&sm.kp_empty[s], 1);
     mbar_init(&sm.vp_full, 2);
-    mbar_init(&sm.dq_done, 1);
+    mbar_init(&sm.dq_done, 1); mbar_init(&sm.dq_staged, 256);
     sm.abort = 0;
     fence_barrier_init();
   }
@@ -430,9 +430,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int wg = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int row_in_tile = quarter * 32 + lane;
-    const int r = mt * 128 + row_in_tile;
-    const int a = r / dm.Bq, t = r % dm.Bq;
-    const int hq = h * dm.G + a, srow = qb * dm.Bq + t;
+    const int t = (mt * 128 + row_in_tile) % dm.Bq;         // position of the row inside its query block
     const int limit = n_keys - dm.Bq + t + 1;
     const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
     const float sl2 = dm.scale * 1.4426950408889634f;
@@ -545,22 +543,36 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.dq_done, 0, abort));
     HGA_TRACE_POINT(20);
     if (ok) {
-      // dQ epilogue: each warpgroup writes half of the row (64 columns)
+      // dQ epilogue through shared memory and TMA: a thread's own row is 256 bytes away from its
+      // neighbour's, so direct 16-byte stores would touch 32 different sectors per instruction.
+      // Warpgroup wg holds columns 64*wg .. 64*wg+63 of its rows = panel wg of the Q-shaped tile,
+      // which goes into Q's shared memory (all GEMMs that read it are complete) in the swizzled
+      // [panel][128 rows][128 B] layout and leaves as four boxes.
       tc_fence_after_sync();
-      uint16_t* qrow = dQ + b * dm.qs[0] + hq * dm.qs[1] + (int64_t)srow * dm.qs[2] + wg * 64;
       uint32_t x[2][32];
       tmem_ld32(lane_base + kColDQ + wg * 64, x[0]);
       tmem_ld32(lane_base + kColDQ + wg * 64 + 32, x[1]);
       tmem_wait_ld();
+      const uint32_t key = (uint32_t)(row_in_tile & 7);
+      const uint32_t line = smem_u32(sm.q) + (uint32_t)wg * 16384 + (uint32_t)row_in_tile * 128;
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint4* dst = reinterpret_cast<uint4*>(qrow + c * 32);
+      for (int c = 0; c < 2; ++c)
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          dst[i] = make_uint4(pack_bf16(__uint_as_float(x[c][8 * i]), __uint_as_float(x[c][8 * i + 1])),
-                              pack_bf16(__uint_as_float(x[c][8 * i + 2]), __uint_as_float(x[c][8 * i + 3])),
-                              pack_bf16(__uint_as_float(x[c][8 * i + 4]), __uint_as_float(x[c][8 * i + 5])),
-                              pack_bf16(__uint_as_float(x[c][8 * i + 6]), __uint_as_float(x[c][8 * i + 7])));
+          st_shared_v4(line + (((uint32_t)(4 * c + i) ^ key) * 16),
+                       pack_bf16(__uint_as_float(x[c][8 * i]), __uint_as_float(x[c][8 * i + 1])),
+                       pack_bf16(__uint_as_float(x[c][8 * i + 2]), __uint_as_float(x[c][8 * i + 3])),
+                       pack_bf16(__uint_as_float(x[c][8 * i + 4]), __uint_as_float(x[c][8 * i + 5])),
+                       pack_bf16(__uint_as_float(x[c][8 * i + 6]), __uint_as_float(x[c][8 * i + 7])));
+      fence_proxy_async_smem();
+      mbar_arrive(&sm.dq_staged);
+      if (warp == 2 && lane < 4 && bwd_wait(&sm.dq_staged, 0, abort)) {      // all 256 rows are in shared memory
+        const int half = lane & 1, panel = lane >> 1;
+        const int r0 = mt * 128 + 64 * half;
+        tma_store_5d(&map_dq, sm.q + panel * 16384 + half * 8192, 0, qb * dm.Bq + r0 % dm.Bq, panel,
+                     h * dm.G + r0 / dm.Bq, b);
+        tma_store_commit();
+        tma_store_wait_all();
       }
     }
   } else {
@@ -659,7 +671,7 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
                           const float* LSE, const void* dO, const int32_t* group_idx,
                           const int32_t* n_groups, void* dQ, float* dK, float* dV, float* delta_ws,
                           bool zero_grads, int32_t* status_word, cudaStream_t st) {
-  CUtensorMap mq, mdo, mk, mv;
+  CUtensorMap mq, mdo, mk, mv, mdq;
   const uint32_t box[5] = {64, 8, 2, 1, 1};
   const uint32_t box_q[5] = {64, 64, 1, 1, 1};
   const uint64_t dq[5] = {64, (uint64_t)dm.S, 2, (uint64_t)dm.Hq, (uint64_t)dm.B};
@@ -670,6 +682,7 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
   const uint64_t sv[4] = {(uint64_t)dm.vs[2] * 2, 128, (uint64_t)dm.vs[1] * 2, (uint64_t)dm.vs[0] * 2};
   if (encode_tensor_map_bf16(&mq, Q, 5, dq, sq, box_q, true) ||
       encode_tensor_map_bf16(&mdo, dO, 5, dq, so, box_q, true) ||
+      encode_tensor_map_bf16(&mdq, dQ, 5, dq, sq, box_q, true) ||
       encode_tensor_map_bf16(&mk, K, 5, dk, sk, box, true) ||
       encode_tensor_map_bf16(&mv, V, 5, dk, sv, box, true))
     return HGA_ERR_UNSUPPORTED;
@@ -700,8 +713,8 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
     if ((e = cudaMemsetAsync(dV, 0, bytes, st)) != cudaSuccess) return record_cuda(e);
   }
   const int units = dm.B * dm.Hkv * dm.NQB * (dm.rows / 128);
-  k_attn_bwd_sm100<<<units, kBwdThreads, smem, st>>>(mq, mdo, mk, mv, delta_ws, LSE, group_idx, n_groups, dm,
-                                                    (uint16_t*)dQ, dK, dV, band_done, status_word);
+  k_attn_bwd_sm100<<<units, kBwdThreads, smem, st>>>(mq, mdo, mk, mv, mdq, delta_ws, LSE, group_idx, n_groups, dm,
+                                                    dK, dV, band_done, status_word);
   count_launch(2);
   return record_cuda(cudaGetLastError());
 }
