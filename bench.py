@@ -84,8 +84,8 @@ def active_group_pairs(cfg, group_idx, n_groups):
 
 # dram__bytes_read.sum + dram__bytes_write.sum per call, summed over the call's kernels, from the
 # ncu captures summarised under profiles/ (forward: k_attn_fwd_sm100; backward: k_bwd_delta_sm100
-# 33.58 MB + k_attn_bwd_band_sm100 42.94 MB + k_attn_bwd_sm100 88.62 MB).
-NCU_TRAFFIC_BYTES = {3: {"hga_attn_fwd": 64.08e6, "hga_attn_bwd": 165.14e6}}
+# 33.58 MB + k_attn_bwd_band_sm100 42.88 MB + k_attn_bwd_sm100 88.73 MB).
+NCU_TRAFFIC_BYTES = {3: {"hga_attn_fwd": 63.34e6, "hga_attn_bwd": 165.19e6}}
 
 
 def roofline_entry(name, flops, nbytes, seconds, peaks, sustained=False):
