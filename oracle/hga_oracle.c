@@ -201,8 +201,10 @@ int hga_ref_route(const hga_ref_params* p, const uint16_t* Q, const uint16_t* ch
     int j0 = se / c, n_cand = (ls - se) / c;
     int n_rows = G * Bq;
     double* rows = (double*)malloc(sizeof(double) * (size_t)n_rows * d);
-    double* sc = (double*)malloc(sizeof(double) * (size_t)(n_cand > per ? n_cand : per) + 8);
-    char* taken = (char*)malloc((size_t)(n_cand > per ? n_cand : per) + 8);
+    /* room for the candidate chunk scores, or for the group scores of all selected chunks */
+    size_t n_sc = (size_t)(n_cand > kc * per ? n_cand : kc * per) + 8;
+    double* sc = (double*)malloc(sizeof(double) * n_sc);
+    char* taken = (char*)malloc(n_sc);
     if (!rows || !sc || !taken) { failed = 1; free(rows); free(sc); free(taken); continue; }
     for (int a = 0; a < G; ++a)
       for (int t = 0; t < Bq; ++t)
@@ -226,17 +228,30 @@ int hga_ref_route(const hga_ref_params* p, const uint16_t* Q, const uint16_t* ch
     int nsel = 0;
     for (int i = 0; i < n_cand; ++i)
       if (taken[i]) ci[nsel++] = j0 + i; /* ascending */
-    /* item 2: open each selected chunk, keep its k_g best groups */
     int ng = 0;
-    for (int r = 0; r < nsel; ++r) {
-      int m0 = ci[r] * per;
-      for (int u = 0; u < per; ++u) {
-        sc[u] = block_score(rows, n_rows, d, group_sum + (bh * Ng + m0 + u) * (long)d);
-        if (group_scores) group_scores[item * (long)kc * per + (long)r * per + u] = sc[u];
+    if (!p->global_group_budget) {
+      /* item 2: open each selected chunk, keep its k_g best groups */
+      for (int r = 0; r < nsel; ++r) {
+        int m0 = ci[r] * per;
+        for (int u = 0; u < per; ++u) {
+          sc[u] = block_score(rows, n_rows, d, group_sum + (bh * Ng + m0 + u) * (long)d);
+          if (group_scores) group_scores[item * (long)kc * per + (long)r * per + u] = sc[u];
+        }
+        top_k(sc, per, kge, taken);
+        for (int u = 0; u < per; ++u)
+          if (taken[u]) gi[ng++] = m0 + u;
       }
-      top_k(sc, per, kge, taken);
-      for (int u = 0; u < per; ++u)
-        if (taken[u]) gi[ng++] = m0 + u;
+    } else {
+      /* item 2, global budget: the groups of all selected chunks compete for nsel * kg_eff places;
+       * slots are in ascending group order (chunks ascend), so "first wins ties" = lowest group id */
+      for (int r = 0; r < nsel; ++r)
+        for (int u = 0; u < per; ++u) {
+          sc[r * per + u] = block_score(rows, n_rows, d, group_sum + (bh * Ng + (long)ci[r] * per + u) * (long)d);
+          if (group_scores) group_scores[item * (long)kc * per + (long)r * per + u] = sc[r * per + u];
+        }
+      top_k(sc, nsel * per, nsel * kge, taken);
+      for (int i = 0; i < nsel * per; ++i)
+        if (taken[i]) gi[ng++] = ci[i / per] * per + i % per;
     }
     n_groups[item] = ng;
     free(rows); free(sc); free(taken);

@@ -34,6 +34,10 @@ typedef struct hga_ref_params {
   int32_t topk_chunks, topk_groups;    /* k_c, k_g (per opened chunk) */
   int32_t sink, local;                 /* tokens */
   double  softmax_scale;               /* <= 0 : 1/sqrt(d) */
+  int32_t global_group_budget;         /* 0: the k_g best groups inside EACH selected chunk;
+                                          1: the other reading of Section 2.1 item 2 ("the best groups
+                                          inside the chosen chunks"): the (selected chunks * kg_eff)
+                                          best groups over ALL selected chunks together */
 } hga_ref_params;
 
 /* Round a double to bf16, nearest-even, directly (single rounding). */

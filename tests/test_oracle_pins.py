@@ -190,6 +190,48 @@ def test_topk_brute_force_with_ties():
     assert saw_tie
 
 
+def test_global_group_budget_brute_force_with_ties():
+    """Section 2.1 item 2 read as one budget over all selected chunks: the selected groups are the
+    (chunks * kg_eff) best of every opened group, scores from the definition, ties to the lowest id
+    (planted by duplicating groups across chunks); chunk selection itself is unchanged."""
+    cfg = tiny(total_len=128, seg_len=32, topk_chunks=3, topk_groups=2)
+    x = make_inputs(cfg)
+    K = x["K"].copy()
+    c, g = cfg.chunk, cfg.group
+    per = c // g
+    for dst, src in ((4, 2), (9, 2), (7, 5)):            # duplicated chunks => tied groups across chunks
+        K[0, 0, dst * c:(dst + 1) * c] = K[0, 0, src * c:(src + 1) * c]
+    cs, gs = oracle.build_summaries(cfg, K)
+    base = oracle.route(cfg, x["Q"], cs, gs)
+    r = oracle.route(cfg, x["Q"], cs, gs, global_group_budget=True)
+    assert np.array_equal(r["chunk_idx"], base["chunk_idx"])
+    differs = saw_tie = False
+    for qb in range(cfg.n_q_blocks):
+        chunks = [j for j in r["chunk_idx"][0, 0, qb] if j >= 0]
+        ids = [j * per + u for j in chunks for u in range(per)]
+        sg = _scores_from_definition(cfg, x["Q"], gs, qb, ids)
+        n = len(chunks) * cfg.kg_eff
+        order = sorted(range(len(ids)), key=lambda i: (-sg[i], ids[i]))[:n]     # best scores, lowest id on ties
+        want = sorted(ids[i] for i in order)
+        got = [m for m in r["group_idx"][0, 0, qb] if m >= 0]
+        assert got == want, (qb, got, want)
+        assert r["n_groups"][0, 0, qb] == n and np.all(r["group_idx"][0, 0, qb, n:] == -1)
+        differs |= got != [m for m in base["group_idx"][0, 0, qb] if m >= 0]
+        kth = sg[order[-1]]
+        saw_tie |= sum(1 for v in sg if abs(v - kth) < 1e-12) > 1
+    assert differs and saw_tie          # the variant is not the per-chunk rule, and a tie decided a place
+
+
+def test_global_group_budget_equals_per_chunk_rule_when_chunks_open_whole():
+    cfg = tiny(total_len=256, seg_len=64, topk_chunks=3, topk_groups=8)     # kg_eff = c/g: every group of a chunk
+    x = make_inputs(cfg)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    a = oracle.route(cfg, x["Q"], cs, gs)
+    b = oracle.route(cfg, x["Q"], cs, gs, global_group_budget=True)
+    for k in ("chunk_idx", "group_idx", "n_groups"):
+        assert np.array_equal(a[k], b[k])
+
+
 def test_router_structure_and_permutation():
     cfg = tiny(n_q_heads=4, n_kv_heads=2, total_len=256, seg_len=64, topk_chunks=4)
     x = make_inputs(cfg)
