@@ -68,6 +68,10 @@ extern "C" {
 #define HGA_FLAG_BWD_ACCUMULATE 1  /* hga_attn_bwd adds into dK/dV instead of overwriting */
 #define HGA_FLAG_GENERIC_KERNELS 2 /* use the shape-generic CUDA-core kernels even where a
                                       tensor-core kernel exists (debugging / cross-checks) */
+#define HGA_FLAG_GLOBAL_GROUP_BUDGET 4 /* hga_route: Section 2.1 item 2 read as ONE budget over all
+                                          selected chunks: the (selected chunks * kg_eff) best groups of
+                                          all opened chunks together, instead of the kg_eff best inside
+                                          each chunk.  Needs k_c * (c/g) <= 4096. */
 
 /* bits OR-ed into *status_word by the attention kernels */
 #define HGA_STATUS_BAD_INDEX 1     /* a group_idx entry was out of range, inside the sink or

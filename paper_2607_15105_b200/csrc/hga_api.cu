@@ -44,6 +44,8 @@ static int resolve(const hga_params* p, Dims& dm) {
   if (p->sink < 0 || p->local < 0 || p->sink % p->chunk || p->local % p->chunk) return HGA_ERR_SHAPE;
   if (p->chunk / p->group > 64) return HGA_ERR_UNSUPPORTED;
   if (p->topk_chunks > 1024) return HGA_ERR_UNSUPPORTED;
+  if ((p->flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) && (int64_t)p->topk_chunks * (p->chunk / p->group) > 4096)
+    return HGA_ERR_UNSUPPORTED;
   dm.B = p->batch; dm.Hq = p->n_q_heads; dm.Hkv = p->n_kv_heads; dm.G = dm.Hq / dm.Hkv;
   dm.d = p->head_dim; dm.L = p->total_len; dm.S = p->seg_len; dm.H = dm.L - dm.S;
   dm.c = p->chunk; dm.g = p->group; dm.Bq = p->q_block;
@@ -78,8 +80,10 @@ static int resolve(const hga_params* p, Dims& dm) {
 int resolve_params(const hga_params* p, Dims& dm) { return resolve(p, dm); }
 
 size_t route_workspace_bytes(const Dims& dm) {
-  // chunk scores fp32 [items, Nc]
-  return (size_t)dm.B * dm.Hkv * dm.NQB * dm.Nc * sizeof(float) + 16;
+  // chunk scores fp32 [items, Nc]; with a global group budget also the group scores of the opened
+  // chunks, fp32 [items, k_c * (c/g)] (the generic router keeps them there until it selects)
+  const size_t per_item = (size_t)dm.Nc + ((dm.flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) ? (size_t)dm.kc * dm.per : 0);
+  return (size_t)dm.B * dm.Hkv * dm.NQB * per_item * sizeof(float) + 16;
 }
 
 size_t bwd_workspace_bytes(const Dims& dm) {

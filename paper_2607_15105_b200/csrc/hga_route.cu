@@ -3,7 +3,8 @@
 // Three kernels per call:
 //   k_chunk_scores   scores[item][j] = max over the item's G*Bq rows of q . chunk_sum[j]
 //   k_select_chunks  top-k_c of the candidate scores, ties to the lowest index
-//   k_route_groups   scores of the opened chunks' group summaries, top-kg_eff per chunk
+//   k_route_groups   scores of the opened chunks' group summaries, top-kg_eff per chunk (or, with
+//                    HGA_FLAG_GLOBAL_GROUP_BUDGET, the best chunks*kg_eff groups over all of them)
 // bf16 x bf16 products are exact in fp32; only the fp32 accumulation order differs from
 // an exact evaluation (about 1e-6 relative).
 #include <cfloat>
@@ -174,7 +175,8 @@ template <int D>
 __global__ void __launch_bounds__(kScoreThreads)
 k_route_groups(const uint16_t* __restrict__ Q, const uint16_t* __restrict__ group_sum, Dims dm,
                const int32_t* __restrict__ chunk_idx, int32_t* __restrict__ group_idx,
-               int32_t* __restrict__ n_groups, float* __restrict__ group_scores_out) {
+               int32_t* __restrict__ n_groups, float* __restrict__ group_scores_out,
+               float* __restrict__ gscratch /* [items][kc * per], global budget only */) {
   extern __shared__ float smem[];
   float* s_sum = smem;
   float* s_q = s_sum + kScoreTile * (D + 1);
@@ -182,6 +184,8 @@ k_route_groups(const uint16_t* __restrict__ Q, const uint16_t* __restrict__ grou
   float* s_out = s_red + kScoreThreads;
   int* s_rows = reinterpret_cast<int*>(s_out + kScoreTile);
   __shared__ int s_count;
+  __shared__ unsigned long long s_flags[64];          // global budget: bit i = slot i selected (<= 4096 slots)
+  const bool global_budget = (dm.flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) != 0;
   const int item = blockIdx.x;
   int b, h, qb;
   item_coords(dm, item, b, h, qb);
@@ -210,9 +214,13 @@ k_route_groups(const uint16_t* __restrict__ Q, const uint16_t* __restrict__ grou
     score_tile<D>(dm, Qitem, group_sum + (int64_t)bh * dm.NgS * D, s_rows, s_sum, s_q, s_red, s_out);
     if (group_scores_out && tid < chunks_per_tile * dm.per && base + tid < total)
       group_scores_out[(int64_t)item * dm.kc * dm.per + base + tid] = s_out[tid];
-    // one thread per opened chunk of this tile: top-kg_eff of its `per` groups.  Chunks are
-    // handled in ascending order by thread 0 so the output list is ascending.
-    if (tid == 0) {
+    if (global_budget) {
+      // keep the scores: the selection runs over all opened chunks at the end
+      if (tid < chunks_per_tile * dm.per && base + tid < total)
+        gscratch[(int64_t)item * dm.kc * dm.per + base + tid] = s_out[tid];
+    } else if (tid == 0) {
+      // one thread per opened chunk of this tile: top-kg_eff of its `per` groups.  Chunks are
+      // handled in ascending order by thread 0 so the output list is ascending.
       int n = s_count;
       for (int cc = 0; cc < chunks_per_tile && base + cc * dm.per < total; ++cc) {
         const float* v = s_out + cc * dm.per;
@@ -231,6 +239,30 @@ k_route_groups(const uint16_t* __restrict__ Q, const uint16_t* __restrict__ grou
     }
     __syncthreads();
   }
+  if (global_budget) {
+    // slot i (chunk-major = ascending group id) is selected when fewer than nsel * kg_eff slots beat
+    // it (higher score, or equal score and lower id); its output place is the number of selected
+    // slots below it
+    const float* v = gscratch + (int64_t)item * dm.kc * dm.per;
+    const int want = nsel * dm.kge;
+    if (tid < 64) s_flags[tid] = 0;
+    __syncthreads();                        // also orders the score writes above before the reads below
+    for (int i = tid; i < total; i += blockDim.x) {
+      const float mine = v[i];
+      int beat = 0;
+      for (int q = 0; q < total; ++q) beat += v[q] > mine || (v[q] == mine && q < i);
+      if (beat < want) atomicOr(&s_flags[i >> 6], 1ull << (i & 63));
+    }
+    __syncthreads();
+    for (int i = tid; i < total; i += blockDim.x)
+      if ((s_flags[i >> 6] >> (i & 63)) & 1ull) {
+        int pos = __popcll(s_flags[i >> 6] & ((1ull << (i & 63)) - 1));
+        for (int q = 0; q < (i >> 6); ++q) pos += __popcll(s_flags[q]);
+        gi[pos] = ci[i / dm.per] * dm.per + i % dm.per;
+      }
+    if (tid == 0) n_groups[item] = want;
+    return;
+  }
   if (tid == 0) n_groups[item] = s_count;
 }
 
@@ -245,6 +277,7 @@ int launch_route_generic(const Dims& dm, const void* Q, const void* chunk_sum,
                          void* workspace, cudaStream_t st) {
   const int items = dm.B * dm.Hkv * dm.NQB;
   float* scores = (float*)workspace;
+  float* gscratch = scores + (size_t)items * dm.Nc;      // behind the chunk scores (global group budget only)
   auto Qp = (const uint16_t*)Q;
   auto cs = (const uint16_t*)chunk_sum;
   auto gs = (const uint16_t*)group_sum;
@@ -278,9 +311,9 @@ int launch_route_generic(const Dims& dm, const void* Q, const void* chunk_sum,
   int rc = record_cuda(cudaGetLastError());
   if (rc) return rc;
   if (dm.d == 128)
-    k_route_groups<128><<<items, kScoreThreads, smem, st>>>(Qp, gs, dm, chunk_idx, group_idx, n_groups, group_scores);
+    k_route_groups<128><<<items, kScoreThreads, smem, st>>>(Qp, gs, dm, chunk_idx, group_idx, n_groups, group_scores, gscratch);
   else
-    k_route_groups<64><<<items, kScoreThreads, smem, st>>>(Qp, gs, dm, chunk_idx, group_idx, n_groups, group_scores);
+    k_route_groups<64><<<items, kScoreThreads, smem, st>>>(Qp, gs, dm, chunk_idx, group_idx, n_groups, group_scores, gscratch);
   count_launch();
   return record_cuda(cudaGetLastError());
 }

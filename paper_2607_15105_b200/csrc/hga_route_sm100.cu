@@ -276,6 +276,29 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   __syncthreads();
   if (!sm.abort) {
     int32_t* gi = group_idx + (int64_t)item * dm.width;
+    if (dm.flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) {
+      // One budget over all opened chunks: slot i (chunk-major, i.e. ascending group id) is selected
+      // when fewer than k_sel * kg_eff slots beat it (higher score, or equal score and lower id); its
+      // place in the ascending output is the number of selected slots below it.
+      const int total = k_sel * dm.per, want = k_sel * dm.kge;
+      unsigned long long* flags = reinterpret_cast<unsigned long long*>(sm.sel);   // 4096 bits
+      for (int i = tid; i < (total + 63) / 64; i += kRtThreads) flags[i] = 0;
+      __syncthreads();
+      for (int i = tid; i < total; i += kRtThreads) {
+        const float mine = gscore[i];
+        int beat = 0;
+        for (int q = 0; q < total; ++q) beat += gscore[q] > mine || (gscore[q] == mine && q < i);
+        if (beat < want) atomicOr(&flags[i >> 6], 1ull << (i & 63));
+        if (group_scores) group_scores[(int64_t)item * dm.kc * dm.per + i] = mine;
+      }
+      __syncthreads();
+      for (int i = tid; i < total; i += kRtThreads)
+        if ((flags[i >> 6] >> (i & 63)) & 1ull) {
+          int pos = __popcll(flags[i >> 6] & ((1ull << (i & 63)) - 1));
+          for (int q = 0; q < (i >> 6); ++q) pos += __popcll(flags[q]);
+          gi[pos] = sm.sorted[i / dm.per] * dm.per + i % dm.per;
+        }
+    } else
     for (int r = tid; r < dm.kc; r += kRtThreads) {
       if (r < k_sel) {
         const float* v = gscore + r * dm.per;
@@ -325,6 +348,7 @@ bool route_sm100_supported(const Dims& dm) {
   if (dm.rows > 256 && dm.rows % 256 != 0) return false;
   if (dm.per != 8 && dm.per != 16) return false;            // opened chunk = 1 or 2 octets of summaries
   if (dm.kc > 1024) return false;
+  if ((dm.flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) && dm.kc * dm.per > 4096) return false;   // bitmap in sel[]
   return route_sm100_smem(dm, route_max_cand(dm)) <= 227 * 1024;
 }
 

@@ -30,12 +30,14 @@ def rel_fro(a: np.ndarray, ref: np.ndarray) -> float:
     return num / den if den > 0 else num
 
 
-def check_routing(cfg, ref, chunk_idx, group_idx, n_groups, items=None):
+def check_routing(cfg, ref, chunk_idx, group_idx, n_groups, items=None, global_budget=False):
     """Compare GPU routing with the oracle's (ref holds oracle indices and fp64 scores).
 
     Index sets must be equal, except that an index in the symmetric difference is excused
     when its oracle score lies within SCORE_GAP of the oracle's k-th best score; set sizes
-    must match.  Groups are compared inside chunks both sides selected.
+    must match.  Groups are compared inside chunks both sides selected; with global_budget (one
+    budget over all opened chunks) the whole group sets are compared, against the oracle's
+    N-th best group score, for the items whose chunk sets agree.
     Returns (items checked, items with an excused chunk, chunks with an excused group).
     """
     per, kge = cfg.chunk // cfg.group, min(cfg.topk_groups, cfg.chunk // cfg.group)
@@ -62,6 +64,17 @@ def check_routing(cfg, ref, chunk_idx, group_idx, n_groups, items=None):
         assert ng == len(g_c) * kge, (item, ng)
         g_g = [int(m) for m in group_idx[b, h, qb, :ng]]
         assert g_g == sorted(set(g_g)) and np.all(group_idx[b, h, qb, ng:] == -1), (item, g_g)
+        if global_budget:
+            assert all(m // per in g_c for m in g_g), (item, g_g)
+            o_set = {int(m) for m in ref["group_idx"][b, h, qb] if m >= 0}
+            if set(o_c) == set(g_c) and o_set != set(g_g):
+                sg = ref["group_scores"][b, h, qb]
+                slot = lambda m: o_c.index(m // per) * per + m % per
+                nth = min(sg[slot(m)] for m in o_set)
+                for m in o_set ^ set(g_g):
+                    assert abs(sg[slot(m)] - nth) < SCORE_GAP, ("group not excused", item, m)
+                exc_g += 1
+            continue
         for r, j in enumerate(o_c):
             if j not in g_c:
                 continue
