@@ -34,7 +34,7 @@ class RefParams(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "batch", "n_q_heads", "n_kv_heads", "head_dim", "total_len", "seg_len", "chunk",
         "group", "q_block", "topk_chunks", "topk_groups", "sink", "local")] + [
-        ("softmax_scale", C.c_double), ("global_group_budget", C.c_int32)]
+        ("softmax_scale", C.c_double), ("global_group_budget", C.c_int32), ("score_agg", C.c_int32)]
 
 
 def lib():
@@ -48,11 +48,15 @@ def lib():
     return _lib
 
 
-def params(cfg, softmax_scale: float = 0.0, global_group_budget: bool = False) -> RefParams:
+SCORE_AGG = {"max": 0, "mean": 1, "lse": 2}
+
+
+def params(cfg, softmax_scale: float = 0.0, global_group_budget: bool = False, score_agg: str = "max") -> RefParams:
     """Build the oracle's parameter block from any object with the HGA shape fields."""
     return RefParams(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.total_len,
                      cfg.seg_len, cfg.chunk, cfg.group, cfg.q_block, cfg.topk_chunks,
-                     cfg.topk_groups, cfg.sink, cfg.local, softmax_scale, int(global_group_budget))
+                     cfg.topk_groups, cfg.sink, cfg.local, softmax_scale, int(global_group_budget),
+                     SCORE_AGG[score_agg])
 
 
 def _p(a, dtype):
@@ -113,7 +117,8 @@ def build_summaries(cfg, K, tok_begin=None, tok_end=None, chunk_sum=None, group_
     return chunk_sum, group_sum
 
 
-def route(cfg, Q, chunk_sum, group_sum, items=None, want_scores=False, global_group_budget=False):
+def route(cfg, Q, chunk_sum, group_sum, items=None, want_scores=False, global_group_budget=False,
+          score_agg="max"):
     B, Hkv, nqb = cfg.batch, cfg.n_kv_heads, cfg.seg_len // cfg.q_block
     kc, kge, per = cfg.topk_chunks, kg_eff(cfg), cfg.chunk // cfg.group
     chunk_idx = np.full((B, Hkv, nqb, kc), -1, np.int32)
@@ -124,7 +129,7 @@ def route(cfg, Q, chunk_sum, group_sum, items=None, want_scores=False, global_gr
         cs = np.full((B, Hkv, nqb, cfg.total_len // cfg.chunk), -np.inf, np.float64)
         gs = np.full((B, Hkv, nqb, kc * per), -np.inf, np.float64)
     keep, ip, n = _items(items)
-    _ok(lib().hga_ref_route(C.byref(params(cfg, 0.0, global_group_budget)), _p(Q, np.uint16), _p(chunk_sum, np.uint16),
+    _ok(lib().hga_ref_route(C.byref(params(cfg, 0.0, global_group_budget, score_agg)), _p(Q, np.uint16), _p(chunk_sum, np.uint16),
                             _p(group_sum, np.uint16), _p(chunk_idx, np.int32),
                             _p(group_idx, np.int32), _p(n_groups, np.int32), _p(cs, np.float64),
                             _p(gs, np.float64), ip, C.c_int32(n)), "route")

@@ -79,6 +79,7 @@ static int check(const hga_ref_params* p) {
   if (p->total_len % p->chunk) return ERR_ARG;
   if (p->topk_chunks < 0 || p->topk_groups < 1) return ERR_ARG;
   if (p->sink < 0 || p->local < 0 || p->sink % p->chunk || p->local % p->chunk) return ERR_ARG;
+  if (p->score_agg < 0 || p->score_agg > 2) return ERR_ARG;
   return 0;
 }
 
@@ -154,15 +155,29 @@ int hga_ref_build_summaries(const hga_ref_params* p, const uint16_t* K, int32_t 
   return 0;
 }
 
-/* max over the block's rows of (row . summary) */
-static double block_score(const double* rows, int n_rows, int d, const uint16_t* summary) {
+/* the block's score of one summary from its rows' dot products (row . summary):
+ * agg 0 maximum, 1 mean, 2 log-sum-exp */
+static double block_score(const double* rows, int n_rows, int d, const uint16_t* summary, int agg) {
+  double* s = (double*)malloc(sizeof(double) * (size_t)n_rows);
+  if (!s) return NAN;
   double best = -INFINITY;
   for (int r = 0; r < n_rows; ++r) {
-    double s = 0;
-    for (int e = 0; e < d; ++e) s += rows[(long)r * d + e] * hga_ref_bf16_to_f64(summary[e]);
-    if (s > best) best = s;
+    s[r] = 0;
+    for (int e = 0; e < d; ++e) s[r] += rows[(long)r * d + e] * hga_ref_bf16_to_f64(summary[e]);
+    if (s[r] > best) best = s[r];
   }
-  return best;
+  double out = best;
+  if (agg == 1) {
+    out = 0;
+    for (int r = 0; r < n_rows; ++r) out += s[r];
+    out /= (double)n_rows;
+  } else if (agg == 2) {
+    double z = 0;
+    for (int r = 0; r < n_rows; ++r) z += exp(s[r] - best);
+    out = best + log(z);
+  }
+  free(s);
+  return out;
 }
 
 /* choose the k best of ids[0..n) by (score descending, id ascending); mark them in taken[] */
@@ -221,7 +236,7 @@ int hga_ref_route(const hga_ref_params* p, const uint16_t* Q, const uint16_t* ch
       for (int i = 0; i < kc * per; ++i) group_scores[item * (long)kc * per + i] = -INFINITY;
     /* item 1: score every candidate chunk summary, keep the k_c best */
     for (int i = 0; i < n_cand; ++i) {
-      sc[i] = block_score(rows, n_rows, d, chunk_sum + (bh * Nc + j0 + i) * (long)d);
+      sc[i] = block_score(rows, n_rows, d, chunk_sum + (bh * Nc + j0 + i) * (long)d, p->score_agg);
       if (chunk_scores) chunk_scores[item * Nc + j0 + i] = sc[i];
     }
     top_k(sc, n_cand, kc, taken);
@@ -234,7 +249,7 @@ int hga_ref_route(const hga_ref_params* p, const uint16_t* Q, const uint16_t* ch
       for (int r = 0; r < nsel; ++r) {
         int m0 = ci[r] * per;
         for (int u = 0; u < per; ++u) {
-          sc[u] = block_score(rows, n_rows, d, group_sum + (bh * Ng + m0 + u) * (long)d);
+          sc[u] = block_score(rows, n_rows, d, group_sum + (bh * Ng + m0 + u) * (long)d, p->score_agg);
           if (group_scores) group_scores[item * (long)kc * per + (long)r * per + u] = sc[u];
         }
         top_k(sc, per, kge, taken);
@@ -246,7 +261,8 @@ int hga_ref_route(const hga_ref_params* p, const uint16_t* Q, const uint16_t* ch
        * slots are in ascending group order (chunks ascend), so "first wins ties" = lowest group id */
       for (int r = 0; r < nsel; ++r)
         for (int u = 0; u < per; ++u) {
-          sc[r * per + u] = block_score(rows, n_rows, d, group_sum + (bh * Ng + (long)ci[r] * per + u) * (long)d);
+          sc[r * per + u] = block_score(rows, n_rows, d, group_sum + (bh * Ng + (long)ci[r] * per + u) * (long)d,
+                                        p->score_agg);
           if (group_scores) group_scores[item * (long)kc * per + (long)r * per + u] = sc[r * per + u];
         }
       top_k(sc, nsel * per, nsel * kge, taken);

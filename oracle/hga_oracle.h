@@ -38,6 +38,12 @@ typedef struct hga_ref_params {
                                           1: the other reading of Section 2.1 item 2 ("the best groups
                                           inside the chosen chunks"): the (selected chunks * kg_eff)
                                           best groups over ALL selected chunks together */
+  int32_t score_agg;                   /* how the block's G*Bq per-row dot products with one summary become
+                                          the block's score of it (Section 2.1 item 1 says only that the
+                                          query block scores the summaries; Section 5 that scores come from
+                                          several query positions): 0 = maximum over the rows;
+                                          1 = mean over the rows (equal to the mean query row's dot
+                                          product); 2 = ln sum_rows exp(dot) */
 } hga_ref_params;
 
 /* Round a double to bf16, nearest-even, directly (single rounding). */

@@ -232,6 +232,65 @@ def test_global_group_budget_equals_per_chunk_rule_when_chunks_open_whole():
         assert np.array_equal(a[k], b[k])
 
 
+def _block_rows(cfg, Q, h, qb):
+    G, Bq = cfg.gqa, cfg.q_block
+    return bf16_bits_to_f64(Q[0, h * G:(h + 1) * G, qb * Bq:(qb + 1) * Bq]).reshape(G * Bq, -1)
+
+
+def test_score_aggregators_mean_and_lse():
+    """The other ways a query block can score a summary.  Mean over rows is pinned by linearity: it
+    equals ONE dot product with the mean query row (a different computation from the oracle's, which
+    averages per-row dot products).  Log-sum-exp is pinned against scipy's routine on a matrix
+    product, by max <= lse <= max + ln(rows), and by its limit: with the queries scaled by 2^7 the
+    exponentials are dominated by the best row, so it must route exactly like the maximum."""
+    from scipy.special import logsumexp
+    cfg = tiny(n_q_heads=4, n_kv_heads=2, total_len=256, seg_len=64, topk_chunks=4, topics=0)
+    x = make_inputs(cfg)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    r_max = oracle.route(cfg, x["Q"], cs, gs, want_scores=True)
+    r_mean = oracle.route(cfg, x["Q"], cs, gs, want_scores=True, score_agg="mean")
+    r_lse = oracle.route(cfg, x["Q"], cs, gs, want_scores=True, score_agg="lse")
+    c, per = cfg.chunk, cfg.chunk // cfg.group
+    n_rows = cfg.gqa * cfg.q_block
+    for h in range(2):
+        for qb in range(cfg.n_q_blocks):
+            ls, se = oracle.window(cfg, qb)
+            cand = list(range(se // c, ls // c))
+            if not cand:
+                continue
+            rows = _block_rows(cfg, x["Q"], h, qb)
+            summ = bf16_bits_to_f64(cs[0, h, cand])
+            want_mean = summ @ rows.mean(axis=0)
+            dots = rows @ summ.T
+            assert np.allclose(r_mean["chunk_scores"][0, h, qb, cand], want_mean, rtol=0, atol=1e-12)
+            assert np.allclose(r_lse["chunk_scores"][0, h, qb, cand], logsumexp(dots, axis=0), rtol=0, atol=1e-12)
+            mx = r_max["chunk_scores"][0, h, qb, cand]
+            lse = r_lse["chunk_scores"][0, h, qb, cand]
+            assert np.all(lse >= mx) and np.all(lse <= mx + np.log(n_rows) + 1e-12)
+            for r, want in ((r_mean, want_mean), (r_lse, logsumexp(dots, axis=0))):
+                k = min(cfg.topk_chunks, len(cand))
+                order = sorted(range(len(cand)), key=lambda i: (-want[i], cand[i]))[:k]
+                got = [j for j in r["chunk_idx"][0, h, qb] if j >= 0]
+                assert got == sorted(cand[i] for i in order)
+                # groups of the opened chunks, same aggregator
+                ng = 0
+                for rr, j in enumerate(got):
+                    ids = list(range(j * per, (j + 1) * per))
+                    gsum = bf16_bits_to_f64(gs[0, h, ids])
+                    sg = gsum @ rows.mean(axis=0) if r is r_mean else logsumexp(rows @ gsum.T, axis=0)
+                    assert np.allclose(r["group_scores"][0, h, qb, rr * per:(rr + 1) * per], sg, rtol=0, atol=1e-12)
+                    og = sorted(range(per), key=lambda i: (-sg[i], i))[:cfg.kg_eff]
+                    assert [m for m in r["group_idx"][0, h, qb, ng:ng + cfg.kg_eff]] == sorted(ids[i] for i in og)
+                    ng += cfg.kg_eff
+    assert not np.array_equal(r_mean["chunk_idx"], r_max["chunk_idx"])    # the aggregators do differ on this input
+    # limit: queries * 128 (exact in bf16: an exponent shift) => lse routes like max
+    Qbig = f32_to_bf16_bits((bf16_bits_to_f64(x["Q"]) * 128.0).astype(np.float32))
+    a = oracle.route(cfg, Qbig, cs, gs)
+    b = oracle.route(cfg, Qbig, cs, gs, score_agg="lse")
+    for k in ("chunk_idx", "group_idx", "n_groups"):
+        assert np.array_equal(a[k], b[k])
+
+
 def test_router_structure_and_permutation():
     cfg = tiny(n_q_heads=4, n_kv_heads=2, total_len=256, seg_len=64, topk_chunks=4)
     x = make_inputs(cfg)
