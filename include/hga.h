@@ -72,6 +72,11 @@ extern "C" {
                                           selected chunks: the (selected chunks * kg_eff) best groups of
                                           all opened chunks together, instead of the kg_eff best inside
                                           each chunk.  Needs k_c * (c/g) <= 4096. */
+#define HGA_FLAG_SCORE_MEAN 8  /* hga_route: a query block's score of a summary is the MEAN over its
+                                  G*Bq rows of the dot product (= the mean query row's dot product)
+                                  instead of the maximum (Section 2.1 item 1 leaves the reduction open) */
+#define HGA_FLAG_SCORE_LSE 16  /* hga_route: the score is ln sum_rows exp(dot product).  At most one of
+                                  SCORE_MEAN / SCORE_LSE may be set (else HGA_ERR_UNSUPPORTED). */
 
 /* bits OR-ed into *status_word by the attention kernels */
 #define HGA_STATUS_BAD_INDEX 1     /* a group_idx entry was out of range, inside the sink or

@@ -17,6 +17,8 @@ LIB_PATH = os.path.join(_HERE, "libhga.so")
 HGA_FLAG_BWD_ACCUMULATE = 1
 HGA_FLAG_GENERIC_KERNELS = 2
 HGA_FLAG_GLOBAL_GROUP_BUDGET = 4
+HGA_FLAG_SCORE_MEAN = 8
+HGA_FLAG_SCORE_LSE = 16
 HGA_STATUS_BAD_INDEX = 1
 HGA_STATUS_WAIT_TIMEOUT = 2
 

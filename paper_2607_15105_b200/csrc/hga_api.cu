@@ -44,6 +44,7 @@ static int resolve(const hga_params* p, Dims& dm) {
   if (p->sink < 0 || p->local < 0 || p->sink % p->chunk || p->local % p->chunk) return HGA_ERR_SHAPE;
   if (p->chunk / p->group > 64) return HGA_ERR_UNSUPPORTED;
   if (p->topk_chunks > 1024) return HGA_ERR_UNSUPPORTED;
+  if ((p->flags & HGA_FLAG_SCORE_MEAN) && (p->flags & HGA_FLAG_SCORE_LSE)) return HGA_ERR_UNSUPPORTED;
   if ((p->flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) && (int64_t)p->topk_chunks * (p->chunk / p->group) > 4096)
     return HGA_ERR_UNSUPPORTED;
   dm.B = p->batch; dm.Hq = p->n_q_heads; dm.Hkv = p->n_kv_heads; dm.G = dm.Hq / dm.Hkv;

@@ -9,6 +9,11 @@
 
 namespace hga {
 
+// Block score aggregator selected by hga_params.flags: 0 maximum, 1 mean, 2 log-sum-exp over the rows.
+__host__ __device__ inline int score_agg_of(int flags) {
+  return (flags & HGA_FLAG_SCORE_MEAN) ? 1 : (flags & HGA_FLAG_SCORE_LSE) ? 2 : 0;
+}
+
 // Resolved problem description handed to kernels by value.
 struct Dims {
   int B, Hq, Hkv, G, d;

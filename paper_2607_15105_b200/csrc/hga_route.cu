@@ -1,7 +1,8 @@
 // hga_route, shape-generic CUDA-core version (Section 2.1, items 1-2).
 //
 // Three kernels per call:
-//   k_chunk_scores   scores[item][j] = max over the item's G*Bq rows of q . chunk_sum[j]
+//   k_chunk_scores   scores[item][j] = max (or mean, or log-sum-exp: HGA_FLAG_SCORE_*) over the item's
+//                    G*Bq rows of q . chunk_sum[j]
 //   k_select_chunks  top-k_c of the candidate scores, ties to the lowest index
 //   k_route_groups   scores of the opened chunks' group summaries, top-kg_eff per chunk (or, with
 //                    HGA_FLAG_GLOBAL_GROUP_BUDGET, the best chunks*kg_eff groups over all of them)
@@ -39,7 +40,8 @@ __device__ void score_tile(const Dims& dm, const uint16_t* __restrict__ Qitem,
     s_sum[r * (D + 1) + 2 * e2 + 1] = bf16_hi(w);
   }
   const int jj = tid % kScoreTile, part = tid / kScoreTile;
-  float best = -FLT_MAX;
+  const int agg = score_agg_of(dm.flags);
+  float best = -FLT_MAX, sum = 0.f;       // log-sum-exp keeps (running maximum, sum of exp(dot - maximum))
   for (int r0 = 0; r0 < dm.rows; r0 += kRowTile) {
     __syncthreads();
     for (int i = tid; i < kRowTile * (D / 2); i += kScoreThreads) {
@@ -59,15 +61,38 @@ __device__ void score_tile(const Dims& dm, const uint16_t* __restrict__ Qitem,
       float acc = 0.f;
 #pragma unroll 16
       for (int e = 0; e < D; ++e) acc = fmaf(qv[e], sv[e], acc);
-      best = fmaxf(best, acc);
+      if (agg == 0) {
+        best = fmaxf(best, acc);
+      } else if (agg == 1) {
+        sum += acc;
+      } else {
+        if (acc > best) { sum *= expf(best - acc); best = acc; }
+        sum += expf(acc - best);
+      }
     }
   }
-  s_red[part * kScoreTile + jj] = best;
+  constexpr int kParts = kScoreThreads / kScoreTile;
+  s_red[part * kScoreTile + jj] = agg == 1 ? sum : best;
   __syncthreads();
+  float m = 0.f;
   if (tid < kScoreTile) {
-    float m = s_red[tid];
-    for (int q = 1; q < kScoreThreads / kScoreTile; ++q) m = fmaxf(m, s_red[q * kScoreTile + tid]);
-    out[tid] = m;
+    m = s_red[tid];
+    for (int q = 1; q < kParts; ++q) m = agg == 1 ? m + s_red[q * kScoreTile + tid] : fmaxf(m, s_red[q * kScoreTile + tid]);
+    if (agg == 1) m *= 1.f / (float)dm.rows;
+    if (agg != 2) out[tid] = m;
+  }
+  if (agg == 2) {
+    // second round: every part's sum rescaled to the common maximum
+    const float mj = fmaxf(fmaxf(s_red[jj], s_red[kScoreTile + jj]), fmaxf(s_red[2 * kScoreTile + jj], s_red[3 * kScoreTile + jj]));
+    static_assert(kParts == 4, "four row parts per summary");
+    __syncthreads();
+    s_red[part * kScoreTile + jj] = sum * expf(best - mj);
+    __syncthreads();
+    if (tid < kScoreTile) {
+      float s = 0.f;
+      for (int q = 0; q < kParts; ++q) s += s_red[q * kScoreTile + tid];
+      out[tid] = m + logf(s);
+    }
   }
   __syncthreads();
 }

@@ -1,7 +1,7 @@
 // hga_route for sm_100a: chunk selection and group selection (Section 2.1 items 1-2) as one
 // fused tcgen05 kernel per item (b, kv head, query block).
 //
-// Scores are max over the item's G*Bq query rows of q . summary.  The GEMM puts 128 summaries
+// Scores are the max (or mean / log-sum-exp, HGA_FLAG_SCORE_*) over the item's G*Bq query rows of q . summary.  The GEMM puts 128 summaries
 // on the MMA M dimension (= TMEM lanes) and up to 256 query rows on N (= TMEM columns), so the
 // maximum over rows is an in-thread reduction over the columns a thread reads back with
 // tcgen05.ld: thread = summary.
@@ -83,6 +83,8 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   const int n_ct = (n_cand + 127) / 128;                     // chunk tiles
   const int n_gt = (k_sel * dm.per + 127) / 128;             // group tiles
   volatile int* abort = &sm.abort;
+  const int agg = score_agg_of(dm.flags);
+  constexpr float kLog2e = 1.4426950408889634f;
 
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
@@ -172,7 +174,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       bool ok = true;
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int tg = t_begin + t;
-        float best = -FLT_MAX;
+        float best = -FLT_MAX, sum = 0.f;    // log-sum-exp: (running maximum, sum of exp(dot - maximum))
         for (int hf = 0; hf < n_halves; ++hf) {
           const int step = tg * n_halves + hf, buf = step % kRtAccs;
           ok = __all_sync(0xffffffffu, rt_wait(&sm.acc_full[buf], (step / kRtAccs) & 1, abort));
@@ -182,13 +184,27 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             uint32_t x[32];
             tmem_ld32(lane_base + buf * 256 + c, x);
             tmem_wait_ld();
+            if (agg == 0) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) best = fmaxf(best, __uint_as_float(x[i]));
+              for (int i = 0; i < 32; ++i) best = fmaxf(best, __uint_as_float(x[i]));
+            } else if (agg == 1) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) sum += __uint_as_float(x[i]);
+            } else {
+              float cm = -FLT_MAX;
+#pragma unroll
+              for (int i = 0; i < 32; ++i) cm = fmaxf(cm, __uint_as_float(x[i]));
+              if (cm > best) { sum *= exp2f((best - cm) * kLog2e); best = cm; }
+#pragma unroll
+              for (int i = 0; i < 32; ++i) sum += exp2f((__uint_as_float(x[i]) - best) * kLog2e);
+            }
           }
           tc_fence_before_sync();
           mbar_arrive(&sm.acc_free[buf]);
         }
         if (!ok) break;
+        if (agg == 1) best = sum * (1.f / (float)dm.rows);
+        else if (agg == 2) best += logf(sum);
         const int i = 128 * t + row;
         if (!phase2) {
           if (i < n_cand) keys[i] = ((unsigned long long)rt_orderable(best) << 32) | (uint32_t)(0x7fffffff - (j0 + i));
