@@ -34,7 +34,7 @@ class RefParams(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "batch", "n_q_heads", "n_kv_heads", "head_dim", "total_len", "seg_len", "chunk",
         "group", "q_block", "topk_chunks", "topk_groups", "sink", "local")] + [
-        ("softmax_scale", C.c_double), ("global_group_budget", C.c_int32), ("score_agg", C.c_int32)]
+        ("softmax_scale", C.c_double), ("global_group_budget", C.c_int32), ("score_agg", C.c_int32), ("decode", C.c_int32)]
 
 
 def lib():
@@ -56,7 +56,7 @@ def params(cfg, softmax_scale: float = 0.0, global_group_budget: bool = False, s
     return RefParams(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.total_len,
                      cfg.seg_len, cfg.chunk, cfg.group, cfg.q_block, cfg.topk_chunks,
                      cfg.topk_groups, cfg.sink, cfg.local, softmax_scale, int(global_group_budget),
-                     SCORE_AGG[score_agg])
+                     SCORE_AGG[score_agg], int(bool(getattr(cfg, "decode", False))))
 
 
 def _p(a, dtype):
@@ -110,7 +110,7 @@ def build_summaries(cfg, K, tok_begin=None, tok_end=None, chunk_sum=None, group_
     if group_sum is None:
         group_sum = np.zeros((B, Hkv, L // cfg.group, d), np.uint16)
     tb = 0 if tok_begin is None else tok_begin
-    te = L if tok_end is None else tok_end
+    te = (L // cfg.chunk) * cfg.chunk if tok_end is None else tok_end
     _ok(lib().hga_ref_build_summaries(C.byref(params(cfg)), _p(K, np.uint16), C.c_int32(tb),
                                       C.c_int32(te), _p(chunk_sum, np.uint16),
                                       _p(group_sum, np.uint16)), "build_summaries")

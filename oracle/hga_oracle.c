@@ -74,9 +74,12 @@ static int check(const hga_ref_params* p) {
   if (p->n_q_heads % p->n_kv_heads) return ERR_ARG;
   if (p->seg_len < 1 || p->total_len < p->seg_len) return ERR_ARG;
   if (p->group < 1 || p->chunk < p->group || p->chunk % p->group) return ERR_ARG;
-  if (p->q_block < p->chunk || p->q_block % p->chunk) return ERR_ARG;
-  if (p->seg_len % p->q_block || (p->total_len - p->seg_len) % p->q_block) return ERR_ARG;
-  if (p->total_len % p->chunk) return ERR_ARG;
+  if (p->q_block < 1 || p->seg_len % p->q_block) return ERR_ARG;
+  if (!p->decode) {
+    if (p->q_block < p->chunk || p->q_block % p->chunk) return ERR_ARG;
+    if ((p->total_len - p->seg_len) % p->q_block) return ERR_ARG;
+    if (p->total_len % p->chunk) return ERR_ARG;
+  }
   if (p->topk_chunks < 0 || p->topk_groups < 1) return ERR_ARG;
   if (p->sink < 0 || p->local < 0 || p->sink % p->chunk || p->local % p->chunk) return ERR_ARG;
   if (p->score_agg < 0 || p->score_agg > 2) return ERR_ARG;

@@ -44,6 +44,14 @@ typedef struct hga_ref_params {
                                           several query positions): 0 = maximum over the rows;
                                           1 = mean over the rows (equal to the mean query row's dot
                                           product); 2 = ln sum_rows exp(dot) */
+  int32_t decode;                      /* generation-shaped use (Sections 1 and 5: the same routed attention
+                                          serves retrieval and generation): the query block is the few
+                                          newest tokens.  Lifts the rules q_block % chunk == 0,
+                                          history % q_block == 0 and total_len % chunk == 0 (q_block >= 1,
+                                          any history); nothing else changes: same windows, same
+                                          candidates (closed chunks wholly before the local window),
+                                          same selection, same attention.  Summary arrays then hold
+                                          floor(L/c) and floor(L/g) rows. */
 } hga_ref_params;
 
 /* Round a double to bf16, nearest-even, directly (single rounding). */

@@ -44,6 +44,7 @@ class HgaConfig:
     needles: int        # planted key-group / query-block matches
     backward: bool
     seed: int
+    decode: bool = False   # generation-shaped: q_block = the few newest tokens, any history length
 
     @property
     def history(self) -> int:
@@ -127,7 +128,7 @@ def make_inputs(cfg: HgaConfig, with_dO: bool | None = None) -> dict:
         with_dO = cfg.backward
     B, Hq, Hkv, d = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
     L, S, c, g, Bq = cfg.total_len, cfg.seg_len, cfg.chunk, cfg.group, cfg.q_block
-    G, H, nqb, nch = cfg.gqa, cfg.history, cfg.n_q_blocks, cfg.total_len // cfg.chunk
+    G, H, nqb, nch = cfg.gqa, cfg.history, cfg.n_q_blocks, -(-cfg.total_len // cfg.chunk)
     Q = np.empty((B, Hq, S, d), np.uint16)
     K = np.empty((B, Hkv, L, d), np.uint16)
     V = np.empty((B, Hkv, L, d), np.uint16)
@@ -143,7 +144,7 @@ def make_inputs(cfg: HgaConfig, with_dO: bool | None = None) -> dict:
                 U = rng.standard_normal((cfg.topics, d)).astype(np.float32)
                 U /= np.linalg.norm(U, axis=1, keepdims=True)
                 tau = rng.integers(0, cfg.topics, nch)
-                k += _KEY_TOPIC_GAIN * np.repeat(U[tau], c, axis=0)
+                k += _KEY_TOPIC_GAIN * np.repeat(U[tau], c, axis=0)[:L]
                 for qb in range(nqb):
                     # a block follows the topics of two earlier chunks (of two random
                     # topics when nothing precedes it)

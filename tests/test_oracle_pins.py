@@ -377,6 +377,82 @@ def test_routed_attention_equals_masked_dense_restatement(hist):
         assert np.max(np.abs(lse - LSE[0, hq])) < 1e-12
 
 
+def _decode_cfg(hist, n, **kw):
+    return tiny(n_q_heads=4, n_kv_heads=2, total_len=hist + n, seg_len=n, q_block=n, decode=True, **kw)
+
+
+@pytest.mark.parametrize("hist,n", [(77, 1), (83, 5), (3, 2), (130, 16), (64, 8)])
+def test_decode_shape_routing_and_attention_from_the_definitions(hist, n):
+    """Generation-shaped use: the query block is the n newest tokens behind an arbitrary history.
+    Candidates, scores and selection are recomputed from their definitions, attention against the
+    separately written masked-dense restatement (whose mask is built per query position)."""
+    cfg = _decode_cfg(hist, n)
+    x = make_inputs(cfg)
+    c, g, per = cfg.chunk, cfg.group, cfg.chunk // cfg.group
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    assert cs.shape[2] == cfg.total_len // c and gs.shape[2] == cfg.total_len // g
+    r = oracle.route(cfg, x["Q"], cs, gs, want_scores=True)
+    local_start = max(0, ((hist - cfg.local) // c) * c)
+    sink_end = min(cfg.sink, local_start)
+    assert oracle.window(cfg, 0) == (local_start, sink_end)
+    cand = list(range(sink_end // c, local_start // c))
+    G = cfg.gqa
+    for h in range(cfg.n_kv_heads):
+        rows = bf16_bits_to_f64(x["Q"][0, h * G:(h + 1) * G]).reshape(G * n, -1)
+        sc = np.array([max(float(np.dot(q, bf16_bits_to_f64(cs[0, h, j]))) for q in rows) for j in cand])
+        k = min(cfg.topk_chunks, len(cand))
+        want = sorted(cand[i] for i in sorted(range(len(cand)), key=lambda i: (-sc[i], cand[i]))[:k])
+        got = [int(j) for j in r["chunk_idx"][0, h, 0] if j >= 0]
+        assert got == want
+        want_g = []
+        for j in got:
+            sg = [max(float(np.dot(q, bf16_bits_to_f64(gs[0, h, j * per + u]))) for q in rows) for u in range(per)]
+            want_g += sorted(j * per + u for u in sorted(range(per), key=lambda u: (-sg[u], u))[:cfg.kg_eff])
+        assert [int(m) for m in r["group_idx"][0, h, 0] if m >= 0] == want_g
+        assert r["n_groups"][0, h, 0] == len(want_g)
+    O, LSE = oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], r["group_idx"], r["n_groups"])
+    scale = 1.0 / np.sqrt(cfg.head_dim)
+    for hq in range(cfg.n_q_heads):
+        h = hq // G
+        mask = _mask_from_definition(cfg, h, r["group_idx"], r["n_groups"])
+        assert mask[:, hist:].sum() == n * (n + 1) // 2                  # causal among the new tokens
+        o, lse = _masked_attention_numpy(bf16_bits_to_f64(x["Q"][0, hq]), bf16_bits_to_f64(x["K"][0, h]),
+                                         bf16_bits_to_f64(x["V"][0, h]), mask, scale)
+        assert np.max(np.abs(o - O[0, hq])) < 1e-12
+        assert np.max(np.abs(lse - LSE[0, hq])) < 1e-12
+
+
+def test_decode_of_one_token_equals_its_row_in_block_mode():
+    """A token at position p has the same windows whether it is scored alone (generation) or as a row
+    of its c-aligned query block (training): floor((p - W)/c) = floor((floor(p/c)c - W)/c) when W is a
+    multiple of c.  Given the same group list, both must return the same O and LSE for it."""
+    c = 8
+    full = tiny(n_q_heads=4, n_kv_heads=2, total_len=128, seg_len=64)       # block mode: Bq = c = 8
+    x = make_inputs(full)
+    cs, gs = oracle.build_summaries(full, x["K"])
+    r = oracle.route(full, x["Q"], cs, gs)
+    O, LSE = oracle.attn_fwd(full, x["Q"], x["K"], x["V"], r["group_idx"], r["n_groups"])
+    for p in (64, 69, 71, 100, 127):
+        t = p - full.history
+        dec = _decode_cfg(p, 1)
+        Qd = np.ascontiguousarray(x["Q"][:, :, t:t + 1])
+        Kd, Vd = np.ascontiguousarray(x["K"][:, :, :p + 1]), np.ascontiguousarray(x["V"][:, :, :p + 1])
+        gi = np.ascontiguousarray(r["group_idx"][:, :, t // c:t // c + 1])
+        ng = np.ascontiguousarray(r["n_groups"][:, :, t // c:t // c + 1])
+        assert oracle.window(dec, 0) == oracle.window(full, t // c)
+        Od, LSEd = oracle.attn_fwd(dec, Qd, Kd, Vd, gi, ng)
+        assert np.max(np.abs(Od[:, :, 0] - O[:, :, t])) < 1e-13
+        assert np.max(np.abs(LSEd[:, :, 0] - LSE[:, :, t])) < 1e-13
+
+
+def test_decode_flag_is_what_lifts_the_shape_rules():
+    cfg = _decode_cfg(77, 1)
+    x = make_inputs(cfg)
+    from dataclasses import replace
+    with pytest.raises(RuntimeError):
+        oracle.window(replace(cfg, decode=False), 0)
+
+
 def _torch_attention_grads(cfg, x, mask_fn):
     """Library special case: torch SDPA in fp64 with autograd (boolean mask or causal)."""
     G, H = cfg.gqa, cfg.history
