@@ -77,6 +77,16 @@ extern "C" {
                                   instead of the maximum (Section 2.1 item 1 leaves the reduction open) */
 #define HGA_FLAG_SCORE_LSE 16  /* hga_route: the score is ln sum_rows exp(dot product).  At most one of
                                   SCORE_MEAN / SCORE_LSE may be set (else HGA_ERR_UNSUPPORTED). */
+#define HGA_FLAG_DECODE 32     /* generation-shaped use (Sections 1 and 5 name generation as a use of the
+                                  same routed attention): the query block is the few newest tokens
+                                  behind a history of any length.  Lifts the rules Bq % c == 0,
+                                  (L - S) % Bq == 0 and L % c == 0 (Bq >= 1, S % Bq == 0 stay); windows,
+                                  candidates (closed chunks wholly before the local window), selection
+                                  and attention are unchanged.  Summary buffers then hold
+                                  floor(L/c) / floor(L/g) rows (or summary_len/c, summary_len/g), and
+                                  hga_build_summaries still takes chunk-aligned ranges: call it when a
+                                  chunk closes.  Forward only: hga_attn_bwd, hga_step_host and
+                                  hga_tbptt_walk return HGA_ERR_UNSUPPORTED with this flag. */
 
 /* bits OR-ed into *status_word by the attention kernels */
 #define HGA_STATUS_BAD_INDEX 1     /* a group_idx entry was out of range, inside the sink or
@@ -87,7 +97,8 @@ typedef struct hga_params {
   int32_t batch, n_q_heads, n_kv_heads, head_dim; /* Hq % Hkv == 0; head_dim in {64, 128}      */
   int32_t total_len, seg_len;                      /* L >= S >= 1                                */
   int32_t chunk, group, q_block;                   /* c % g == 0; Bq % c == 0; S % Bq == 0;
-                                                      (L - S) % Bq == 0; L % c == 0            */
+                                                      (L - S) % Bq == 0; L % c == 0 (but see
+                                                      HGA_FLAG_DECODE)                         */
   int32_t topk_chunks, topk_groups;                /* k_c >= 0; k_g >= 1 (per opened chunk)      */
   int32_t sink, local;                             /* tokens, multiples of c                     */
   float   softmax_scale;                           /* <= 0 selects 1/sqrt(head_dim)              */

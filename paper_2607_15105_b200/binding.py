@@ -19,6 +19,7 @@ HGA_FLAG_GENERIC_KERNELS = 2
 HGA_FLAG_GLOBAL_GROUP_BUDGET = 4
 HGA_FLAG_SCORE_MEAN = 8
 HGA_FLAG_SCORE_LSE = 16
+HGA_FLAG_DECODE = 32
 HGA_STATUS_BAD_INDEX = 1
 HGA_STATUS_WAIT_TIMEOUT = 2
 
@@ -79,6 +80,8 @@ def lib():
 def make_params(cfg, softmax_scale: float = 0.0, flags: int = 0, q_stride=None, k_stride=None,
                 v_stride=None, o_stride=None, summary_len: int = 0) -> HgaParams:
     """hga_params from any object with the HGA shape fields (e.g. workloads.HgaConfig)."""
+    if getattr(cfg, "decode", False):
+        flags |= HGA_FLAG_DECODE
     p = HgaParams(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.total_len,
                   cfg.seg_len, cfg.chunk, cfg.group, cfg.q_block, cfg.topk_chunks,
                   cfg.topk_groups, cfg.sink, cfg.local, softmax_scale, flags, summary_len)

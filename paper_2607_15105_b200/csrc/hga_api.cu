@@ -37,9 +37,12 @@ static int resolve(const hga_params* p, Dims& dm) {
   if (p->head_dim != 64 && p->head_dim != 128) return HGA_ERR_UNSUPPORTED;
   if (p->seg_len < 1 || p->total_len < p->seg_len) return HGA_ERR_SHAPE;
   if (p->group < 1 || p->chunk < p->group || p->chunk % p->group) return HGA_ERR_SHAPE;
-  if (p->q_block < p->chunk || p->q_block % p->chunk) return HGA_ERR_SHAPE;
-  if (p->seg_len % p->q_block || (p->total_len - p->seg_len) % p->q_block) return HGA_ERR_SHAPE;
-  if (p->total_len % p->chunk) return HGA_ERR_SHAPE;
+  if (p->q_block < 1 || p->seg_len % p->q_block) return HGA_ERR_SHAPE;
+  if (!(p->flags & HGA_FLAG_DECODE)) {
+    if (p->q_block < p->chunk || p->q_block % p->chunk) return HGA_ERR_SHAPE;
+    if ((p->total_len - p->seg_len) % p->q_block) return HGA_ERR_SHAPE;
+    if (p->total_len % p->chunk) return HGA_ERR_SHAPE;
+  }
   if (p->topk_chunks < 0 || p->topk_groups < 1) return HGA_ERR_SHAPE;
   if (p->sink < 0 || p->local < 0 || p->sink % p->chunk || p->local % p->chunk) return HGA_ERR_SHAPE;
   if (p->chunk / p->group > 64) return HGA_ERR_UNSUPPORTED;
@@ -218,6 +221,7 @@ int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* 
   Dims dm;
   int rc = resolve(p, dm);
   if (rc) return rc;
+  if (dm.flags & HGA_FLAG_DECODE) return HGA_ERR_UNSUPPORTED;     // forward only
   if (!Q || !K || !V || !O || !LSE || !dO || (!group_idx && dm.width > 0) || !n_groups || !dQ || !dK || !dV)
     return HGA_ERR_NULL;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) ||
@@ -269,6 +273,7 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   Dims dm;
   int rc = resolve(p, dm);
   if (rc) return rc;
+  if (dm.flags & HGA_FLAG_DECODE) return HGA_ERR_UNSUPPORTED;
   if (!Q_host || !Kseg_host || !Vseg_host || !K_dev || !V_dev || !chunk_sum || !group_sum ||
       !O_host || !arena)
     return HGA_ERR_NULL;
@@ -371,6 +376,7 @@ int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void
                    int32_t* n_groups, void* O, float* LSE, void* dQ, float* dK, float* dV,
                    void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream) {
   if (!p) return HGA_ERR_NULL;
+  if (p->flags & HGA_FLAG_DECODE) return HGA_ERR_UNSUPPORTED;
   if (p->seg_len < 1 || p->total_len < p->seg_len || p->total_len % p->seg_len) return HGA_ERR_SHAPE;
   hga_params full = *p;                 // the last segment's problem: validates shapes, resolves the full-length strides
   full.summary_len = 0;

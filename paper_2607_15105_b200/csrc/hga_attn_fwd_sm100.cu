@@ -61,12 +61,7 @@ struct FwdSmem {
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort) {
-  for (uint32_t i = 0; i < (1u << 20); ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && *abort) return false;
-  }
-  *abort = 1;
-  return false;
+  return mbar_wait_bounded(bar, parity, abort);
 }
 
 template <int D>
@@ -86,7 +81,10 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   HGA_TRACE_DECL;
-  const int n_mt_item = dm.rows / 128;
+  // rows of the item: every head's Bq rows padded to whole octets (padding rows compute garbage
+  // in their own TMEM lanes and are never stored)
+  const int bq_pad = bq_padded(dm), rows_pad = rows_padded(dm);
+  const int n_mt_item = (rows_pad + 127) / 128;
   const int item = blockIdx.x / n_mt_item;
   const int mt0 = blockIdx.x % n_mt_item;               // this CTA's M-tile inside the item
   int b, h, qb;
@@ -113,12 +111,13 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // Q does not depend on the routing: start its copy first (tid 0 initialised the barriers above)
     if (lane == 0) {
       prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
-      mbar_arrive_expect_tx(&sm.q_full, (uint32_t)kQBytes);
     }
+    const int q_oct = min(16, rows_pad / 8 - 16 * mt0);   // octets of real rows in this M-tile
+    if (lane == 0) mbar_arrive_expect_tx(&sm.q_full, (uint32_t)q_oct * kOctBytes);
     __syncwarp();
-    if (lane < 16) {
+    if (lane < q_oct) {
       const int r = mt0 * 128 + 8 * lane;              // first row of the octet inside the item
-      const int a = r / dm.Bq, t = r % dm.Bq;
+      const int a = r / bq_pad, t = r % bq_pad;        // token rows past the segment arrive as zeros
       tma_load_5d(sm.q + lane * kOctBytes, &map_q, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
     }
     bool bad;
@@ -135,7 +134,8 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   const uint32_t tmem = sm.tmem_base;
   const int n_oct = sm.n_oct;
-  const int n_keys = n_oct * 8;
+  // exact key count: only the last octet of the local window can be partial
+  const int n_keys = n_oct * 8 - ((8 - ((w.p0 + dm.Bq - w.ls) & 7)) & 7);
   const int n_tiles = (n_oct + 7) / 8;
   volatile int* abort = &sm.abort;
   HGA_TRACE_POINT(1);
@@ -236,7 +236,8 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const int quarter = warp & 3;                       // TMEM lanes this warp may touch
       const int row_in_tile = quarter * 32 + lane;
       const int r = mt0 * 128 + row_in_tile;              // row inside the item
-      const int a = r / dm.Bq, t = r % dm.Bq;
+      const int a = r / bq_pad, t = r % bq_pad;
+      const bool real_row = r < rows_pad && t < dm.Bq;
       const int limit = n_keys - dm.Bq + t + 1;           // visible key slots (causal inside the block)
       const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
       const uint32_t o_addr = lane_base + kColO;
@@ -270,7 +271,7 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const float mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])) * sl2;
         HGA_TRACE_POINT(12);
         float corr = 1.f;
-        bool raise = mx > m_used + kRescaleThreshold;     // also true for the first visible tile
+        bool raise = real_row && mx > m_used + kRescaleThreshold;   // also true for the first visible tile
         if (raise) {
           corr = fast_exp2(m_used - mx);                  // 0 when m_used is -inf
           m_used = mx;
@@ -342,6 +343,7 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(&sm.o_done, 0, abort));
       HGA_TRACE_POINT(20);
       if (ok) {
+        // every lane takes part in the TMEM loads (warp-wide instructions); only real rows are stored
         tc_fence_after_sync();
         const float inv = 1.f / l_mma;
         const int hq = h * dm.G + a, srow = qb * dm.Bq + t;
@@ -362,11 +364,13 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               pk[i] = *reinterpret_cast<const uint32_t*>(&hh);
             }
             uint4* dst = reinterpret_cast<uint4*>(orow + c2 * 64 + c * 32);
+            if (real_row) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+              for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+            }
           }
         }
-        LSE[((int64_t)b * dm.Hq + hq) * dm.S + srow] = (m_used + log2f(l)) * 0.6931471805599453f;
+        if (real_row) LSE[((int64_t)b * dm.Hq + hq) * dm.S + srow] = (m_used + log2f(l)) * 0.6931471805599453f;
         HGA_TRACE_POINT(21);
       }
     }
@@ -388,7 +392,9 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
 bool attn_fwd_sm100_supported(const Dims& dm) {
   if (dm.flags & HGA_FLAG_GENERIC_KERNELS) return false;
-  if (dm.rows % 128 != 0) return false;
+  const int rows_pad = rows_padded(dm);
+  if (rows_pad > 128 && (rows_pad % 128 != 0 || rows_pad != dm.rows)) return false;
+  if (rows_pad < 128 && !(dm.flags & HGA_FLAG_DECODE)) return false;   // small training shapes stay on the generic kernel
   if (dm.g % 8 != 0) return false;
   return true;
 }
@@ -416,7 +422,7 @@ static int launch_fwd(const Dims& dm, const void* Q, const void* K, const void* 
     e = cudaFuncSetAttribute(k_attn_fwd_sm100<D>, cudaFuncAttributePreferredSharedMemoryCarveout,
                              (int)cudaSharedmemCarveoutMaxShared);
   if (e != cudaSuccess) return record_cuda(e);
-  const int units = dm.B * dm.Hkv * dm.NQB * (dm.rows / 128);
+  const int units = dm.B * dm.Hkv * dm.NQB * ((rows_padded(dm) + 127) / 128);
   k_attn_fwd_sm100<D><<<units, kFwdThreads, smem, st>>>(mq, mk, mv, group_idx, n_groups, dm, (uint16_t*)O, LSE,
                                                        status_word);
   count_launch();

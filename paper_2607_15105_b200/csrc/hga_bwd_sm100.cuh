@@ -14,16 +14,11 @@
 
 namespace hga {
 
-// Bounded wait on an mbarrier phase.  Gives up after 2^20 polls (sets the CTA's abort flag) or as
+// Bounded wait on an mbarrier phase.  Gives up after the time limit (sets the CTA's abort flag) or as
 // soon as another thread of the CTA has given up; the caller then unwinds without touching TMEM.
 __device__ __forceinline__ bool bwd_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
   if (sm100::mbar_test_wait(bar, parity)) return true;    // fast path: the phase is already over
-  for (uint32_t i = 0; i < (1u << 20); ++i) {
-    if (sm100::mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && *abort) return false;
-  }
-  *abort = 1;
-  return false;
+  return sm100::mbar_wait_bounded(bar, parity, abort);
 }
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {

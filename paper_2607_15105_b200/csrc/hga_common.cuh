@@ -51,6 +51,13 @@ __host__ __device__ inline void item_coords(const Dims& dm, int item, int& b, in
   b = bh / dm.Hkv;
 }
 
+// Row layout of an item inside the tensor-core kernels: every query head's Bq rows are padded to
+// whole octets (8 rows = one TMA box / swizzle atom), so row r of the item is (head r / bq_pad,
+// token r % bq_pad) and rows with token >= Bq are padding.  Bq is a multiple of 8 except in
+// generation-shaped problems (HGA_FLAG_DECODE), where bq_pad = 8 or 16 for 1..16 new tokens.
+__host__ __device__ inline int bq_padded(const Dims& dm) { return (dm.Bq + 7) & ~7; }
+__host__ __device__ inline int rows_padded(const Dims& dm) { return dm.G * bq_padded(dm); }
+
 // Upper bound of routed tokens per item (sink + groups + local window + the block itself).
 __host__ __device__ inline int max_routed_tokens(const Dims& dm) {
   return dm.sink + dm.width * dm.g + dm.local + dm.Bq + dm.c;

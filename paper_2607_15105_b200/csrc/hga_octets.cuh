@@ -57,7 +57,7 @@ __device__ inline int build_octet_table(const Dims& dm, const Window& w, const i
     n_far = __shfl_sync(full, n, 0);
   }
   for (int o = lane; o < n_sink; o += 32) oct_row[o] = 8 * o;
-  const int n_local = (w.p0 + dm.Bq - w.ls) / 8;
+  const int n_local = (w.p0 + dm.Bq - w.ls + 7) / 8;      // the last octet may be partial (decode shapes)
   for (int o = lane; o < n_local; o += 32) oct_row[n_far + o] = w.ls + 8 * o;
   __syncwarp();
   *bad_out = bad;

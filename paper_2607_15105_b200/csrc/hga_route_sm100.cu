@@ -43,12 +43,7 @@ struct RouteSmem {
 };
 
 __device__ __forceinline__ bool rt_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
-  for (uint32_t i = 0; i < (1u << 20); ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && *abort) return false;
-  }
-  *abort = 1;
-  return false;
+  return mbar_wait_bounded(bar, parity, abort);
 }
 
 __device__ __forceinline__ uint32_t rt_orderable(float f) {
@@ -76,8 +71,13 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   item_coords(dm, item, b, h, qb);
   const Window w = window_of(dm, qb);
   const int j0 = w.se / dm.c, n_cand = (w.ls - w.se) / dm.c;
-  const int n_halves = dm.rows > 256 ? dm.rows / 256 : 1;
-  const int rows_half = dm.rows / n_halves;                  // N of one MMA: <= 256, multiple of 32
+  // query rows on N: every head's Bq rows padded to whole octets, the total padded to a multiple of 32
+  // (padding columns hold whatever shared memory held and are masked when the columns are reduced)
+  const int bq_pad = bq_padded(dm), rows_pad = rows_padded(dm);
+  const int n_cols = (rows_pad + 31) & ~31;
+  const bool all_rows_real = n_cols == dm.rows;
+  const int n_halves = n_cols > 256 ? n_cols / 256 : 1;
+  const int rows_half = n_cols / n_halves;                   // N of one MMA: <= 256, multiple of 32
   const int k_sel = dm.kc < n_cand ? dm.kc : n_cand;
   const int opc = dm.per / 8;                                // octets per opened chunk
   const int n_ct = (n_cand + 127) / 128;                     // chunk tiles
@@ -113,10 +113,10 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     if (warp == 0) {
       // ---------------------------------------------------------------- producer
       if (!phase2) {
-        if (lane == 0) mbar_arrive_expect_tx(&sm.q_full, (uint32_t)q_bytes);
+        if (lane == 0) mbar_arrive_expect_tx(&sm.q_full, (uint32_t)(rows_pad / 8) * kOctBytes);
         __syncwarp();
-        for (int o = lane; o < dm.rows / 8; o += 32) {
-          const int r = 8 * o, a = r / dm.Bq, t = r % dm.Bq;
+        for (int o = lane; o < rows_pad / 8; o += 32) {
+          const int r = 8 * o, a = r / bq_pad, t = r % bq_pad;    // rows past the segment arrive as zeros
           tma_load_5d(q_smem + o * kOctBytes, &map_q, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
         }
       }
@@ -184,6 +184,15 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             uint32_t x[32];
             tmem_ld32(lane_base + buf * 256 + c, x);
             tmem_wait_ld();
+            if (!all_rows_real) {
+              // padding columns become the neutral element of the reduction
+              const float neutral = agg == 1 ? 0.f : -INFINITY;
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                const int col = hf * rows_half + c + i;
+                if (col >= rows_pad || col % bq_pad >= dm.Bq) x[i] = __float_as_uint(neutral);
+              }
+            }
             if (agg == 0) {
 #pragma unroll
               for (int i = 0; i < 32; ++i) best = fmaxf(best, __uint_as_float(x[i]));
@@ -347,7 +356,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 }
 
 static size_t route_sm100_smem(const Dims& dm, int max_cand) {
-  const size_t q_bytes = (size_t)dm.rows * dm.d * 2;
+  const size_t q_bytes = (size_t)((rows_padded(dm) + 31) & ~31) * dm.d * 2;
   const size_t base = dm.d == 128 ? sizeof(RouteSmem<128>) : sizeof(RouteSmem<64>);
   return base + 1024 + q_bytes + 1024 + sizeof(unsigned long long) * (max_cand + 2) +
          sizeof(float) * ((size_t)dm.kc * dm.per + 8);
@@ -360,8 +369,8 @@ static int route_max_cand(const Dims& dm) {
 
 bool route_sm100_supported(const Dims& dm) {
   if (dm.flags & HGA_FLAG_GENERIC_KERNELS) return false;
-  if (dm.rows % 32 != 0) return false;
-  if (dm.rows > 256 && dm.rows % 256 != 0) return false;
+  const int n_cols = (rows_padded(dm) + 31) & ~31;
+  if (n_cols > 256 && (n_cols % 256 != 0 || n_cols != dm.rows)) return false;
   if (dm.per != 8 && dm.per != 16) return false;            // opened chunk = 1 or 2 octets of summaries
   if (dm.kc > 1024) return false;
   if ((dm.flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) && dm.kc * dm.per > 4096) return false;   // bitmap in sel[]
@@ -393,7 +402,7 @@ static int launch_route(const Dims& dm, const void* Q, const void* chunk_sum, co
   if (e != cudaSuccess) return record_cuda(e);
   const int items = dm.B * dm.Hkv * dm.NQB;
   k_route_sm100<D><<<items, kRtThreads, smem, st>>>(mq, mc, mg, dm, chunk_idx, group_idx, n_groups, chunk_scores,
-                                                   group_scores, dm.rows * D * 2, max_cand);
+                                                   group_scores, ((rows_padded(dm) + 31) & ~31) * D * 2, max_cand);
   count_launch();
   return record_cuda(cudaGetLastError());
 }

@@ -61,15 +61,30 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: each try_wait may itself block for a hardware-defined time slice, so the
-// limit below is seconds of wall clock at most.  Returns false when it gives up.
+// Bounded waits give up after kWaitCycles SM cycles (about half a second; a legitimate wait in these
+// kernels lasts microseconds) or kWaitLimit polls, whichever comes first: each try_wait may itself
+// block for a hardware-defined time slice, so a poll count alone can add up to minutes.
 constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr long long kWaitCycles = 1ll << 30;
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// One bounded wait shared by the kernels: polls until the phase completes, the CTA's abort flag is
+// seen (checked every 64 polls), or the time limit runs out (then sets the flag).  abort may be null.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
   for (uint32_t i = 0; i < kWaitLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 63u) {
+      if (abort && *abort) return false;
+      if (clock64() - t0 > kWaitCycles) break;
+    }
   }
+  if (abort) *abort = 1;
   return false;
+}
+
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  return mbar_wait_bounded(bar, parity, nullptr);
 }
 
 // ----------------------------------------------------------------------------- proxies / fences
