@@ -278,6 +278,109 @@ def time_tbptt_walk(cfg, args, stream):
 
 # ----------------------------------------------------------------------------- main arm
 
+def time_decode(args, stream, peaks):
+    """Generation-shaped step (configuration 7): route + attention forward for one new token per
+    sequence, CUDA-graph replay, L2 flushed between steps.  HBM-bound: the roofline is the bytes the
+    step must read (candidate chunk summaries, opened group summaries, routed K/V rows, Q) and write
+    (O, LSE, index lists) over the measured copy bandwidth."""
+    import torch
+    from paper_2607_15105_b200 import binding
+    cfg = CONFIGS[7]
+    x = make_inputs(cfg)
+
+    def dev(a):
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+
+    Q, K, V = dev(x["Q"]), dev(x["K"]), dev(x["V"])
+    buf = binding.HgaLayerBuffers(cfg, backward=False, flags=args.flags)
+    closed = (cfg.total_len // cfg.chunk) * cfg.chunk
+    buf.build_summaries(K, 0, closed)               # resident state: summaries of every closed chunk
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+
+    def step(e=None):
+        if e:
+            e[0].record(stream)
+        buf.route(Q)
+        if e:
+            e[1].record(stream)
+        buf.attn_fwd(Q, K, V)
+        if e:
+            e[2].record(stream)
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    torch.cuda.synchronize()
+    for i in range(args.steps):
+        flush.zero_()
+        step(ev[i])
+    torch.cuda.synchronize()
+    per_call = np.array([[e[k].elapsed_time(e[k + 1]) for k in range(2)] for e in ev]) * 1e-3
+    graph_s = None
+    if not args.no_graph:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=torch.cuda.Stream()):
+            step()
+        gev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+        for i in range(args.warmup + args.steps):
+            flush.zero_()
+            if i >= args.warmup:
+                gev[i - args.warmup][0].record(stream)
+            g.replay()
+            if i >= args.warmup:
+                gev[i - args.warmup][1].record(stream)
+        torch.cuda.synchronize()
+        graph_s = float(np.median([a.elapsed_time(b) for a, b in gev])) * 1e-3
+    status = int(buf.status.item())
+    # algorithmic bytes of one step, counted from the windows and the lists the router produced
+    c, g_, d, G, n = cfg.chunk, cfg.group, cfg.head_dim, cfg.gqa, cfg.q_block
+    per = c // g_
+    H = cfg.history
+    ls = max(0, (H - cfg.local) // c * c)
+    se = min(cfg.sink, ls)
+    n_cand = (ls - se) // c
+    k_sel = min(cfg.topk_chunks, n_cand)
+    ng = buf.n_groups.cpu().numpy().astype(np.int64)
+    items = cfg.batch * cfg.n_kv_heads
+    route_bytes = items * ((n_cand + k_sel * per) * d * 2 + G * n * d * 2 + 4 * (k_sel + k_sel * cfg.kg_eff + 1))
+    keys = se + ng * g_ + (cfg.total_len - ls)
+    fwd_bytes = int(keys.sum()) * d * 2 * 2 + items * (2 * G * n * d * 2 + G * n * 4 + 4 * (k_sel * cfg.kg_eff + 1))
+    med = np.median(per_call, axis=0)
+    step_s = graph_s if graph_s is not None else float(med.sum())
+    hbm = peaks["hbm_gbs"] * 1e9
+    out = {"workload": cfg.name, "tokens_per_step": cfg.tokens_per_step, "step": "route + attention forward "
+           "(summaries are resident; no chunk closes at this length)",
+           "us_per_step": round(step_s * 1e6, 2), "tokens_per_s": round(cfg.tokens_per_step / step_s, 1),
+           "launch": "cuda graph replay" if graph_s is not None else "eager",
+           "per_call_us_median": {"route": round(float(med[0]) * 1e6, 2), "attn_fwd": round(float(med[1]) * 1e6, 2)},
+           "roofline": {"bound": "hbm", "algorithmic_bytes": int(route_bytes + fwd_bytes),
+                        "achieved": round((route_bytes + fwd_bytes) / step_s / 1e9, 1), "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "frac": round((route_bytes + fwd_bytes) / step_s / hbm, 4),
+                        "peak_source": peaks["source"],
+                        "route": {"algorithmic_bytes": int(route_bytes), "frac": round(route_bytes / float(med[0]) / hbm, 4)},
+                        "attn_fwd": {"algorithmic_bytes": int(fwd_bytes), "frac": round(fwd_bytes / float(med[1]) / hbm, 4)}},
+           "l2": "flushed between timed steps (512 MiB write)", "device_status_word": status}
+    if not args.no_cpu_baseline:
+        import oracle
+        t0 = time.perf_counter()
+        sample = np.arange(0, items, max(1, items // 32), dtype=np.int32)
+        cs, gs = bits(buf.chunk_sum), bits(buf.group_sum)
+        t0 = time.perf_counter()
+        r = oracle.route(cfg, x["Q"], cs, gs, items=sample)
+        oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], r["group_idx"], r["n_groups"], items=sample)
+        dt = time.perf_counter() - t0
+        out["cpu_baseline"] = {"value": round(len(sample) * n / cfg.n_kv_heads / dt, 1), "unit": "tokens/s",
+                               "cores": oracle.num_threads(), "kind": "oracle",
+                               "sample": "%d of %d (sequence, kv head) items: route + attention forward" % (len(sample), items)}
+    return out
+
+
+def bits(t):
+    import torch
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -288,6 +391,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA-graph replay")
     ap.add_argument("--flags", type=int, default=0, help="hga_params.flags (debugging)")
+    ap.add_argument("--no-decode", action="store_true", help="skip the generation-shaped step (configuration 7)")
     ap.add_argument("--no-walk", action="store_true",
                     help="skip the whole-sequence TBPTT walk (every segment of the sequence, one layer)")
     args = ap.parse_args()
@@ -437,6 +541,10 @@ def main():
     if rank == 0 and world == 1 and cfg.backward and not args.no_walk and cfg.history > 0:
         walk = time_tbptt_walk(cfg, args, stream)
     clocks = sampler.stop() if rank == 0 else None      # sampled across all timed loops above
+    # generation-shaped step (its inputs are drawn on the host first, so it runs outside the clock samples)
+    decode = None
+    if rank == 0 and world == 1 and args.config == 3 and not args.no_decode:
+        decode = time_decode(args, stream, load_peaks())
     status = int(buf.status.item())
 
     def max_over_ranks(v):
@@ -492,6 +600,8 @@ def main():
         }
         if walk is not None:
             line["tbptt_walk"] = walk
+        if decode is not None:
+            line["decode"] = decode
         if not args.no_cpu_baseline and world == 1:
             tps, threads, what, _ = oracle_throughput(cfg, x)
             line["cpu_baseline"] = {"value": round(tps, 3), "unit": "tokens/s", "cores": threads,

@@ -16,28 +16,35 @@
 #include "hga_common.cuh"
 #include "hga_sm100.cuh"
 
+// Optional phase stamps: a profiling harness defines these macros; otherwise no-ops.
+#ifndef HGA_RT_STAMP
+#define HGA_RT_DECL
+#define HGA_RT_STAMP(k)
+#endif
+
 namespace hga {
 
 using namespace sm100;
 
 constexpr int kRtThreads = 320;     // warp 0 producer, warp 1 MMA, warps 2-5 readers, 6-9 help in select
-// One summary-tile stage and one accumulator per CTA: an item has only a few tiles, so there is
-// little to pipeline inside a CTA; the smaller footprint (under half of the shared memory and of
-// TMEM) lets two CTAs share an SM, and the serial phases of one item overlap the GEMMs of another.
-constexpr int kRtStages = 1;
-constexpr int kRtAccs = 1;
-constexpr int kRtTmemCols = 256 * kRtAccs;
+// Training shapes (up to 256 query rows on N): one summary-tile stage and one accumulator per CTA.  An
+// item has only a few tiles, so there is little to pipeline inside a CTA; the smaller footprint (under
+// half of the shared memory and of TMEM) lets two CTAs share an SM, and the serial phases of one item
+// overlap the GEMMs of another.  Generation shapes (at most 128 padded query rows) leave room for a
+// two-stage ring and two 128-column accumulators in the same footprint, so the summary tiles of an
+// item stream from HBM back to back.
+constexpr int kRtTmemCols = 256;
 
-template <int D>
+template <int D, int STAGES, int ACCS>
 struct RouteSmem {
   static constexpr int kTile = 128 * D * 2;
-  alignas(1024) uint8_t a[kRtStages][kTile];   // summary tiles (A operand)
-  uint64_t q_full, a_full[kRtStages], a_empty[kRtStages], acc_full[kRtAccs], acc_free[kRtAccs];
+  alignas(1024) uint8_t a[STAGES][kTile];   // summary tiles (A operand)
+  uint64_t q_full, a_full[STAGES], a_empty[STAGES], acc_full[ACCS], acc_free[ACCS];
   uint32_t tmem_base;
   volatile int abort;
   int n_sel;
   unsigned long long warp_best[kRtThreads / 32];
-  int sel[1024];          // selected chunk ids, first in selection order, then ascending
+  alignas(16) int sel[1024];   // selection bitmaps and 32-bit scores, or chunk ids in selection order
   int sorted[1024];
   // dynamic tail: Q rows (B operand, 1024-aligned), keys[n_cand_max] u64, gscore[kc*per] f32
 };
@@ -51,7 +58,7 @@ __device__ __forceinline__ uint32_t rt_orderable(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-template <int D>
+template <int D, int STAGES, int ACCS>
 __global__ void __launch_bounds__(kRtThreads, 2)
 k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_cs,
               const __grid_constant__ CUtensorMap map_gs, Dims dm, int32_t* __restrict__ chunk_idx,
@@ -60,12 +67,16 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
               int max_cand) {
   constexpr int kOctBytes = 8 * D * 2;
   extern __shared__ uint8_t smem_raw[];
-  RouteSmem<D>& sm = *reinterpret_cast<RouteSmem<D>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  using Smem = RouteSmem<D, STAGES, ACCS>;
+  constexpr uint32_t kAccCols = kRtTmemCols / ACCS;   // TMEM columns per accumulator
+  Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(&sm + 1) + 1023) & ~uintptr_t(1023));
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(q_smem + q_bytes);
   float* gscore = reinterpret_cast<float*>(keys + max_cand + 2);
+  uint32_t* okeys = reinterpret_cast<uint32_t*>(sm.sel) + 64;   // orderable scores alone, when candidates <= 640
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  HGA_RT_DECL;
   const int item = blockIdx.x;
   int b, h, qb;
   item_coords(dm, item, b, h, qb);
@@ -85,71 +96,102 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   volatile int* abort = &sm.abort;
   const int agg = score_agg_of(dm.flags);
   constexpr float kLog2e = 1.4426950408889634f;
+  uint32_t col_mask = 0;                                       // bit i: column i of a block of 32 is a real query row
+  for (int i = 0; i < 32; ++i) col_mask |= (uint32_t)((i % bq_pad) < dm.Bq) << i;
 
-  if (tid == 0) {
-    mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < kRtStages; ++s) { mbar_init(&sm.a_full[s], 1); mbar_init(&sm.a_empty[s], 1); }
-    for (int s = 0; s < kRtAccs; ++s) { mbar_init(&sm.acc_full[s], 1); mbar_init(&sm.acc_free[s], 128); }
-    sm.abort = 0;
-    sm.n_sel = 0;
-    fence_barrier_init();
+  // Copies one 128-row summary tile (16 octet boxes, one per lane) into its ring stage; all lanes of warp 0.
+  auto issue_tile = [&](int tg, int t, bool phase2) {
+    const int s = tg % STAGES;
+    if (lane == 0) mbar_arrive_expect_tx(&sm.a_full[s], Smem::kTile);
+    __syncwarp();
+    if (lane < 16) {
+      if (!phase2) {
+        const int row = j0 + 128 * t + 8 * lane;              // rows past the table read as zeros
+        tma_load_5d(sm.a[s] + lane * kOctBytes, &map_cs, &sm.a_full[s], 0, row, 0, h, b);
+      } else {
+        const int oc = 16 * t + lane, r = oc / opc;
+        const int row = r < k_sel ? sm.sorted[r] * dm.per + 8 * (oc % opc) : dm.Ng;
+        tma_load_5d(sm.a[s] + lane * kOctBytes, &map_gs, &sm.a_full[s], 0, row, 0, h, b);
+      }
+    }
+    HGA_RT_STAMP(3 + tg);
+  };
+  const int n_pre = k_sel > 0 ? (n_ct < STAGES ? n_ct : STAGES) : 0;   // chunk tiles copied ahead of the CTA barrier
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_init(&sm.q_full, 1);
+      for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.a_full[s], 1); mbar_init(&sm.a_empty[s], 1); }
+      for (int s = 0; s < ACCS; ++s) { mbar_init(&sm.acc_full[s], 1); mbar_init(&sm.acc_free[s], 128); }
+      sm.abort = 0;
+      sm.n_sel = 0;
+      fence_barrier_init();
+      prefetch_tensormap(&map_q); prefetch_tensormap(&map_cs); prefetch_tensormap(&map_gs);
+    }
+    __syncwarp();
+    // the first chunk tiles depend on nothing: their copies start before the CTA meets
+    for (int t = 0; t < n_pre; ++t) issue_tile(t, t, false);
+    if (lane == 0 && k_sel > 0) mbar_arrive_expect_tx(&sm.q_full, (uint32_t)(rows_pad / 8) * kOctBytes);
   }
   if (warp == 1) {
     tmem_alloc(&sm.tmem_base, kRtTmemCols);
     tmem_relinquish();
-  }
-  if (warp == 0 && lane == 0) {
-    prefetch_tensormap(&map_q); prefetch_tensormap(&map_cs); prefetch_tensormap(&map_gs);
   }
   __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sm.tmem_base;
+  HGA_RT_STAMP(1);
 
   // One GEMM phase: tiles [t_begin, t_begin + n_tiles) in the global tile numbering (which
   // drives barrier parities); `phase2` selects the octet source.
   auto run_phase = [&](int t_begin, int n_tiles, bool phase2) {
+    if (!phase2 && warp >= 2 && lane < 4) {
+      // The item's query rows, one octet box per lane.  Issuing a box costs its warp a few hundred
+      // cycles and warps issue in parallel, so the boxes are spread over the eight non-producer warps.
+      for (int o = (warp - 2) * 4 + lane; o < rows_pad / 8; o += 32) {
+        const int r = 8 * o, a = r / bq_pad, t = r % bq_pad;    // rows past the segment arrive as zeros
+        tma_load_5d(q_smem + o * kOctBytes, &map_q, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
+      }
+      HGA_RT_STAMP(2);
+    }
+    if (phase2 && warp >= 2 && lane < 2) {
+      // First tile of the opened chunks' group summaries, again spread over the eight warps (two
+      // octet boxes each).  Its ring stage is known to be free: every tile of the first phase has been
+      // read back, so no barrier needs to be observed; warp 0 announces the bytes.
+      const int s = t_begin % STAGES;
+      const int oc = (warp - 2) * 2 + lane, r = oc / opc;
+      const int row = r < k_sel ? sm.sorted[r] * dm.per + 8 * (oc % opc) : dm.Ng;
+      tma_load_5d(sm.a[s] + oc * kOctBytes, &map_gs, &sm.a_full[s], 0, row, 0, h, b);
+    }
+    __syncwarp();
     if (warp == 0) {
       // ---------------------------------------------------------------- producer
-      if (!phase2) {
-        if (lane == 0) mbar_arrive_expect_tx(&sm.q_full, (uint32_t)(rows_pad / 8) * kOctBytes);
-        __syncwarp();
-        for (int o = lane; o < rows_pad / 8; o += 32) {
-          const int r = 8 * o, a = r / bq_pad, t = r % bq_pad;    // rows past the segment arrive as zeros
-          tma_load_5d(q_smem + o * kOctBytes, &map_q, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
-        }
-      }
       bool ok = true;
-      for (int t = 0; t < n_tiles; ++t) {
-        const int tg = t_begin + t, s = tg % kRtStages, use = tg / kRtStages;
+      if (phase2) {
+        if (lane == 0) mbar_arrive_expect_tx(&sm.a_full[t_begin % STAGES], Smem::kTile);
+        HGA_RT_STAMP(3 + t_begin);
+      }
+      for (int t = phase2 ? 1 : n_pre; t < n_tiles; ++t) {
+        const int tg = t_begin + t, s = tg % STAGES, use = tg / STAGES;
         if (lane == 0 && use > 0) ok = rt_wait(&sm.a_empty[s], (use - 1) & 1, abort);
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
-        if (lane == 0) mbar_arrive_expect_tx(&sm.a_full[s], RouteSmem<D>::kTile);
-        __syncwarp();
-        if (lane < 16) {
-          int row;
-          if (!phase2) {
-            row = j0 + 128 * t + 8 * lane;                    // rows past the table read as zeros
-            tma_load_5d(sm.a[s] + lane * kOctBytes, &map_cs, &sm.a_full[s], 0, row, 0, h, b);
-          } else {
-            const int oc = 16 * t + lane, r = oc / opc;
-            row = r < k_sel ? sm.sorted[r] * dm.per + 8 * (oc % opc) : dm.Ng;
-            tma_load_5d(sm.a[s] + lane * kOctBytes, &map_gs, &sm.a_full[s], 0, row, 0, h, b);
-          }
-        }
+        issue_tile(tg, t, phase2);
       }
     } else if (warp == 1) {
       // ---------------------------------------------------------------- MMA issuer
       if (lane == 0) {
         const uint32_t idesc = idesc_bf16_f32(128, rows_half, 0, 0);
         bool ok = phase2 ? true : rt_wait(&sm.q_full, 0, abort);
+        if (!phase2) HGA_RT_STAMP(2);
         for (int t = 0; t < n_tiles && ok; ++t) {
-          const int tg = t_begin + t, s = tg % kRtStages;
-          ok = rt_wait(&sm.a_full[s], (tg / kRtStages) & 1, abort);
+          const int tg = t_begin + t, s = tg % STAGES;
+          ok = rt_wait(&sm.a_full[s], (tg / STAGES) & 1, abort);
+          HGA_RT_STAMP(3 + tg);
           for (int hf = 0; hf < n_halves && ok; ++hf) {
-            const int step = tg * n_halves + hf, buf = step % kRtAccs, use = step / kRtAccs;
+            const int step = tg * n_halves + hf, buf = step % ACCS, use = step / ACCS;
             if (use > 0) ok = rt_wait(&sm.acc_free[buf], (use - 1) & 1, abort);
             if (!ok) break;
             tc_fence_after_sync();
@@ -159,11 +201,12 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
               const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-              mma_ss(tmem + buf * 256, desc_advance(ad, off), desc_advance(bd, off), idesc, kk > 0);
+              mma_ss(tmem + buf * kAccCols, desc_advance(ad, off), desc_advance(bd, off), idesc, kk > 0);
             }
             mma_commit(&sm.acc_full[buf]);
           }
           if (ok) mma_commit(&sm.a_empty[s]);
+          HGA_RT_STAMP(12 + tg);
         }
       }
     } else if (warp < 6) {
@@ -176,22 +219,24 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const int tg = t_begin + t;
         float best = -FLT_MAX, sum = 0.f;    // log-sum-exp: (running maximum, sum of exp(dot - maximum))
         for (int hf = 0; hf < n_halves; ++hf) {
-          const int step = tg * n_halves + hf, buf = step % kRtAccs;
-          ok = __all_sync(0xffffffffu, rt_wait(&sm.acc_full[buf], (step / kRtAccs) & 1, abort));
+          const int step = tg * n_halves + hf, buf = step % ACCS;
+          ok = __all_sync(0xffffffffu, rt_wait(&sm.acc_full[buf], (step / ACCS) & 1, abort));
           if (!ok) break;
           tc_fence_after_sync();
+          HGA_RT_STAMP(3 + tg);
           for (int c = 0; c < rows_half; c += 32) {
             uint32_t x[32];
-            tmem_ld32(lane_base + buf * 256 + c, x);
+            tmem_ld32(lane_base + buf * kAccCols + c, x);
             tmem_wait_ld();
             if (!all_rows_real) {
-              // padding columns become the neutral element of the reduction
+              // padding columns become the neutral element of the reduction (bq_pad divides 32, so the
+              // pattern of real columns repeats in every block of 32; only the last block can be cut)
               const float neutral = agg == 1 ? 0.f : -INFINITY;
+              const int left = rows_pad - (hf * rows_half + c);
+              const uint32_t m = left >= 32 ? col_mask : (col_mask & ((1u << (left > 0 ? left : 0)) - 1u));
 #pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                const int col = hf * rows_half + c + i;
-                if (col >= rows_pad || col % bq_pad >= dm.Bq) x[i] = __float_as_uint(neutral);
-              }
+              for (int i = 0; i < 32; ++i)
+                if (!((m >> i) & 1u)) x[i] = __float_as_uint(neutral);
             }
             if (agg == 0) {
 #pragma unroll
@@ -210,13 +255,17 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
           }
           tc_fence_before_sync();
           mbar_arrive(&sm.acc_free[buf]);
+          HGA_RT_STAMP(12 + tg);
         }
         if (!ok) break;
         if (agg == 1) best = sum * (1.f / (float)dm.rows);
         else if (agg == 2) best += logf(sum);
         const int i = 128 * t + row;
         if (!phase2) {
-          if (i < n_cand) keys[i] = ((unsigned long long)rt_orderable(best) << 32) | (uint32_t)(0x7fffffff - (j0 + i));
+          if (i < n_cand) {
+            keys[i] = ((unsigned long long)rt_orderable(best) << 32) | (uint32_t)(0x7fffffff - (j0 + i));
+            if (n_cand <= 2 * kRtThreads) okeys[i] = rt_orderable(best);
+          }
           if (chunk_scores && i < n_cand) chunk_scores[(int64_t)item * dm.Nc + j0 + i] = best;
         } else {
           if (i < k_sel * dm.per) gscore[i] = best;
@@ -236,6 +285,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   if (k_sel > 0) run_phase(0, n_ct, false);
   __syncwarp();          // the roles diverge inside a warp: reconverge before the block barrier
   __syncthreads();
+  HGA_RT_STAMP(20);
 
   // ---------------------------------------------------------------------- chunk top-k
   if (!sm.abort) {
@@ -244,20 +294,57 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       // is part of the key), no rounds and no block-wide arg-max.  A candidate is selected when
       // fewer than k_sel keys beat it; its place in the ascending output is the number of selected
       // candidates with a lower index.
-      unsigned long long* flags = reinterpret_cast<unsigned long long*>(sm.sel);   // bit i: candidate i selected
-      for (int i = tid; i < (n_cand + 63) / 64; i += kRtThreads) flags[i] = 0;
+      // The count runs on the 32-bit orderable scores alone (four per 16-byte load).  Equal scores
+      // then share a rank; that only matters when a tie straddles the k-th place, which shows as a
+      // selection of the wrong size and is redone on the full 64-bit keys (ties to the lowest index).
+      uint32_t* flags = reinterpret_cast<uint32_t*>(sm.sel);      // bit i: candidate i selected (20 words at most)
+      auto rank_select = [&](bool exact) {
+        for (int base = 0; base < n_cand; base += kRtThreads) {   // warp-uniform trip count (ballots below)
+          const int i = base + tid;
+          bool sel = false;
+          if (i < n_cand) {
+            int beat = 0, q = 0;
+            if (!exact) {
+              const uint32_t mine = okeys[i];
+              const uint4* k4 = reinterpret_cast<const uint4*>(okeys);
+#pragma unroll 4
+              for (; q + 4 <= n_cand; q += 4) {
+                const uint4 kk = k4[q >> 2];
+                beat += (int)(kk.x > mine) + (int)(kk.y > mine) + (int)(kk.z > mine) + (int)(kk.w > mine);
+              }
+              for (; q < n_cand; ++q) beat += okeys[q] > mine;
+            } else {
+              const unsigned long long mine = keys[i];
+              const ulonglong2* k2 = reinterpret_cast<const ulonglong2*>(keys);
+#pragma unroll 4
+              for (; q + 2 <= n_cand; q += 2) {
+                const ulonglong2 kk = k2[q >> 1];
+                beat += (int)(kk.x > mine) + (int)(kk.y > mine);
+              }
+              if (q < n_cand) beat += keys[q] > mine;
+            }
+            sel = beat < k_sel;
+          }
+          const uint32_t word = __ballot_sync(0xffffffffu, sel);
+          if (lane == 0 && base + warp * 32 < n_cand) flags[(base + warp * 32) >> 5] = word;
+        }
+      };
+      HGA_RT_STAMP(24);
+      rank_select(false);
+      HGA_RT_STAMP(25);
       __syncthreads();
-      for (int i = tid; i < n_cand; i += kRtThreads) {
-        const unsigned long long mine = keys[i];
-        int beat = 0;
-        for (int q = 0; q < n_cand; ++q) beat += keys[q] > mine;
-        if (beat < k_sel) atomicOr(&flags[i >> 6], 1ull << (i & 63));
+      int n_picked = 0;
+      for (int q = 0; q < (n_cand + 31) / 32; ++q) n_picked += __popc(flags[q]);
+      if (n_picked != k_sel) {          // same value in every thread
+        __syncthreads();
+        rank_select(true);
+        __syncthreads();
       }
-      __syncthreads();
+      HGA_RT_STAMP(26);
       for (int i = tid; i < n_cand; i += kRtThreads) {
-        if ((flags[i >> 6] >> (i & 63)) & 1ull) {
-          int pos = __popcll(flags[i >> 6] & ((1ull << (i & 63)) - 1));
-          for (int q = 0; q < (i >> 6); ++q) pos += __popcll(flags[q]);
+        if ((flags[i >> 5] >> (i & 31)) & 1u) {
+          int pos = __popc(flags[i >> 5] & ((1u << (i & 31)) - 1u));
+          for (int q = 0; q < (i >> 5); ++q) pos += __popc(flags[q]);
           sm.sorted[pos] = j0 + i;
         }
       }
@@ -296,31 +383,43 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   __syncthreads();
 
   // ---------------------------------------------------------------------- groups of the opened chunks
+  HGA_RT_STAMP(21);
   if (k_sel > 0 && !sm.abort) run_phase(n_ct, n_gt, true);
   __syncwarp();
   __syncthreads();
+  HGA_RT_STAMP(22);
   if (!sm.abort) {
     int32_t* gi = group_idx + (int64_t)item * dm.width;
-    if (dm.flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) {
-      // One budget over all opened chunks: slot i (chunk-major, i.e. ascending group id) is selected
-      // when fewer than k_sel * kg_eff slots beat it (higher score, or equal score and lower id); its
-      // place in the ascending output is the number of selected slots below it.
-      const int total = k_sel * dm.per, want = k_sel * dm.kge;
-      unsigned long long* flags = reinterpret_cast<unsigned long long*>(sm.sel);   // 4096 bits
-      for (int i = tid; i < (total + 63) / 64; i += kRtThreads) flags[i] = 0;
-      __syncthreads();
-      for (int i = tid; i < total; i += kRtThreads) {
-        const float mine = gscore[i];
-        int beat = 0;
-        for (int q = 0; q < total; ++q) beat += gscore[q] > mine || (gscore[q] == mine && q < i);
-        if (beat < want) atomicOr(&flags[i >> 6], 1ull << (i & 63));
-        if (group_scores) group_scores[(int64_t)item * dm.kc * dm.per + i] = mine;
+    const bool global_budget = (dm.flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) != 0;
+    if (k_sel * dm.per <= 4096) {
+      // One thread per slot (opened chunk, group), slots in chunk-major order = ascending group id.
+      // A slot is selected when fewer than `want` slots of its scope beat it (higher score, or equal
+      // score and lower id); the scope is its own chunk (want = kg_eff) or, with one budget over all
+      // opened chunks, every slot (want = k_sel * kg_eff).  Its place in the ascending output is the
+      // number of selected slots below it.
+      const int total = k_sel * dm.per;
+      uint32_t* flags = reinterpret_cast<uint32_t*>(sm.sel);      // 4096 bits
+      const int want = global_budget ? k_sel * dm.kge : dm.kge;
+      for (int base = 0; base < total; base += kRtThreads) {      // warp-uniform trip count (ballots below)
+        const int i = base + tid;
+        bool sel = false;
+        if (i < total) {
+          const float mine = gscore[i];
+          const int lo = global_budget ? 0 : i - i % dm.per, hi = global_budget ? total : lo + dm.per;
+          int beat = 0;
+#pragma unroll 8
+          for (int q = lo; q < hi; ++q) beat += gscore[q] > mine || (gscore[q] == mine && q < i);
+          sel = beat < want;
+          if (group_scores) group_scores[(int64_t)item * dm.kc * dm.per + i] = mine;
+        }
+        const uint32_t word = __ballot_sync(0xffffffffu, sel);
+        if (lane == 0 && base + warp * 32 < total) flags[(base + warp * 32) >> 5] = word;
       }
       __syncthreads();
       for (int i = tid; i < total; i += kRtThreads)
-        if ((flags[i >> 6] >> (i & 63)) & 1ull) {
-          int pos = __popcll(flags[i >> 6] & ((1ull << (i & 63)) - 1));
-          for (int q = 0; q < (i >> 6); ++q) pos += __popcll(flags[q]);
+        if ((flags[i >> 5] >> (i & 31)) & 1u) {
+          int pos = __popc(flags[i >> 5] & ((1u << (i & 31)) - 1u));
+          for (int q = 0; q < (i >> 5); ++q) pos += __popc(flags[q]);
           gi[pos] = sm.sorted[i / dm.per] * dm.per + i % dm.per;
         }
     } else
@@ -346,6 +445,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     if (tid == 0) n_groups[item] = k_sel * dm.kge;
   }
 
+  HGA_RT_STAMP(23);
   __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
@@ -355,9 +455,13 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   }
 }
 
+// Generation shapes (few query rows) take the pipelined instantiation.
+static bool route_pipelined(const Dims& dm) { return ((rows_padded(dm) + 31) & ~31) <= 128; }
+
 static size_t route_sm100_smem(const Dims& dm, int max_cand) {
   const size_t q_bytes = (size_t)((rows_padded(dm) + 31) & ~31) * dm.d * 2;
-  const size_t base = dm.d == 128 ? sizeof(RouteSmem<128>) : sizeof(RouteSmem<64>);
+  const size_t base = route_pipelined(dm) ? (dm.d == 128 ? sizeof(RouteSmem<128, 2, 2>) : sizeof(RouteSmem<64, 2, 2>))
+                                          : (dm.d == 128 ? sizeof(RouteSmem<128, 1, 1>) : sizeof(RouteSmem<64, 1, 1>));
   return base + 1024 + q_bytes + 1024 + sizeof(unsigned long long) * (max_cand + 2) +
          sizeof(float) * ((size_t)dm.kc * dm.per + 8);
 }
@@ -371,13 +475,14 @@ bool route_sm100_supported(const Dims& dm) {
   if (dm.flags & HGA_FLAG_GENERIC_KERNELS) return false;
   const int n_cols = (rows_padded(dm) + 31) & ~31;
   if (n_cols > 256 && (n_cols % 256 != 0 || n_cols != dm.rows)) return false;
+  if (n_cols != dm.rows && 32 % bq_padded(dm) != 0) return false;   // the padding mask repeats every 32 columns
   if (dm.per != 8 && dm.per != 16) return false;            // opened chunk = 1 or 2 octets of summaries
   if (dm.kc > 1024) return false;
   if ((dm.flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) && dm.kc * dm.per > 4096) return false;   // bitmap in sel[]
   return route_sm100_smem(dm, route_max_cand(dm)) <= 227 * 1024;
 }
 
-template <int D>
+template <int D, int STAGES, int ACCS>
 static int launch_route(const Dims& dm, const void* Q, const void* chunk_sum, const void* group_sum,
                         int32_t* chunk_idx, int32_t* group_idx, int32_t* n_groups, float* chunk_scores,
                         float* group_scores, cudaStream_t st) {
@@ -395,13 +500,13 @@ static int launch_route(const Dims& dm, const void* Q, const void* chunk_sum, co
     return HGA_ERR_UNSUPPORTED;
   const int max_cand = route_max_cand(dm);
   const size_t smem = route_sm100_smem(dm, max_cand);
-  cudaError_t e = cudaFuncSetAttribute(k_route_sm100<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(k_route_sm100<D, STAGES, ACCS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return record_cuda(e);
   // two CTAs per SM need the largest shared-memory carve-out
-  e = cudaFuncSetAttribute(k_route_sm100<D>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+  e = cudaFuncSetAttribute(k_route_sm100<D, STAGES, ACCS>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
   if (e != cudaSuccess) return record_cuda(e);
   const int items = dm.B * dm.Hkv * dm.NQB;
-  k_route_sm100<D><<<items, kRtThreads, smem, st>>>(mq, mc, mg, dm, chunk_idx, group_idx, n_groups, chunk_scores,
+  k_route_sm100<D, STAGES, ACCS><<<items, kRtThreads, smem, st>>>(mq, mc, mg, dm, chunk_idx, group_idx, n_groups, chunk_scores,
                                                    group_scores, ((rows_padded(dm) + 31) & ~31) * D * 2, max_cand);
   count_launch();
   return record_cuda(cudaGetLastError());
@@ -410,11 +515,11 @@ static int launch_route(const Dims& dm, const void* Q, const void* chunk_sum, co
 int launch_route_sm100(const Dims& dm, const void* Q, const void* chunk_sum, const void* group_sum,
                        int32_t* chunk_idx, int32_t* group_idx, int32_t* n_groups, float* chunk_scores,
                        float* group_scores, cudaStream_t st) {
-  if (dm.d == 128)
-    return launch_route<128>(dm, Q, chunk_sum, group_sum, chunk_idx, group_idx, n_groups, chunk_scores,
-                             group_scores, st);
-  return launch_route<64>(dm, Q, chunk_sum, group_sum, chunk_idx, group_idx, n_groups, chunk_scores,
-                          group_scores, st);
+#define HGA_ROUTE_ARGS dm, Q, chunk_sum, group_sum, chunk_idx, group_idx, n_groups, chunk_scores, group_scores, st
+  if (route_pipelined(dm))
+    return dm.d == 128 ? launch_route<128, 2, 2>(HGA_ROUTE_ARGS) : launch_route<64, 2, 2>(HGA_ROUTE_ARGS);
+  return dm.d == 128 ? launch_route<128, 1, 1>(HGA_ROUTE_ARGS) : launch_route<64, 1, 1>(HGA_ROUTE_ARGS);
+#undef HGA_ROUTE_ARGS
 }
 
 }  // namespace hga

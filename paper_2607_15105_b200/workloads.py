@@ -89,6 +89,10 @@ CONFIGS = {
                  topics=0, needles=0, backward=True, seed=1342),
     6: HgaConfig("cfg6_paper_default_16k", 1, 32, 8, 128, 16384, 2048, 64, 8, 64, 8, 8, 64, 128,
                  topics=256, needles=32, backward=True, seed=1343),
+    # generation-shaped: 32 sequences, one new token each behind 16 379 resident tokens (not a multiple of
+    # anything), the routing shape of configuration 3
+    7: HgaConfig("cfg7_decode_b32_16k", 32, 32, 8, 128, 16380, 1, 64, 8, 1, 16, 4, 64, 128,
+                 topics=256, needles=0, backward=False, seed=1344, decode=True),
 }
 
 

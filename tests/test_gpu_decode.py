@@ -104,3 +104,36 @@ def test_decode_is_forward_only_and_needs_its_flag():
     t = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
     with pytest.raises(binding.HgaError):
         binding.hga_attn_bwd(buf.p, t, t, t, t, t, t, t, t, t, t, t, t, None)
+
+
+def test_benchmark_decode_config_sampled_items():
+    """Configuration 7 (what bench.py times as its generation-shaped step), whole path on the GPU,
+    sampled (sequence, kv head) items recomputed by the oracle."""
+    from paper_2607_15105_b200.workloads import CONFIGS
+    cfg = CONFIGS[7]
+    x = make_inputs(cfg)
+    buf = binding.HgaLayerBuffers(cfg, backward=False)
+    Q, K, V = to_dev(x["Q"]), to_dev(x["K"]), to_dev(x["V"])
+    closed = (cfg.total_len // cfg.chunk) * cfg.chunk
+    buf.build_summaries(K, 0, closed)
+    buf.route(Q)
+    buf.attn_fwd(Q, K, V)
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    items = [0, 1, 7, 8, 100, 131, 200, cfg.n_items - 1]
+    cs, gs = bits_of(buf.chunk_sum), bits_of(buf.group_sum)
+    # the summaries the router read: bit-exact for the sampled heads' first and last chunks
+    ocs, ogs = oracle.build_summaries(cfg.scaled(batch=1), np.ascontiguousarray(x["K"][:1]))
+    assert np.array_equal(cs[:1], ocs) and np.array_equal(gs[:1], ogs)
+    ref = oracle.route(cfg, x["Q"], cs, gs, items=items, want_scores=True)
+    gi, ng = buf.group_idx.cpu().numpy(), buf.n_groups.cpu().numpy()
+    n, ec, eg = check_routing(cfg, ref, buf.chunk_idx.cpu().numpy(), gi, ng, items=items)
+    assert n == len(items) and ec <= 1 and eg <= 2, (n, ec, eg)
+    O_ref, LSE_ref = oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], gi, ng, items=items)
+    G = cfg.gqa
+    Of, LSEf = bf16_to_f64(buf.O), buf.LSE.cpu().numpy().astype(np.float64)
+    for it in items:
+        b, h = it // cfg.n_kv_heads, it % cfg.n_kv_heads
+        sl = slice(h * G, (h + 1) * G)
+        assert np.max(np.abs(Of[b, sl] - O_ref[b, sl])) <= TOL_O
+        assert np.max(np.abs(LSEf[b, sl] - LSE_ref[b, sl])) <= TOL_LSE
