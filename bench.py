@@ -285,7 +285,7 @@ def time_decode(args, stream, peaks):
     (O, LSE, index lists) over the measured copy bandwidth."""
     import torch
     from paper_2607_15105_b200 import binding
-    cfg = CONFIGS[7]
+    cfg = CONFIGS[7] if args.decode_batch <= 0 else CONFIGS[7].scaled(batch=args.decode_batch)
     x = make_inputs(cfg)
 
     def dev(a):
@@ -392,6 +392,10 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA-graph replay")
     ap.add_argument("--flags", type=int, default=0, help="hga_params.flags (debugging)")
     ap.add_argument("--no-decode", action="store_true", help="skip the generation-shaped step (configuration 7)")
+    ap.add_argument("--only-decode", action="store_true",
+                    help="run only the generation-shaped step and print its object (profiling captures)")
+    ap.add_argument("--decode-batch", type=int, default=0,
+                    help="sequences in the generation-shaped step (default: configuration 7's 32)")
     ap.add_argument("--no-walk", action="store_true",
                     help="skip the whole-sequence TBPTT walk (every segment of the sequence, one layer)")
     args = ap.parse_args()
@@ -401,6 +405,11 @@ def main():
         return
     if args.warmup < 3:
         args.warmup = 3
+    if args.only_decode:
+        import torch
+        torch.cuda.set_device(0)
+        print(json.dumps({"decode": time_decode(args, torch.cuda.current_stream(), load_peaks())}))
+        return
 
     import torch
     import torch.distributed as dist

@@ -87,6 +87,12 @@ extern "C" {
                                   hga_build_summaries still takes chunk-aligned ranges: call it when a
                                   chunk closes.  Forward only: hga_attn_bwd, hga_step_host and
                                   hga_tbptt_walk return HGA_ERR_UNSUPPORTED with this flag. */
+#define HGA_FLAG_BWD_BF16_GRADS 64 /* hga_attn_bwd / hga_tbptt_walk: dK and dV are written as bf16
+                                  [B,Hkv,S,d] (the dtype of K and V, so the call is a drop-in autograd
+                                  node) instead of fp32.  The sums over query blocks still run in fp32,
+                                  in the workspace (hga_workspace_bytes grows accordingly), and are
+                                  rounded once at the end.  Not with HGA_FLAG_BWD_ACCUMULATE, not in
+                                  hga_step_host (HGA_ERR_UNSUPPORTED). */
 
 /* bits OR-ed into *status_word by the attention kernels */
 #define HGA_STATUS_BAD_INDEX 1     /* a group_idx entry was out of range, inside the sink or
@@ -173,12 +179,13 @@ HGA_API int hga_attn_fwd(const hga_params* p, const void* Q, const void* K, cons
  * earlier segment): writes dQ for all S rows and dK/dV for the
  * S active rows only; history keys contribute to dQ but receive no gradient.
  * O and LSE are hga_attn_fwd's outputs, dO the upstream gradient (layout of O).
- * dK/dV are overwritten unless HGA_FLAG_BWD_ACCUMULATE is set.  The sum over query blocks
+ * dK/dV are fp32 [B,Hkv,S,d] (bf16 with HGA_FLAG_BWD_BF16_GRADS) and are overwritten unless
+ * HGA_FLAG_BWD_ACCUMULATE is set.  The sum over query blocks
  * uses floating-point atomics: results may differ in the last bits from run to run.
  * workspace: device scratch of at least hga_workspace_bytes().bwd bytes. */
 HGA_API int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* V, const void* O,
                  const float* LSE, const void* dO, const int32_t* group_idx,
-                 const int32_t* n_groups, void* dQ, float* dK, float* dV, void* workspace,
+                 const int32_t* n_groups, void* dQ, void* dK, void* dV, void* workspace,
                  size_t workspace_bytes, int32_t* status_word, void* stream);
 
 /* Scratch sizes (bytes) the two calls above need for `p`; either output may be NULL. */
@@ -221,7 +228,7 @@ HGA_API int hga_step_arena_bytes(const hga_params* p, size_t* bytes);
  * `stream` in order. */
 HGA_API int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void* V, const void* dO,
                    void* chunk_sum, void* group_sum, int32_t* chunk_idx, int32_t* group_idx,
-                   int32_t* n_groups, void* O, float* LSE, void* dQ, float* dK, float* dV,
+                   int32_t* n_groups, void* O, float* LSE, void* dQ, void* dK, void* dV,
                    void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
 
 HGA_API const char* hga_status_string(int status);

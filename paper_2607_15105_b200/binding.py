@@ -20,6 +20,7 @@ HGA_FLAG_GLOBAL_GROUP_BUDGET = 4
 HGA_FLAG_SCORE_MEAN = 8
 HGA_FLAG_SCORE_LSE = 16
 HGA_FLAG_DECODE = 32
+HGA_FLAG_BWD_BF16_GRADS = 64
 HGA_STATUS_BAD_INDEX = 1
 HGA_STATUS_WAIT_TIMEOUT = 2
 
@@ -233,8 +234,9 @@ class HgaLayerBuffers:
         self.backward = backward
         if backward:
             self.dQ = torch.zeros(B, Hq, S, d, dtype=bf, device=dev)
-            self.dK = torch.zeros(B, Hkv, S, d, dtype=torch.float32, device=dev)
-            self.dV = torch.zeros(B, Hkv, S, d, dtype=torch.float32, device=dev)
+            gdt = bf if (self.p.flags & HGA_FLAG_BWD_BF16_GRADS) else torch.float32
+            self.dK = torch.zeros(B, Hkv, S, d, dtype=gdt, device=dev)
+            self.dV = torch.zeros(B, Hkv, S, d, dtype=gdt, device=dev)
             self.bwd_ws = torch.empty(bb, dtype=torch.uint8, device=dev)
 
     # the four steps, in path order

@@ -90,9 +90,15 @@ size_t route_workspace_bytes(const Dims& dm) {
   return (size_t)dm.B * dm.Hkv * dm.NQB * per_item * sizeof(float) + 16;
 }
 
+static size_t bwd_delta_bytes(const Dims& dm) {
+  return (((size_t)dm.B * dm.Hq * dm.S * sizeof(float)) + 255) & ~(size_t)255;
+}
+
 size_t bwd_workspace_bytes(const Dims& dm) {
-  // delta = rowsum(dO * O), fp32 [B, Hq, S]
-  return (size_t)dm.B * dm.Hq * dm.S * sizeof(float) + 16;
+  // delta = rowsum(dO * O), fp32 [B, Hq, S]; with bf16 gradient outputs also the fp32 dK and dV sums
+  size_t bytes = bwd_delta_bytes(dm) + 16;
+  if (dm.flags & HGA_FLAG_BWD_BF16_GRADS) bytes += 2 * (size_t)dm.B * dm.Hkv * dm.S * dm.d * sizeof(float);
+  return bytes;
 }
 
 // Copy streams and events of hga_step_host, created once per device and kept until exit.
@@ -216,12 +222,16 @@ int hga_attn_fwd(const hga_params* p, const void* Q, const void* K, const void* 
 
 int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* V, const void* O,
                  const float* LSE, const void* dO, const int32_t* group_idx,
-                 const int32_t* n_groups, void* dQ, float* dK, float* dV, void* workspace,
+                 const int32_t* n_groups, void* dQ, void* dK_out, void* dV_out, void* workspace,
                  size_t workspace_bytes, int32_t* status_word, void* stream) {
   Dims dm;
   int rc = resolve(p, dm);
   if (rc) return rc;
   if (dm.flags & HGA_FLAG_DECODE) return HGA_ERR_UNSUPPORTED;     // forward only
+  const bool bf16_grads = (dm.flags & HGA_FLAG_BWD_BF16_GRADS) != 0;
+  if (bf16_grads && (dm.flags & HGA_FLAG_BWD_ACCUMULATE)) return HGA_ERR_UNSUPPORTED;
+  float* dK = (float*)dK_out;
+  float* dV = (float*)dV_out;
   if (!Q || !K || !V || !O || !LSE || !dO || (!group_idx && dm.width > 0) || !n_groups || !dQ || !dK || !dV)
     return HGA_ERR_NULL;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) ||
@@ -231,21 +241,32 @@ int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* 
   if (!aligned16(workspace)) return HGA_ERR_ALIGN;
   cudaStream_t st = (cudaStream_t)stream;
   const bool zero_grads = !(dm.flags & HGA_FLAG_BWD_ACCUMULATE);
+  const size_t n_kv = (size_t)dm.B * dm.Hkv * dm.S * dm.d;
+  if (bf16_grads) {
+    // the sums over query blocks run in fp32 in the workspace and are rounded once at the end
+    dK = (float*)((char*)workspace + bwd_delta_bytes(dm));
+    dV = dK + n_kv;
+  }
+  rc = HGA_ERR_UNSUPPORTED;
   if (attn_bwd_sm100_supported(dm)) {
     // zero-fills dK/dV itself where its kernels need it; UNSUPPORTED is returned before any launch
     rc = launch_attn_bwd_sm100(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV, (float*)workspace,
                                zero_grads, status_word, st);
-    if (rc != HGA_ERR_UNSUPPORTED) return rc;
   }
-  if (zero_grads) {
-    size_t bytes = (size_t)dm.B * dm.Hkv * dm.S * dm.d * sizeof(float);
-    rc = record_cuda(cudaMemsetAsync(dK, 0, bytes, st));
-    if (rc) return rc;
-    rc = record_cuda(cudaMemsetAsync(dV, 0, bytes, st));
-    if (rc) return rc;
-  }
-  return launch_attn_bwd_generic(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV,
+  if (rc == HGA_ERR_UNSUPPORTED) {
+    if (zero_grads) {
+      rc = record_cuda(cudaMemsetAsync(dK, 0, n_kv * sizeof(float), st));
+      if (rc) return rc;
+      rc = record_cuda(cudaMemsetAsync(dV, 0, n_kv * sizeof(float), st));
+      if (rc) return rc;
+    }
+    rc = launch_attn_bwd_generic(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV,
                                  (float*)workspace, status_word, st);
+  }
+  if (rc || !bf16_grads) return rc;
+  rc = launch_grads_to_bf16(dK, dK_out, n_kv, st);
+  if (rc) return rc;
+  return launch_grads_to_bf16(dV, dV_out, n_kv, st);
 }
 
 int hga_step_arena_bytes(const hga_params* p, size_t* bytes) {
@@ -273,7 +294,7 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   Dims dm;
   int rc = resolve(p, dm);
   if (rc) return rc;
-  if (dm.flags & HGA_FLAG_DECODE) return HGA_ERR_UNSUPPORTED;
+  if (dm.flags & (HGA_FLAG_DECODE | HGA_FLAG_BWD_BF16_GRADS)) return HGA_ERR_UNSUPPORTED;
   if (!Q_host || !Kseg_host || !Vseg_host || !K_dev || !V_dev || !chunk_sum || !group_sum ||
       !O_host || !arena)
     return HGA_ERR_NULL;
@@ -373,7 +394,7 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
 
 int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void* V, const void* dO,
                    void* chunk_sum, void* group_sum, int32_t* chunk_idx, int32_t* group_idx,
-                   int32_t* n_groups, void* O, float* LSE, void* dQ, float* dK, float* dV,
+                   int32_t* n_groups, void* O, float* LSE, void* dQ, void* dK, void* dV,
                    void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream) {
   if (!p) return HGA_ERR_NULL;
   if (p->flags & HGA_FLAG_DECODE) return HGA_ERR_UNSUPPORTED;
@@ -407,6 +428,7 @@ int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void
   fill(ps.v_stride, p->v_stride, p->n_kv_heads);
   const size_t items = (size_t)dmf.B * dmf.Hkv * dmf.NQB;
   const size_t lse_seg = (size_t)dmf.B * dmf.Hq * S, kv_seg = (size_t)dmf.B * dmf.Hkv * S * dmf.d;
+  const size_t grad_bytes = (p->flags & HGA_FLAG_BWD_BF16_GRADS) ? 2 : 4;    // element size of dK/dV
   for (int s = 0; s < n_seg; ++s) {
     ps.total_len = (s + 1) * S;
     const int64_t q_off = (int64_t)s * S * ps.q_stride[2] * 2, o_off = (int64_t)s * S * ps.o_stride[2] * 2;   // bytes
@@ -424,7 +446,8 @@ int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void
     if (rc) return rc;
     if (bwd) {
       rc = hga_attn_bwd(&ps, Qs, K, V, Os, lse, (const char*)dO + o_off, gi, ng, (char*)dQ + q_off,
-                        dK + s * kv_seg, dV + s * kv_seg, (char*)workspace + route_ws_up, bwd_ws, status_word, stream);
+                        (char*)dK + s * kv_seg * grad_bytes, (char*)dV + s * kv_seg * grad_bytes,
+                        (char*)workspace + route_ws_up, bwd_ws, status_word, stream);
       if (rc) return rc;
     }
   }

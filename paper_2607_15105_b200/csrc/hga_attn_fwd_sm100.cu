@@ -238,6 +238,8 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const int r = mt0 * 128 + row_in_tile;              // row inside the item
       const int a = r / bq_pad, t = r % bq_pad;
       const bool real_row = r < rows_pad && t < dm.Bq;
+      // a warp whose 32 lanes are all padding (generation shapes) only keeps the barriers moving
+      const bool warp_real = __any_sync(0xffffffffu, real_row);
       const int limit = n_keys - dm.Bq + t + 1;           // visible key slots (causal inside the block)
       const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
       const uint32_t o_addr = lane_base + kColO;
@@ -248,6 +250,11 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t s_addr = lane_base + (j & 1) * 64;
         ok = __all_sync(0xffffffffu, wait_or_abort(&sm.s_full[j & 1], (j >> 1) & 1, abort));
         if (!ok) break;                                   // warp-uniform
+        if (!warp_real) {
+          // S(j) complete implies that the previous use of this P barrier is over: arriving now is safe
+          mbar_arrive(&sm.p_full[j & 1]);
+          continue;
+        }
         tc_fence_after_sync();
         HGA_TRACE_POINT(11);     // waiting for S
         const int vis = limit - kFT * j;                  // visible columns of this tile (may be <= 0)
@@ -342,7 +349,7 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(&sm.o_done, 0, abort));
       HGA_TRACE_POINT(20);
-      if (ok) {
+      if (ok && warp_real) {
         // every lane takes part in the TMEM loads (warp-wide instructions); only real rows are stored
         tc_fence_after_sync();
         const float inv = 1.f / l_mma;

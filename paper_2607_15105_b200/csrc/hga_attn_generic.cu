@@ -298,6 +298,24 @@ static size_t token_smem_bytes(const Dims& dm) {
   return sizeof(int) * ((size_t)max_routed_tokens(dm) + dm.width + 4);
 }
 
+// dK/dV accumulators (fp32) -> bf16 output, eight elements per thread
+__global__ void __launch_bounds__(256) k_grads_to_bf16(const float4* __restrict__ src, uint4* __restrict__ dst, size_t n8) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n8) return;
+  const float4 a = src[2 * i], b = src[2 * i + 1];
+  const __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x, a.y), h1 = __floats2bfloat162_rn(a.z, a.w);
+  const __nv_bfloat162 h2 = __floats2bfloat162_rn(b.x, b.y), h3 = __floats2bfloat162_rn(b.z, b.w);
+  dst[i] = make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
+                      *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
+}
+
+int launch_grads_to_bf16(const float* src, void* dst, size_t n, cudaStream_t st) {
+  const size_t n8 = n / 8;
+  k_grads_to_bf16<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>((const float4*)src, (uint4*)dst, n8);
+  count_launch();
+  return record_cuda(cudaGetLastError());
+}
+
 int launch_attn_fwd_generic(const Dims& dm, const void* Q, const void* K, const void* V,
                             const int32_t* group_idx, const int32_t* n_groups, void* O, float* LSE,
                             int32_t* status_word, cudaStream_t st) {

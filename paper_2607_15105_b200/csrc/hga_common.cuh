@@ -109,4 +109,7 @@ int resolve_params(const hga_params* p, Dims& dm);
 size_t route_workspace_bytes(const Dims& dm);
 size_t bwd_workspace_bytes(const Dims& dm);
 
+// fp32 -> bf16 (round to nearest even) of n elements, n a multiple of 8 (hga_attn_generic.cu)
+int launch_grads_to_bf16(const float* src, void* dst, size_t n, cudaStream_t st);
+
 }  // namespace hga

@@ -324,3 +324,42 @@ def test_forward_is_deterministic_and_launches_are_counted():
     torch.cuda.synchronize()
     assert binding.hga_kernel_launch_count() - before >= 2 * 4
     assert all(torch.equal(a, b) for a, b in zip(first, (buf.O, buf.LSE, buf.dQ, buf.group_idx)))
+
+
+@pytest.mark.parametrize("flags", FLAG_SETS)
+@pytest.mark.parametrize("name", ["d128_hist", "bq128_c128_g16", "d64_tiny"])
+def test_bf16_gradient_outputs(name, flags):
+    """HGA_FLAG_BWD_BF16_GRADS: dK/dV leave as bf16; the sums still run in fp32, so the result is the
+    fp32 result rounded once (compared with it to bf16 precision, and with the oracle)."""
+    c = get_case(name)
+    cfg = c.cfg
+    outs = {}
+    for extra in (0, binding.HGA_FLAG_BWD_BF16_GRADS):
+        buf = binding.HgaLayerBuffers(cfg, flags=flags | extra)
+        buf.attn_fwd(c.Q, c.K, c.V, c.gi, c.ng)
+        buf.attn_bwd(c.Q, c.K, c.V, c.dO, c.gi, c.ng)
+        torch.cuda.synchronize()
+        assert int(buf.status.item()) == 0
+        outs[extra] = (buf.dQ.clone(), buf.dK.clone(), buf.dV.clone())
+    (dQ32, dK32, dV32), (dQ16, dK16, dV16) = outs[0], outs[binding.HGA_FLAG_BWD_BF16_GRADS]
+    assert dK16.dtype == torch.bfloat16 and dV16.dtype == torch.bfloat16
+    assert torch.equal(dQ32, dQ16)
+    for a32, a16 in ((dK32, dK16), (dV32, dV16)):
+        ref = a32.double()
+        err = (a16.double() - ref).abs()
+        # one rounding to 8 significant bits, plus the run-to-run wobble of the fp32 atomics
+        assert bool((err <= ref.abs() * 2.0 ** -8 + 1e-5).all())
+    x = c.x
+    _, dK_ref, dV_ref = oracle.attn_bwd(cfg, x["Q"], x["K"], x["V"], x["dO"], c.ref["group_idx"], c.ref["n_groups"])
+    assert rel_fro(bf16_to_f64(dK16), dK_ref) <= TOL_GRAD
+    assert rel_fro(bf16_to_f64(dV16), dV_ref) <= TOL_GRAD
+
+
+def test_bf16_gradients_reject_accumulate():
+    cfg = SMALL_CASES["d128_hist"]
+    p = binding.make_params(cfg, flags=binding.HGA_FLAG_BWD_BF16_GRADS | binding.HGA_FLAG_BWD_ACCUMULATE)
+    buf = binding.HgaLayerBuffers(cfg)
+    c = get_case("d128_hist")
+    with pytest.raises(binding.HgaError):
+        binding.hga_attn_bwd(p, c.Q, c.K, c.V, buf.O, buf.LSE, c.dO, c.gi, c.ng, buf.dQ, buf.dK, buf.dV,
+                             torch.empty(1 << 24, dtype=torch.uint8, device="cuda"), buf.status)

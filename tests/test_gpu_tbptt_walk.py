@@ -21,7 +21,7 @@ def seq_cfg(total_len, seg_len, **kw):
     return HgaConfig(**base)
 
 
-@pytest.mark.parametrize("backward", [True, False])
+@pytest.mark.parametrize("backward", [True, False, "bf16_grads"])
 def test_walk_matches_oracle_segment_by_segment(backward):
     L, S = 1536, 512
     n_seg = L // S
@@ -31,7 +31,8 @@ def test_walk_matches_oracle_segment_by_segment(backward):
     cfg = seq_cfg(L, S)                     # the walk's parameters: segments of S tokens
     B, Hq, Hkv, d = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
     nqb, kc, kge = S // cfg.q_block, cfg.topk_chunks, min(cfg.topk_groups, cfg.chunk // cfg.group)
-    p = binding.make_params(cfg)
+    bf16_grads = backward == "bf16_grads"
+    p = binding.make_params(cfg, flags=binding.HGA_FLAG_BWD_BF16_GRADS if bf16_grads else 0)
     dev = "cuda"
     Qd, Kd, Vd, dOd = to_dev(Q), to_dev(K), to_dev(V), to_dev(dO)
     cs = torch.zeros(B, Hkv, L // cfg.chunk, d, dtype=torch.bfloat16, device=dev)
@@ -42,7 +43,7 @@ def test_walk_matches_oracle_segment_by_segment(backward):
     O = torch.zeros(B, Hq, L, d, dtype=torch.bfloat16, device=dev)
     LSE = torch.zeros(n_seg, B, Hq, S, dtype=torch.float32, device=dev)
     dQ = torch.zeros_like(O) if backward else None
-    dK = torch.zeros(n_seg, B, Hkv, S, d, dtype=torch.float32, device=dev) if backward else None
+    dK = torch.zeros(n_seg, B, Hkv, S, d, dtype=torch.bfloat16 if bf16_grads else torch.float32, device=dev) if backward else None
     dV = torch.zeros_like(dK) if backward else None
     r_bytes, b_bytes = binding.hga_workspace_bytes(p)
     ws = torch.empty(r_bytes + b_bytes + 512, dtype=torch.uint8, device=dev)
@@ -76,8 +77,8 @@ def test_walk_matches_oracle_segment_by_segment(backward):
             dOs = np.ascontiguousarray(dO[:, :, s * S:Ls])
             dQ_ref, dK_ref, dV_ref = oracle.attn_bwd(cfg_s, Qs, Ks, Vs, dOs, gi_s, ng_s)
             assert rel_fro(dQf[:, :, s * S:Ls], dQ_ref) <= TOL_GRAD, s
-            assert rel_fro(dK[s].cpu().numpy().astype(np.float64), dK_ref) <= TOL_GRAD, s
-            assert rel_fro(dV[s].cpu().numpy().astype(np.float64), dV_ref) <= TOL_GRAD, s
+            assert rel_fro(dK[s].double().cpu().numpy(), dK_ref) <= TOL_GRAD, s
+            assert rel_fro(dV[s].double().cpu().numpy(), dV_ref) <= TOL_GRAD, s
 
 
 def test_walk_rejects_bad_arguments():
