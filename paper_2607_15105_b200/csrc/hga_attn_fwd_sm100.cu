@@ -140,9 +140,11 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   volatile int* abort = &sm.abort;
   HGA_TRACE_POINT(1);
 
-  if (warp == 0 || warp == 6) {
+  if (warp == 0 || warp == 6 || warp == 7) {
     // ------------------------------------------------------------------ producers: warp 0 K, warp 6 V
-    const bool is_k = warp == 0;
+    // K boxes are split between warps 0 and 7 (a box costs its issuing warp a few hundred cycles)
+    const bool is_k = warp != 6;
+    const int first = warp == 7 ? 4 : 0, count = is_k ? 4 : 8;   // this warp's octets of a tile
     uint64_t* full = is_k ? sm.k_full : sm.v_full;
     // a K stage is free as soon as S of its tile is complete: that is s_full of the same index (the K
     // ring and the S buffers both have two slots), which saves the MMA thread one commit per tile
@@ -157,17 +159,17 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (lane == 0 && use > 0) ok = wait_or_abort(&empty[s], (use - 1) & 1, abort);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
-      if (lane == 0) mbar_arrive_expect_tx(&full[s], kTileBytes);
+      if (lane == 0 && warp != 7) mbar_arrive_expect_tx(&full[s], kTileBytes);
       __syncwarp();
-      if (lane < 8) {
-        const int o = 8 * j + lane;
+      if (lane < count) {
+        const int o = 8 * j + first + lane;
         const int row = o < n_oct ? sm.oct_row[o] : dm.L;   // past the list: out of range -> zeros
-        tma_load_5d(ring + s * kTileBytes + lane * kOctBytes, map, &full[s], 0, row, 0, h, b);
+        tma_load_5d(ring + s * kTileBytes + (first + lane) * kOctBytes, map, &full[s], 0, row, 0, h, b);
       }
       issued = j + 1;
       HGA_TRACE_POINT(2);
     }
-    if (*abort && lane == 0) {
+    if (*abort && lane == 0 && warp != 7) {
       // giving up: let the copies still in flight land before shared memory is released
       if (is_k) mbar_wait(&sm.q_full, 0);
       for (int j = issued > kStages ? issued - kStages : 0; j < issued; ++j)
