@@ -137,3 +137,33 @@ def test_benchmark_decode_config_sampled_items():
         sl = slice(h * G, (h + 1) * G)
         assert np.max(np.abs(Of[b, sl] - O_ref[b, sl])) <= TOL_O
         assert np.max(np.abs(LSEf[b, sl] - LSE_ref[b, sl])) <= TOL_LSE
+
+
+@pytest.mark.parametrize("generic", FLAG_SETS)
+@pytest.mark.parametrize("variant", ["mean+global", "lse", "global"])
+@pytest.mark.parametrize("name", ["five_tokens", "sixteen_tokens", "gqa8"])
+def test_decode_with_routing_variants(name, variant, generic):
+    """The routing variants (score aggregators, one group budget over all opened chunks) combine with
+    the generation shape: routing against the oracle's same combination, attention on the lists taken."""
+    cfg = CASES[name]
+    agg = "mean" if "mean" in variant else "lse" if "lse" in variant else "max"
+    gb = "global" in variant
+    flags = generic | {"mean": binding.HGA_FLAG_SCORE_MEAN, "lse": binding.HGA_FLAG_SCORE_LSE, "max": 0}[agg]
+    flags |= binding.HGA_FLAG_GLOBAL_GROUP_BUDGET if gb else 0
+    x = make_inputs(cfg)
+    cs, gs = oracle.build_summaries(cfg, x["K"])
+    ref = oracle.route(cfg, x["Q"], cs, gs, want_scores=True, score_agg=agg, global_group_budget=gb)
+    buf = binding.HgaLayerBuffers(cfg, backward=False, flags=flags)
+    buf.chunk_sum.copy_(to_dev(cs))
+    buf.group_sum.copy_(to_dev(gs))
+    Q, K, V = to_dev(x["Q"]), to_dev(x["K"]), to_dev(x["V"])
+    buf.route(Q)
+    buf.attn_fwd(Q, K, V)
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    gi, ng = buf.group_idx.cpu().numpy(), buf.n_groups.cpu().numpy()
+    n, ec, eg = check_routing(cfg, ref, buf.chunk_idx.cpu().numpy(), gi, ng, global_budget=gb)
+    assert ec <= max(1, n // 10) and eg <= max(1, n // 5), (n, ec, eg)
+    O_ref, LSE_ref = oracle.attn_fwd(cfg, x["Q"], x["K"], x["V"], gi, ng)
+    assert np.max(np.abs(bf16_to_f64(buf.O) - O_ref)) <= TOL_O
+    assert np.max(np.abs(buf.LSE.cpu().numpy().astype(np.float64) - LSE_ref)) <= TOL_LSE
