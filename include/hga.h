@@ -231,6 +231,34 @@ HGA_API int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, co
                    int32_t* n_groups, void* O, float* LSE, void* dQ, void* dK, void* dV,
                    void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
 
+/* Variable-length batches (packed sequences with prefix sums, the usual "cu_seqlens" convention): one
+ * layer step for n_seq sequences of different lengths that share one set of buffers, tokens packed
+ * back to back, token-major.  Sequence i has S_i = cu_q[i+1] - cu_q[i] active tokens (its queries)
+ * and L_i = cu_k[i+1] - cu_k[i] resident tokens (history H_i = L_i - S_i first), and must obey the
+ * shape rules of hga_params on its own (S_i % Bq == 0, H_i % Bq == 0, L_i % c == 0).
+ *   cu_q, cu_k               HOST int32 [n_seq + 1], non-decreasing, cu[0] = 0
+ *   Q, dO (in), O, dQ (out)  bf16 [sum S_i, Hq, d]         K, V  bf16 [sum L_i, Hkv, d]
+ *   chunk_sum, group_sum     bf16 [Hkv, sum L_i / c, d], [Hkv, sum L_i / g, d]; sequence i's rows start
+ *                            at cu_k[i]/c and cu_k[i]/g; history rows already built, the active range
+ *                            of every sequence is built here
+ *   chunk_idx, group_idx, n_groups   the per-sequence arrays [Hkv, S_i/Bq, ...] of the four calls
+ *                            above, sequence after sequence (sequence i starts at item Hkv * cu_q[i] / Bq)
+ *   LSE fp32                 sequence i's [Hq, S_i] block at element Hq * cu_q[i]
+ *   dK, dV                   sequence i's [Hkv, S_i, d] block at element Hkv * d * cu_q[i]; fp32, or bf16
+ *                            with HGA_FLAG_BWD_BF16_GRADS
+ * p gives the head counts, head_dim, chunk/group/q_block, budgets, windows, scale and flags; its
+ * batch, total_len, seg_len, summary_len and strides are ignored.  dO == NULL runs the forward half
+ * only.  Every sequence runs build_summaries(active range) -> route -> attn_fwd -> attn_bwd as a
+ * batch-1 problem on `stream`, one after the other (host logic only: the kernels are the ones
+ * above).  workspace: device scratch of hga_varlen_workspace_bytes() bytes. */
+HGA_API int hga_varlen_step(const hga_params* p, int32_t n_seq, const int32_t* cu_q, const int32_t* cu_k,
+                    const void* Q, const void* K, const void* V, const void* dO, void* chunk_sum,
+                    void* group_sum, int32_t* chunk_idx, int32_t* group_idx, int32_t* n_groups, void* O,
+                    float* LSE, void* dQ, void* dK, void* dV, void* workspace, size_t workspace_bytes,
+                    int32_t* status_word, void* stream);
+HGA_API int hga_varlen_workspace_bytes(const hga_params* p, int32_t n_seq, const int32_t* cu_q,
+                               const int32_t* cu_k, size_t* bytes);
+
 HGA_API const char* hga_status_string(int status);
 HGA_API int hga_version(void);
 /* the cudaError_t (as int) of the most recent failed CUDA call made by this library */

@@ -9,6 +9,8 @@ from __future__ import annotations
 import ctypes as C
 import os
 
+import numpy as np
+
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -27,7 +29,8 @@ HGA_STATUS_WAIT_TIMEOUT = 2
 HGA_ROUTE_STATIC_SCRATCH_BYTES = 4 << 20
 
 EXPORTS = ("hga_build_summaries", "hga_route", "hga_route_static", "hga_attn_fwd", "hga_attn_bwd",
-           "hga_workspace_bytes", "hga_step_host", "hga_step_arena_bytes", "hga_tbptt_walk", "hga_status_string",
+           "hga_workspace_bytes", "hga_step_host", "hga_step_arena_bytes", "hga_tbptt_walk", "hga_varlen_step",
+           "hga_varlen_workspace_bytes", "hga_status_string",
            "hga_version", "hga_last_cuda_error", "hga_kernel_launch_count")
 
 
@@ -74,6 +77,8 @@ def lib():
         L.hga_step_arena_bytes.argtypes = [pp, C.POINTER(sz)]
         L.hga_step_host.argtypes = [pp] + [vp] * 13 + [sz, vp, vp]
         L.hga_tbptt_walk.argtypes = [pp] + [vp] * 15 + [sz, vp, vp]
+        L.hga_varlen_step.argtypes = [pp, C.c_int32] + [vp] * 17 + [sz, vp, vp]
+        L.hga_varlen_workspace_bytes.argtypes = [pp, C.c_int32, vp, vp, C.POINTER(sz)]
         _lib = L
     return _lib
 
@@ -202,6 +207,31 @@ def hga_tbptt_walk(p, Q, K, V, dO, chunk_sum, group_sum, chunk_idx, group_idx, n
         C.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(chunk_sum), _ptr(group_sum),
         _ptr(chunk_idx), _ptr(group_idx), _ptr(n_groups), _ptr(O), _ptr(LSE), _ptr(dQ), _ptr(dK),
         _ptr(dV), _ptr(workspace), nbytes, _ptr(status_word), _stream(stream)))
+
+
+def _host_i32(a):
+    arr = np.ascontiguousarray(a, dtype=np.int32)
+    return arr, arr.ctypes.data_as(C.c_void_p)
+
+
+def hga_varlen_workspace_bytes(p, cu_q, cu_k) -> int:
+    q, qp = _host_i32(cu_q)
+    k, kp = _host_i32(cu_k)
+    n = C.c_size_t()
+    _check("hga_varlen_workspace_bytes", lib().hga_varlen_workspace_bytes(C.byref(p), len(q) - 1, qp, kp, C.byref(n)))
+    return n.value
+
+
+def hga_varlen_step(p, cu_q, cu_k, Q, K, V, dO, chunk_sum, group_sum, chunk_idx, group_idx, n_groups, O, LSE,
+                    dQ, dK, dV, workspace, status_word=None, stream=None):
+    """One layer step over packed variable-length sequences (cu_q / cu_k are host prefix sums; see hga.h)."""
+    q, qp = _host_i32(cu_q)
+    k, kp = _host_i32(cu_k)
+    nbytes = workspace.numel() * workspace.element_size()
+    _check("hga_varlen_step", lib().hga_varlen_step(
+        C.byref(p), len(q) - 1, qp, kp, _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(chunk_sum), _ptr(group_sum),
+        _ptr(chunk_idx), _ptr(group_idx), _ptr(n_groups), _ptr(O), _ptr(LSE), _ptr(dQ), _ptr(dK), _ptr(dV),
+        _ptr(workspace), nbytes, _ptr(status_word), _stream(stream)))
 
 
 class HgaLayerBuffers:

@@ -1,4 +1,5 @@
 // C-ABI entry points of libhga: argument validation, stride resolution, dispatch.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstring>
@@ -448,6 +449,99 @@ int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void
       rc = hga_attn_bwd(&ps, Qs, K, V, Os, lse, (const char*)dO + o_off, gi, ng, (char*)dQ + q_off,
                         (char*)dK + s * kv_seg * grad_bytes, (char*)dV + s * kv_seg * grad_bytes,
                         (char*)workspace + route_ws_up, bwd_ws, status_word, stream);
+      if (rc) return rc;
+    }
+  }
+  return HGA_OK;
+}
+
+// Batch-1 parameters of sequence i of a packed variable-length batch (token-major tensors).
+static int varlen_params(const hga_params* p, int32_t n_seq, const int32_t* cu_q, const int32_t* cu_k, int i,
+                         hga_params& ps) {
+  const int64_t S = (int64_t)cu_q[i + 1] - cu_q[i], L = (int64_t)cu_k[i + 1] - cu_k[i];
+  const int64_t L_all = cu_k[n_seq];
+  if (S < 1 || L < S || cu_q[i] < 0 || cu_k[i] < 0) return HGA_ERR_SHAPE;
+  if (p->chunk < 1 || p->q_block < 1 || cu_k[i] % p->chunk || cu_q[i] % p->q_block) return HGA_ERR_SHAPE;
+  ps = *p;
+  ps.batch = 1;
+  ps.total_len = (int32_t)L;
+  ps.seg_len = (int32_t)S;
+  ps.summary_len = (int32_t)L_all;
+  const int64_t d = p->head_dim;
+  const int64_t qs[3] = {S * p->n_q_heads * d, d, (int64_t)p->n_q_heads * d};
+  const int64_t ks[3] = {L * p->n_kv_heads * d, d, (int64_t)p->n_kv_heads * d};
+  for (int a = 0; a < 3; ++a) { ps.q_stride[a] = ps.o_stride[a] = qs[a]; ps.k_stride[a] = ps.v_stride[a] = ks[a]; }
+  return HGA_OK;
+}
+
+int hga_varlen_workspace_bytes(const hga_params* p, int32_t n_seq, const int32_t* cu_q, const int32_t* cu_k,
+                               size_t* bytes) {
+  if (!p || !cu_q || !cu_k || !bytes) return HGA_ERR_NULL;
+  if (n_seq < 1 || cu_q[0] != 0 || cu_k[0] != 0) return HGA_ERR_SHAPE;
+  if (p->flags & HGA_FLAG_DECODE) return HGA_ERR_UNSUPPORTED;
+  size_t route_max = 0, bwd_max = 0;
+  for (int i = 0; i < n_seq; ++i) {
+    hga_params ps;
+    int rc = varlen_params(p, n_seq, cu_q, cu_k, i, ps);
+    if (rc) return rc;
+    Dims dm;
+    rc = resolve(&ps, dm);
+    if (rc) return rc;
+    route_max = std::max(route_max, route_workspace_bytes(dm));
+    bwd_max = std::max(bwd_max, bwd_workspace_bytes(dm));
+  }
+  *bytes = ((route_max + 255) & ~(size_t)255) + bwd_max;
+  return HGA_OK;
+}
+
+int hga_varlen_step(const hga_params* p, int32_t n_seq, const int32_t* cu_q, const int32_t* cu_k,
+                    const void* Q, const void* K, const void* V, const void* dO, void* chunk_sum,
+                    void* group_sum, int32_t* chunk_idx, int32_t* group_idx, int32_t* n_groups, void* O,
+                    float* LSE, void* dQ, void* dK, void* dV, void* workspace, size_t workspace_bytes,
+                    int32_t* status_word, void* stream) {
+  size_t need = 0;
+  int rc = hga_varlen_workspace_bytes(p, n_seq, cu_q, cu_k, &need);     // validates every sequence
+  if (rc) return rc;
+  if (!Q || !K || !V || !chunk_sum || !group_sum || !group_idx || !n_groups || !O || !LSE || !workspace)
+    return HGA_ERR_NULL;
+  if (p->topk_chunks > 0 && !chunk_idx) return HGA_ERR_NULL;
+  const bool bwd = dO != nullptr;
+  if (bwd && (!dQ || !dK || !dV)) return HGA_ERR_NULL;
+  if (workspace_bytes < need) return HGA_ERR_WORKSPACE;
+  const int64_t d = p->head_dim, Hq = p->n_q_heads, Hkv = p->n_kv_heads;
+  const int per = p->chunk / p->group;
+  const int kge = p->topk_groups < per ? p->topk_groups : per;
+  const size_t grad_bytes = (p->flags & HGA_FLAG_BWD_BF16_GRADS) ? 2 : 4;
+  for (int i = 0; i < n_seq; ++i) {
+    hga_params ps;
+    varlen_params(p, n_seq, cu_q, cu_k, i, ps);
+    Dims dm;
+    rc = resolve(&ps, dm);
+    if (rc) return rc;
+    const int64_t q0 = cu_q[i], k0 = cu_k[i];
+    const char* Qi = (const char*)Q + q0 * Hq * d * 2;
+    const char* Ki = (const char*)K + k0 * Hkv * d * 2;
+    const char* Vi = (const char*)V + k0 * Hkv * d * 2;
+    char* Oi = (char*)O + q0 * Hq * d * 2;
+    char* csi = (char*)chunk_sum + (k0 / p->chunk) * d * 2;
+    char* gsi = (char*)group_sum + (k0 / p->group) * d * 2;
+    const int64_t item0 = Hkv * (q0 / p->q_block);
+    int32_t* ci = chunk_idx ? chunk_idx + item0 * p->topk_chunks : nullptr;
+    int32_t* gi = group_idx + item0 * p->topk_chunks * kge;
+    int32_t* ng = n_groups + item0;
+    float* lse = LSE + Hq * q0;
+    const size_t route_ws = route_workspace_bytes(dm), bwd_ws = bwd_workspace_bytes(dm);
+    rc = hga_build_summaries(&ps, Ki, dm.H, dm.L, csi, gsi, stream);
+    if (rc) return rc;
+    rc = hga_route(&ps, Qi, csi, gsi, ci, gi, ng, nullptr, nullptr, workspace, route_ws, stream);
+    if (rc) return rc;
+    rc = hga_attn_fwd(&ps, Qi, Ki, Vi, gi, ng, Oi, lse, status_word, stream);
+    if (rc) return rc;
+    if (bwd) {
+      rc = hga_attn_bwd(&ps, Qi, Ki, Vi, Oi, lse, (const char*)dO + q0 * Hq * d * 2, gi, ng,
+                        (char*)dQ + q0 * Hq * d * 2, (char*)dK + Hkv * d * q0 * grad_bytes,
+                        (char*)dV + Hkv * d * q0 * grad_bytes,
+                        (char*)workspace + ((route_ws + 255) & ~(size_t)255), bwd_ws, status_word, stream);
       if (rc) return rc;
     }
   }
