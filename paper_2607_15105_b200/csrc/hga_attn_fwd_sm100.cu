@@ -13,7 +13,7 @@
 //
 // Warp roles (256 threads; warps are allocated in fours, and two CTAs of 8 warps leave 128
 // registers per thread):
-//   warp 0      octet table, Q load, K tile ring          warp 6   V tile ring
+//   warp 0      octet table, Q load, K tile ring (boxes 0-3 of a tile; warp 7: boxes 4-7)    warp 6   V tile ring
 //   warp 1      MMA issuer (one thread): S = Q K^T (smem x smem), O += P V (P from TMEM)
 //   warps 2-5   softmax, one thread per row (thread owns TMEM lane = row), then the epilogue
 // K and V have independent producers: K(j+2) is wanted as soon as S(j) has been issued, V(j+1)
@@ -141,7 +141,7 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   HGA_TRACE_POINT(1);
 
   if (warp == 0 || warp == 6 || warp == 7) {
-    // ------------------------------------------------------------------ producers: warp 0 K, warp 6 V
+    // ------------------------------------------------------------------ producers: warps 0 and 7 K, warp 6 V
     // K boxes are split between warps 0 and 7 (a box costs its issuing warp a few hundred cycles)
     const bool is_k = warp != 6;
     const int first = warp == 7 ? 4 : 0, count = is_k ? 4 : 8;   // this warp's octets of a tile
