@@ -75,6 +75,9 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
   while (qb_own + n_qb < dm.NQB && window_of(dm, qb_own + n_qb).ls <= k0) ++n_qb;
   const int n_mt = dm.rows / 128;
   const int n_steps = n_qb * n_mt;
+  // the sweep that follows in the stream may start on SMs this grid leaves idle (it waits for this grid
+  // only before it adds to dK/dV)
+  pdl_launch_dependents();
 
   if (tid == 0) {
     mbar_init(&sm.kv_full, 1);

@@ -583,6 +583,10 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     float* dKb = dK + ((int64_t)(b * dm.Hkv + h) * dm.S) * D + e;
     float* dVb = dV + ((int64_t)(b * dm.Hkv + h) * dm.S) * D + e;
     bool ok = true;
+    // The band kernel, which precedes this one in the stream, stores its dK/dV rows plainly: the adds
+    // below must come after it.  Nothing else in this kernel depends on it, so this is the only wait
+    // (a no-op unless the launch carried the programmatic-serialization attribute).
+    if (n_act > 0) pdl_wait();
     for (int s = 0; s < n_act; ++s) {
       const int j = tile_of_step(s);
       ok = __all_sync(0xffffffffu, bwd_wait(&sm.dkv_full, s & 1, abort));
@@ -713,10 +717,22 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
     if ((e = cudaMemsetAsync(dV, 0, bytes, st)) != cudaSuccess) return record_cuda(e);
   }
   const int units = dm.B * dm.Hkv * dm.NQB * (dm.rows / 128);
-  k_attn_bwd_sm100<<<units, kBwdThreads, smem, st>>>(mq, mdo, mk, mv, mdq, delta_ws, LSE, group_idx, n_groups, dm,
-                                                    dK, dV, band_done, status_word);
+  // After the band kernel the sweep is launched with programmatic serialization: its CTAs may start on
+  // SMs the band kernel's last wave leaves idle (they wait for it only before adding to dK/dV).
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)units);
+  cfg.blockDim = dim3(kBwdThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = band_done ? 1 : 0;
+  e = cudaLaunchKernelEx(&cfg, k_attn_bwd_sm100, mq, mdo, mk, mv, mdq, (const float*)delta_ws, LSE, group_idx, n_groups,
+                         dm, dK, dV, band_done, status_word);
   count_launch(2);
-  return record_cuda(cudaGetLastError());
+  return record_cuda(e);
 }
 
 }  // namespace hga

@@ -87,6 +87,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   return mbar_wait_bounded(bar, parity, nullptr);
 }
 
+// ----------------------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-serialization attribute may start while its predecessor in the
+// stream is still running; it must execute pdl_wait() before touching anything the predecessor writes.
+// The predecessor lets it start early by executing pdl_launch_dependents() in every CTA.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ----------------------------------------------------------------------------- proxies / fences
 
 __device__ __forceinline__ void fence_proxy_async_smem() {
