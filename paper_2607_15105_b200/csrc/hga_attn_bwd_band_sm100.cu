@@ -75,9 +75,6 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
   while (qb_own + n_qb < dm.NQB && window_of(dm, qb_own + n_qb).ls <= k0) ++n_qb;
   const int n_mt = dm.rows / 128;
   const int n_steps = n_qb * n_mt;
-  // the sweep that follows in the stream may start on SMs this grid leaves idle (it waits for this grid
-  // only before it adds to dK/dV)
-  pdl_launch_dependents();
 
   if (tid == 0) {
     mbar_init(&sm.kv_full, 1);
@@ -231,6 +228,13 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
     };
     float lse = 0.f, dl = 0.f;
     int vis = 0;
+    // This kernel is launched with programmatic serialization behind the delta pre-pass: everything up to
+    // here (set-up, the K/V tile and the first Q/dO tiles, which are inputs of the call) may have run
+    // while that kernel was still busy; delta is read from here on.  Only then is the sweep, which follows
+    // in the stream and reads delta too, allowed to start on the SMs this grid leaves idle (it waits for
+    // this grid itself only before it adds to dK/dV).
+    pdl_wait();
+    if (warp == 2 && lane == 0) pdl_launch_dependents();
     if (wg < n_steps) row_of(wg, lse, dl, vis);
     bool ok = true;
     for (int m = wg; m < n_steps; m += 2) {
@@ -347,9 +351,19 @@ int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, con
   cudaError_t e = cudaFuncSetAttribute(k_attn_bwd_band_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return record_cuda(e);
   const int units = dm.B * dm.Hkv * (dm.S / kKT);
-  k_attn_bwd_band_sm100<<<units, kBandThreads, smem, st>>>(mq, mdo, mk, mv, delta_ws, LSE, dm, dK, dV, status_word);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)units);
+  cfg.blockDim = dim3(kBandThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;   // behind the delta pre-pass of the same call
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, k_attn_bwd_band_sm100, mq, mdo, mk, mv, delta_ws, LSE, dm, dK, dV, status_word);
   count_launch(1);
-  return record_cuda(cudaGetLastError());
+  return record_cuda(e);
 }
 
 }  // namespace hga

@@ -641,6 +641,7 @@ k_bwd_delta_sm100(const uint16_t* __restrict__ O, const uint16_t* __restrict__ d
   const int64_t n_rows = (int64_t)dm.B * dm.Hq * dm.S;
   const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  pdl_launch_dependents();      // the band kernel behind this one may set itself up meanwhile (it waits before reading delta)
   for (int64_t base = warp_id * 8; base < n_rows; base += n_warps * 8) {
     uint4 x[4], y[4];
 #pragma unroll
