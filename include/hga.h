@@ -224,8 +224,11 @@ HGA_API int hga_step_arena_bytes(const hga_params* p, size_t* bytes);
  *   LSE fp32 [L/S,B,Hq,S]    dK, dV fp32 [L/S,B,Hkv,S,d] (segment s holds the rows of its own tokens)
  * dO == NULL runs the forward half only (dQ, dK, dV may then be NULL).  p->summary_len is
  * ignored (the summary buffers are laid out for L).  workspace: device scratch of at least
- * route_bytes + bwd_bytes as hga_workspace_bytes(p) reports them.  All work is queued on
- * `stream` in order. */
+ * route_bytes + bwd_bytes as hga_workspace_bytes(p) reports them.  The forward chain of every
+ * segment is queued on `stream`; the backward calls (each depends only on its own segment's forward)
+ * are queued on a second stream the library creates once per device, which starts after the work
+ * already queued on `stream` and is joined back into `stream` before the call returns, so later work
+ * on `stream` sees every result.  The call itself never synchronises. */
 HGA_API int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void* V, const void* dO,
                    void* chunk_sum, void* group_sum, int32_t* chunk_idx, int32_t* group_idx,
                    int32_t* n_groups, void* O, float* LSE, void* dQ, void* dK, void* dV,

@@ -430,6 +430,19 @@ int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void
   const size_t items = (size_t)dmf.B * dmf.Hkv * dmf.NQB;
   const size_t lse_seg = (size_t)dmf.B * dmf.Hq * S, kv_seg = (size_t)dmf.B * dmf.Hkv * S * dmf.d;
   const size_t grad_bytes = (p->flags & HGA_FLAG_BWD_BF16_GRADS) ? 2 : 4;    // element size of dK/dV
+  // The backward of segment s depends on that segment's forward only, and the forward chain of segment
+  // s+1 (summaries -> route -> forward) on nothing the backward writes: the backward calls go to a
+  // second, library-owned stream (the one hga_step_host copies in on), so the two chains fill each
+  // other's idle SMs (kernel tails, the one-wave router).  The caller's stream is joined at the end.
+  cudaStream_t st = (cudaStream_t)stream;
+  StepPipe* pipe = bwd ? step_pipe(n_seg) : nullptr;
+  if (bwd && !pipe) return HGA_ERR_CUDA;
+  if (bwd) {
+    rc = record_cuda(cudaEventRecord(pipe->fork, st));
+    if (rc) return rc;
+    rc = record_cuda(cudaStreamWaitEvent(pipe->in, pipe->fork, 0));
+    if (rc) return rc;
+  }
   for (int s = 0; s < n_seg; ++s) {
     ps.total_len = (s + 1) * S;
     const int64_t q_off = (int64_t)s * S * ps.q_stride[2] * 2, o_off = (int64_t)s * S * ps.o_stride[2] * 2;   // bytes
@@ -446,11 +459,21 @@ int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, const void
     rc = hga_attn_fwd(&ps, Qs, K, V, gi, ng, Os, lse, status_word, stream);
     if (rc) return rc;
     if (bwd) {
+      rc = record_cuda(cudaEventRecord(pipe->in_done[s], st));          // forward of segment s queued
+      if (rc) return rc;
+      rc = record_cuda(cudaStreamWaitEvent(pipe->in, pipe->in_done[s], 0));
+      if (rc) return rc;
       rc = hga_attn_bwd(&ps, Qs, K, V, Os, lse, (const char*)dO + o_off, gi, ng, (char*)dQ + q_off,
                         (char*)dK + s * kv_seg * grad_bytes, (char*)dV + s * kv_seg * grad_bytes,
-                        (char*)workspace + route_ws_up, bwd_ws, status_word, stream);
+                        (char*)workspace + route_ws_up, bwd_ws, status_word, pipe->in);
       if (rc) return rc;
     }
+  }
+  if (bwd) {
+    rc = record_cuda(cudaEventRecord(pipe->join, pipe->in));
+    if (rc) return rc;
+    rc = record_cuda(cudaStreamWaitEvent(st, pipe->join, 0));
+    if (rc) return rc;
   }
   return HGA_OK;
 }
