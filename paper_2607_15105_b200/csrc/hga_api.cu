@@ -49,6 +49,7 @@ static int resolve(const hga_params* p, Dims& dm) {
   if (p->chunk / p->group > 64) return HGA_ERR_UNSUPPORTED;
   if (p->topk_chunks > 1024) return HGA_ERR_UNSUPPORTED;
   if ((p->flags & HGA_FLAG_SCORE_MEAN) && (p->flags & HGA_FLAG_SCORE_LSE)) return HGA_ERR_UNSUPPORTED;
+  if (p->flags & ~0x7f & ~kFlagNoPdl) return HGA_ERR_UNSUPPORTED;      // unknown flag bits
   if ((p->flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) && (int64_t)p->topk_chunks * (p->chunk / p->group) > 4096)
     return HGA_ERR_UNSUPPORTED;
   dm.B = p->batch; dm.Hq = p->n_q_heads; dm.Hkv = p->n_kv_heads; dm.G = dm.Hq / dm.Hkv;
@@ -340,6 +341,7 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   pc.batch = 1;
   pc.n_q_heads = dm.G;
   pc.n_kv_heads = 1;
+  pc.flags |= kFlagNoPdl;                            // this pipeline is bound by the host link (see hga_common.cuh)
   const size_t q_c = (size_t)dm.G * dm.S * dm.d * 2;           // bytes of one pair's Q / dO / O / dQ rows
   const size_t kvseg_c = (size_t)dm.S * dm.d * 2, kv32_c = (size_t)dm.S * dm.d * 4;
   const size_t kv_c = (size_t)dm.L * dm.d * 2;                 // one (batch, kv head) of the resident K / V

@@ -360,7 +360,7 @@ int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, con
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;   // behind the delta pre-pass of the same call
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = (dm.flags & kFlagNoPdl) ? 0 : 1;
   e = cudaLaunchKernelEx(&cfg, k_attn_bwd_band_sm100, mq, mdo, mk, mv, delta_ws, LSE, dm, dK, dV, status_word);
   count_launch(1);
   return record_cuda(e);

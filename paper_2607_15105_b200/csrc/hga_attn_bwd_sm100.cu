@@ -729,7 +729,7 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
-  cfg.numAttrs = band_done ? 1 : 0;
+  cfg.numAttrs = (band_done && !(dm.flags & kFlagNoPdl)) ? 1 : 0;
   e = cudaLaunchKernelEx(&cfg, k_attn_bwd_sm100, mq, mdo, mk, mv, mdq, (const float*)delta_ws, LSE, group_idx, n_groups,
                          dm, dK, dV, band_done, status_word);
   count_launch(2);

@@ -14,6 +14,11 @@ __host__ __device__ inline int score_agg_of(int flags) {
   return (flags & HGA_FLAG_SCORE_MEAN) ? 1 : (flags & HGA_FLAG_SCORE_LSE) ? 2 : 0;
 }
 
+// Internal flag (a bit of hga_params.flags that hga.h does not define): launch the backward's kernels
+// without programmatic serialization.  Set by hga_step_host, whose steps are bound by the host link: there
+// the early-started CTAs only get in the way of the next (batch, kv head) pair's kernels.
+constexpr int kFlagNoPdl = 1 << 30;
+
 // Resolved problem description handed to kernels by value.
 struct Dims {
   int B, Hq, Hkv, G, d;
