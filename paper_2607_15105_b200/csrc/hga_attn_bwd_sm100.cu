@@ -126,27 +126,29 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     sm.abort = 0;
     fence_barrier_init();
   }
+  if (warp < 8) {
+    // Q and dO do not depend on the routing: their copies start first, one box per warp (issuing a box
+    // costs its warp a few hundred cycles; eight warps issue in parallel).  Barrier 2 makes the mbarrier
+    // initialisation above visible to the eight issuing warps.
+    asm volatile("bar.sync 2, 256;" ::: "memory");
+    if (lane == 0) {
+      if (warp == 0) mbar_arrive_expect_tx(&sm.q_full, 2 * 128 * kBwdD * 2);
+      // four boxes of 64 rows x one 64-element panel per tensor, laid out [panel][128 rows][128 B]
+      const int half = warp & 1, panel = (warp >> 1) & 1;
+      const int r = mt * 128 + 64 * half;
+      const int a = r / dm.Bq, t = r % dm.Bq;
+      const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
+      if (warp < 4) tma_load_5d(sm.q + off, &map_q, &sm.q_full, 0, qb * dm.Bq + t, panel, h * dm.G + a, b);
+      else tma_load_5d(sm.dO + off, &map_do, &sm.q_full, 0, qb * dm.Bq + t, panel, h * dm.G + a, b);
+    }
+    __syncwarp();
+  }
   if (warp == 1) {
     tmem_alloc(&sm.tmem_base, 512);
     tmem_relinquish();
   }
   if (warp == 0) {
-    // Q and dO do not depend on the routing: start their copies first
-    if (lane == 0) {
-      prefetch_tensormap(&map_q); prefetch_tensormap(&map_do);
-      prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
-      mbar_arrive_expect_tx(&sm.q_full, 2 * 128 * kBwdD * 2);
-    }
-    __syncwarp();
-    if (lane < 8) {
-      // four boxes of 64 rows x one 64-element panel per tensor, laid out [panel][128 rows][128 B]
-      const int half = lane & 1, panel = (lane >> 1) & 1;
-      const int r = mt * 128 + 64 * half;
-      const int a = r / dm.Bq, t = r % dm.Bq;
-      const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
-      if (lane < 4) tma_load_5d(sm.q + off, &map_q, &sm.q_full, 0, qb * dm.Bq + t, panel, h * dm.G + a, b);
-      else tma_load_5d(sm.dO + off, &map_do, &sm.q_full, 0, qb * dm.Bq + t, panel, h * dm.G + a, b);
-    }
+    if (lane == 0) { prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); }
     bool bad;   // invalid entries are skipped exactly as in the forward kernel (which reports them)
     const int n_oct = build_octet_table(dm, w, group_idx + (int64_t)item * dm.width, n_groups + item, sm.oct_row, &bad);
     // Keys that receive dK/dV from this kernel: positions in [H, hi), where hi is the start of the
