@@ -90,3 +90,55 @@ def test_workspace_sizes(lib):
         assert r >= cfg.n_items * (cfg.total_len // cfg.chunk) * 4
         assert b >= cfg.batch * cfg.n_q_heads * cfg.seg_len * 4
         assert binding.hga_step_arena_bytes(binding.make_params(cfg)) > r + b
+
+
+def _ws(lib, p):
+    r, b = C.c_size_t(), C.c_size_t()
+    rc = lib.hga_workspace_bytes(C.byref(p), C.byref(r), C.byref(b))
+    return rc, r.value, b.value
+
+
+def test_flag_rules_on_the_host(lib):
+    """Variant flags are validated before anything touches the device."""
+    from dataclasses import replace
+    cfg = CONFIGS[1]
+    ok = lambda flags, c=cfg: _ws(lib, binding.make_params(c, flags=flags))[0]
+    assert ok(0) == 0
+    assert ok(binding.HGA_FLAG_SCORE_MEAN) == 0 and ok(binding.HGA_FLAG_SCORE_LSE) == 0
+    assert ok(binding.HGA_FLAG_SCORE_MEAN | binding.HGA_FLAG_SCORE_LSE) == -4      # at most one aggregator
+    assert ok(1 << 9) == -4                                                          # unknown flag bit
+    # generation shapes need their flag: q_block below the chunk, unaligned history and length
+    dec = replace(cfg, total_len=1003, seg_len=3, q_block=3)
+    assert ok(0, dec) == -2
+    assert ok(binding.HGA_FLAG_DECODE, dec) == 0
+    # the global group budget keeps one bit per (opened chunk, group) slot: at most 4096
+    big = replace(cfg, chunk=64, group=1, topk_chunks=65, total_len=8192, seg_len=512)
+    assert ok(0, big) == 0 and ok(binding.HGA_FLAG_GLOBAL_GROUP_BUDGET, big) == -4
+
+
+def test_workspace_sizes_follow_their_formulas(lib):
+    cfg = CONFIGS[3]
+    items = cfg.batch * cfg.n_kv_heads * cfg.n_q_blocks
+    rc, r, b = _ws(lib, binding.make_params(cfg))
+    assert rc == 0
+    assert r == items * (cfg.total_len // cfg.chunk) * 4 + 16
+    delta = cfg.batch * cfg.n_q_heads * cfg.seg_len * 4
+    assert b == ((delta + 255) & ~255) + 16
+    # global group budget: the opened chunks' group scores behind the chunk scores
+    rc, r2, _ = _ws(lib, binding.make_params(cfg, flags=binding.HGA_FLAG_GLOBAL_GROUP_BUDGET))
+    assert rc == 0 and r2 == r + items * cfg.topk_chunks * (cfg.chunk // cfg.group) * 4
+    # bf16 gradient outputs: the fp32 dK and dV sums live in the workspace
+    rc, _, b2 = _ws(lib, binding.make_params(cfg, flags=binding.HGA_FLAG_BWD_BF16_GRADS))
+    assert rc == 0 and b2 == b + 2 * cfg.batch * cfg.n_kv_heads * cfg.seg_len * cfg.head_dim * 4
+
+
+def test_varlen_prefix_sums_are_validated_on_the_host(lib):
+    cfg = CONFIGS[1]
+    p = binding.make_params(cfg)
+    assert binding.hga_varlen_workspace_bytes(p, [0, 256, 512], [0, 1024, 1536]) > 0
+    for cu_q, cu_k in (([0, 256], [0, 1000]),            # length not a multiple of the chunk
+                       ([0, 256, 768], [0, 1024, 1280]),  # more queries than keys in the second sequence
+                       ([64, 320], [0, 1024]),            # does not start at zero
+                       ([0, 100], [0, 1024])):            # segment not a multiple of the query block
+        with pytest.raises(binding.HgaError):
+            binding.hga_varlen_workspace_bytes(p, cu_q, cu_k)
