@@ -136,7 +136,10 @@ HGA_API int hga_build_summaries(const hga_params* p, const void* K, int32_t tok_
  * group_scores (optional, may be NULL) fp32 [B,Hkv,NQB,k_c*(c/g)]: slot (r,u) = group u
  *   of the r-th selected chunk, -inf where unused.
  * workspace: device scratch of at least hga_workspace_bytes().route bytes (16-byte
- *   aligned); contents are overwritten.  Calls that share a workspace must not overlap. */
+ *   aligned); contents are overwritten.  Calls that share a workspace must not overlap. 
+ * An item whose routing could not be completed (a bounded on-chip wait gave up: never in normal
+ * operation) gets n_groups = -1; the attention calls then attend to its sink and local window only
+ * and report HGA_STATUS_BAD_INDEX. */
 HGA_API int hga_route(const hga_params* p, const void* Q, const void* chunk_sum, const void* group_sum,
               int32_t* chunk_idx, int32_t* group_idx, int32_t* n_groups, float* chunk_scores,
               float* group_scores, void* workspace, size_t workspace_bytes, void* stream);

@@ -100,8 +100,10 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   for (int i = 0; i < 32; ++i) col_mask |= (uint32_t)((i % bq_pad) < dm.Bq) << i;
 
   // Copies one 128-row summary tile (16 octet boxes, one per lane) into its ring stage; all lanes of warp 0.
+  int tiles_issued = 0;                 // warp 0's count of summary tiles whose copies were started
   auto issue_tile = [&](int tg, int t, bool phase2) {
     const int s = tg % STAGES;
+    tiles_issued = tg + 1;
     if (lane == 0) mbar_arrive_expect_tx(&sm.a_full[s], Smem::kTile);
     __syncwarp();
     if (lane < 16) {
@@ -170,6 +172,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       // ---------------------------------------------------------------- producer
       bool ok = true;
       if (phase2) {
+        tiles_issued = t_begin + 1;        // (its boxes come from the other warps, see above)
         if (lane == 0) mbar_arrive_expect_tx(&sm.a_full[t_begin % STAGES], Smem::kTile);
         HGA_RT_STAMP(3 + t_begin);
       }
@@ -446,6 +449,17 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   }
 
   HGA_RT_STAMP(23);
+  if (sm.abort) {
+    // A bounded wait gave up: the item's routing is marked invalid (the attention calls report a negative
+    // count and use no routed groups for that item), and the copies still in flight get a bounded time to land
+    // before the CTA's shared memory is released.
+    if (tid == 0) n_groups[item] = -1;
+    if (warp == 0 && lane == 0) {
+      if (k_sel > 0) mbar_wait(&sm.q_full, 0);
+      for (int tg = tiles_issued > STAGES ? tiles_issued - STAGES : 0; tg < tiles_issued; ++tg)
+        mbar_wait(&sm.a_full[tg % STAGES], (tg / STAGES) & 1);
+    }
+  }
   __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
