@@ -149,16 +149,24 @@ HGA_API int hga_route(const hga_params* p, const void* Q, const void* chunk_sum,
  * memory at all -- code that runs while its host framework's allocator is locked or has
  * claimed the whole device, loops that must never enter cudaMalloc because it synchronises
  * the device, processes whose device memory is budgeted at start-up.  The scratch hga_route
- * would take from `workspace` lives in a fixed array inside the library image instead, so
- * every GPU that loads the library holds HGA_ROUTE_STATIC_SCRATCH_BYTES of device memory
- * until the process exits, and the call itself allocates and frees nothing.
- *   - Same inputs, outputs and selection rule as hga_route (no optional score outputs).
- *   - Size limit: hga_workspace_bytes().route must not exceed HGA_ROUTE_STATIC_SCRATCH_BYTES
- *     (batch * n_kv_heads * (seg_len / q_block) * (total_len / chunk) * 4 bytes + 16); a larger
- *     problem returns HGA_ERR_WORKSPACE and launches nothing.  All five benchmark
+ * would take from `workspace` lives in a fixed array inside the library image instead
+ * (HGA_ROUTE_STATIC_SCRATCH_BYTES per GPU, held until the process exits), and the call itself
+ * calls no allocating or freeing routine.
+ *   - Same inputs, outputs and selection rule as hga_route (no optional score outputs), and the
+ *     same kernels: the fused tensor-core router where the shape qualifies (it keeps the scores
+ *     on chip and leaves the array untouched), else the CUDA-core router, whose chunk scores go
+ *     to the array.
+ *   - Size limit: hga_workspace_bytes().route must not exceed HGA_ROUTE_STATIC_SCRATCH_BYTES.
+ *     That is batch * n_kv_heads * (seg_len / q_block) * per_item * 4 bytes + 16 with
+ *     per_item = total_len / chunk, plus k_c * (chunk / group) with HGA_FLAG_GLOBAL_GROUP_BUDGET.
+ *     A larger problem returns HGA_ERR_WORKSPACE and launches nothing.  All five benchmark
  *     configurations fit.
- *   - The first call on each device looks up the array's device address; make that first call
- *     outside any stream capture.  Later calls on the same device do no set-up.
+ *   - The FIRST call on each device looks up the array's device address.  CUDA loads a module's
+ *     device data lazily, so it is this look-up that makes the driver place the array in device
+ *     memory: make that first call at start-up, while device memory is still available and
+ *     outside any stream capture (on a device with no memory left it returns HGA_ERR_CUDA).
+ *     Later calls on the same device do no set-up and leave the amount of free device memory
+ *     unchanged.
  *   - All calls on a device share the one array and it keeps the last call's contents (the
  *     kernels overwrite what they read, nothing needs clearing).  Two calls that overlap on
  *     the GPU (different streams, no ordering between them) race on it: order them. */
@@ -271,6 +279,33 @@ HGA_API int hga_version(void);
 HGA_API int hga_last_cuda_error(void);
 /* number of kernels this library has launched since it was loaded (all calls, all streams) */
 HGA_API int64_t hga_kernel_launch_count(void);
+
+/* The same count per kernel family, so that a caller (or a test) can tell which implementation a
+ * call took: every step has a tensor-core kernel (tcgen05 / TMEM / TMA) for the shapes that qualify
+ * and a shape-generic CUDA-core kernel for the rest (and for HGA_FLAG_GENERIC_KERNELS).
+ * An unknown family returns -1. */
+#define HGA_KERNELS_SUMMARIES 0      /* hga_build_summaries */
+#define HGA_KERNELS_ROUTE_TENSOR 1   /* hga_route, fused tensor-core router */
+#define HGA_KERNELS_ROUTE_GENERIC 2  /* hga_route / hga_route_static, CUDA-core router (three launches) */
+#define HGA_KERNELS_FWD_TENSOR 3     /* hga_attn_fwd, tensor-core kernel */
+#define HGA_KERNELS_FWD_GENERIC 4    /* hga_attn_fwd, one warp per query row */
+#define HGA_KERNELS_BWD_TENSOR 5     /* hga_attn_bwd, tensor-core kernels (local band + routed sweep, and
+                                        the delta pre-pass where one is launched) */
+#define HGA_KERNELS_BWD_GENERIC 6    /* hga_attn_bwd, CUDA-core kernels (delta, dQ, dK/dV) */
+#define HGA_KERNELS_AUX 7            /* conversions (bf16 gradient outputs) and the self-test kernel */
+#define HGA_KERNELS_FAMILIES 8
+HGA_API int64_t hga_kernel_launch_count_by_family(int family);
+
+/* Self-test of the bounded on-chip waits (no counterpart in the paper).  Every wait on an mbarrier
+ * inside the tensor-core kernels is a poll loop with a time limit; a wait that runs out makes its CTA
+ * leave cleanly and OR-s HGA_STATUS_WAIT_TIMEOUT into the status word instead of hanging the GPU.
+ * This call launches one tiny kernel (one CTA, no TMA, no tensor memory) that waits with a limit of
+ * `cycle_limit` SM cycles (1 <= cycle_limit <= 2^24) on a barrier that nothing ever completes, and
+ * then reports exactly as the product kernels do: *status_word (device int32, required) receives
+ * HGA_STATUS_WAIT_TIMEOUT, waited_cycles (device int64, optional) the cycles the wait lasted.
+ * The context stays usable. */
+HGA_API int hga_selftest_bounded_wait(uint32_t cycle_limit, int32_t* status_word, long long* waited_cycles,
+                                      void* stream);
 
 #ifdef __cplusplus
 }

@@ -31,7 +31,13 @@ HGA_ROUTE_STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = ("hga_build_summaries", "hga_route", "hga_route_static", "hga_attn_fwd", "hga_attn_bwd",
            "hga_workspace_bytes", "hga_step_host", "hga_step_arena_bytes", "hga_tbptt_walk", "hga_varlen_step",
            "hga_varlen_workspace_bytes", "hga_status_string",
-           "hga_version", "hga_last_cuda_error", "hga_kernel_launch_count")
+           "hga_version", "hga_last_cuda_error", "hga_kernel_launch_count", "hga_kernel_launch_count_by_family",
+           "hga_selftest_bounded_wait")
+
+# kernel families of hga_kernel_launch_count_by_family
+(HGA_KERNELS_SUMMARIES, HGA_KERNELS_ROUTE_TENSOR, HGA_KERNELS_ROUTE_GENERIC, HGA_KERNELS_FWD_TENSOR,
+ HGA_KERNELS_FWD_GENERIC, HGA_KERNELS_BWD_TENSOR, HGA_KERNELS_BWD_GENERIC, HGA_KERNELS_AUX) = range(8)
+HGA_KERNELS_FAMILIES = 8
 
 
 class HgaParams(C.Structure):
@@ -66,6 +72,9 @@ def lib():
         L.hga_status_string.restype = C.c_char_p
         L.hga_status_string.argtypes = [C.c_int]
         L.hga_kernel_launch_count.restype = C.c_int64
+        L.hga_kernel_launch_count_by_family.restype = C.c_int64
+        L.hga_kernel_launch_count_by_family.argtypes = [C.c_int]
+        L.hga_selftest_bounded_wait.argtypes = [C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p]
         vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
         pp = C.POINTER(HgaParams)
         L.hga_build_summaries.argtypes = [pp, vp, i32, i32, vp, vp, vp]
@@ -135,6 +144,17 @@ def hga_version() -> int:
 
 def hga_kernel_launch_count() -> int:
     return int(lib().hga_kernel_launch_count())
+
+
+def hga_kernel_launch_counts() -> list:
+    """Launch counts per kernel family (index = HGA_KERNELS_*)."""
+    return [int(lib().hga_kernel_launch_count_by_family(f)) for f in range(HGA_KERNELS_FAMILIES)]
+
+
+def hga_selftest_bounded_wait(cycle_limit, status_word, waited_cycles=None, stream=None):
+    """Runs the library's bounded on-chip wait on a barrier nothing completes (see hga.h)."""
+    _check("hga_selftest_bounded_wait", lib().hga_selftest_bounded_wait(
+        int(cycle_limit), _ptr(status_word), _ptr(waited_cycles), _stream(stream)))
 
 
 def hga_workspace_bytes(p: HgaParams):

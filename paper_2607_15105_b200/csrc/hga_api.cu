@@ -11,10 +11,17 @@
 
 namespace hga {
 
-static std::atomic<int64_t> g_launches{0};
+static std::atomic<int64_t> g_launches[HGA_KERNELS_FAMILIES];
 static std::atomic<int> g_last_cuda{0};
 
-void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+void count_launch(int family, int n) { g_launches[family].fetch_add(n, std::memory_order_relaxed); }
+
+// Set while hga_step_host calls the exported steps with the library's internal flag bits.
+static thread_local bool t_internal_flags = false;
+struct InternalFlagsScope {
+  InternalFlagsScope() { t_internal_flags = true; }
+  ~InternalFlagsScope() { t_internal_flags = false; }
+};
 
 int record_cuda(cudaError_t e) {
   if (e == cudaSuccess) return HGA_OK;
@@ -49,7 +56,7 @@ static int resolve(const hga_params* p, Dims& dm) {
   if (p->chunk / p->group > 64) return HGA_ERR_UNSUPPORTED;
   if (p->topk_chunks > 1024) return HGA_ERR_UNSUPPORTED;
   if ((p->flags & HGA_FLAG_SCORE_MEAN) && (p->flags & HGA_FLAG_SCORE_LSE)) return HGA_ERR_UNSUPPORTED;
-  if (p->flags & ~0x7f & ~kFlagNoPdl) return HGA_ERR_UNSUPPORTED;      // unknown flag bits
+  if (p->flags & ~0x7f & ~(t_internal_flags ? kFlagNoPdl : 0)) return HGA_ERR_UNSUPPORTED;   // unknown flag bits
   if ((p->flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) && (int64_t)p->topk_chunks * (p->chunk / p->group) > 4096)
     return HGA_ERR_UNSUPPORTED;
   dm.B = p->batch; dm.Hq = p->n_q_heads; dm.Hkv = p->n_kv_heads; dm.G = dm.Hq / dm.Hkv;
@@ -149,7 +156,16 @@ int hga_version(void) { return HGA_VERSION; }
 
 int hga_last_cuda_error(void) { return g_last_cuda.load(); }
 
-int64_t hga_kernel_launch_count(void) { return g_launches.load(); }
+int64_t hga_kernel_launch_count(void) {
+  int64_t n = 0;
+  for (auto& c : g_launches) n += c.load();
+  return n;
+}
+
+int64_t hga_kernel_launch_count_by_family(int family) {
+  if (family < 0 || family >= HGA_KERNELS_FAMILIES) return -1;
+  return g_launches[family].load();
+}
 
 const char* hga_status_string(int s) {
   switch (s) {
@@ -251,9 +267,8 @@ int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* 
   }
   rc = HGA_ERR_UNSUPPORTED;
   if (attn_bwd_sm100_supported(dm)) {
-    // zero-fills dK/dV itself where its kernels need it; UNSUPPORTED is returned before any launch
-    rc = launch_attn_bwd_sm100(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV, (float*)workspace,
-                               zero_grads, status_word, st);
+    // its band kernel stores every row of dK/dV (or adds to it); UNSUPPORTED is returned before any launch
+    rc = launch_attn_bwd_sm100(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV, status_word, st);
   }
   if (rc == HGA_ERR_UNSUPPORTED) {
     if (zero_grads) {
@@ -278,12 +293,11 @@ int hga_step_arena_bytes(const hga_params* p, size_t* bytes) {
   if (!bytes) return HGA_ERR_NULL;
   size_t q = (size_t)dm.B * dm.Hq * dm.S * dm.d * 2;           // Q, dO, O, dQ (bf16)
   size_t kv32 = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 4;       // dK, dV (fp32)
-  size_t kvseg = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 2;      // staged K/V segment rows
   size_t items = (size_t)dm.B * dm.Hkv * dm.NQB;
   size_t idx = items * (dm.kc + dm.width + 1) * 4 + 64;
   size_t lse = (size_t)dm.B * dm.Hq * dm.S * 4;
   auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
-  *bytes = 4 * up(q) + 2 * up(kv32) + 2 * up(kvseg) + up(idx) + up(lse) +
+  *bytes = 4 * up(q) + 2 * up(kv32) + up(idx) + up(lse) +
            up(route_workspace_bytes(dm)) + up(bwd_workspace_bytes(dm)) + 256;
   return HGA_OK;
 }
@@ -318,11 +332,9 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   auto take = [&](size_t n) { char* r = a; a += up(n); return (void*)r; };
   size_t qb = (size_t)dm.B * dm.Hq * dm.S * dm.d * 2;
   size_t kv32 = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 4;
-  size_t kvseg = (size_t)dm.B * dm.Hkv * dm.S * dm.d * 2;
   size_t items = (size_t)dm.B * dm.Hkv * dm.NQB;
   char* dQin = (char*)take(qb); char* ddO = (char*)take(qb); char* dOut = (char*)take(qb); char* ddQ = (char*)take(qb);
   char* ddK = (char*)take(kv32); char* ddV = (char*)take(kv32);
-  take(kvseg); take(kvseg);                          // (reserved: earlier versions staged the K/V rows here)
   int32_t* cidx = (int32_t*)take(items * (dm.kc + dm.width + 1) * 4 + 64);
   int32_t* gidx = cidx + items * dm.kc;
   int32_t* ng = gidx + items * dm.width;
@@ -342,6 +354,7 @@ int hga_step_host(const hga_params* p, const void* Q_host, const void* Kseg_host
   pc.n_q_heads = dm.G;
   pc.n_kv_heads = 1;
   pc.flags |= kFlagNoPdl;                            // this pipeline is bound by the host link (see hga_common.cuh)
+  InternalFlagsScope internal;                       // lets the exported steps below accept that bit
   const size_t q_c = (size_t)dm.G * dm.S * dm.d * 2;           // bytes of one pair's Q / dO / O / dQ rows
   const size_t kvseg_c = (size_t)dm.S * dm.d * 2, kv32_c = (size_t)dm.S * dm.d * 4;
   const size_t kv_c = (size_t)dm.L * dm.d * 2;                 // one (batch, kv head) of the resident K / V

@@ -5,23 +5,27 @@
 // Every key of the active segment lies in the band of a few consecutive query blocks (its own
 // block and the ones whose local window still reaches it).  Summing those contributions with
 // atomics from the query-major sweep costs one red.add per element per contributing M-tile; here
-// one CTA owns a 64-key tile instead, loops over every 128-row M-tile of every query block whose
-// band holds the tile, accumulates dK^T and dV^T in TMEM and writes the tile once with plain stores.
-// The query-major sweep (k_attn_bwd_sm100) then adds only the contributions of keys selected
-// through routing, and computes dQ for all keys.
+// one CTA owns a 128-key tile instead, loops over every 128-row M-tile of every query block whose
+// band touches the tile, accumulates dK and dV in tensor memory and writes the tile once with plain
+// stores.  The query-major sweep (k_attn_bwd_sm100) then adds only the contributions of keys
+// selected through routing (and of sink keys inside the active segment), and computes dQ.
 //
-// Work unit (one CTA): (batch, kv head, 64-key tile of the active segment).  Per M-tile m:
-//   S = Q K^T, dP = dO V^T                       (smem x smem) -> TMEM, double buffered
-//   P = 2^(S*c - LSE*log2e), dS = scale * P o (dP - delta)     (one thread per query row) -> smem
-//   dV^T += dO^T P,  dK^T += Q^T dS              (M = head_dim, N = 64 keys, K = 128 rows) -> TMEM
-// Q and dO tiles stream through a two-stage ring as boxes of 64 rows x one 64-element panel, laid
-// out [panel][128 rows][128 B]: the 128-byte-swizzled layout the GEMMs read both K-major (S, dP)
-// and MN-major (dK^T, dV^T).  The MMA thread issues whichever GEMM group (S,dP of the next M-tile or
-// dK,dV of the previous one) has its inputs ready, so the two ring stages advance independently.
+// The GEMMs are the TRANSPOSED ones, so that P and dS never pass through shared memory:
+//   S^T  = K Q^T,  dP^T = V dO^T         (M = 128 keys, N = 128 query rows, K = head_dim)  smem x smem
+//   P^T  = 2^(S^T*c - LSE*log2e),  dS^T = scale * P^T o (dP^T - delta)    one thread per KEY (TMEM lane),
+//          written back as bf16 over the columns just read
+//   dV  += P^T dO,  dK += dS^T Q         (M = 128 keys, N = head_dim, K = 128 query rows)  A from TMEM
+// All of them are M = 128, N = 128 instructions (full tensor-pipe rate).
+// delta = rowsum(dO o O) of the M-tile's rows is computed here, by four otherwise idle warps (one
+// thread per query row: its O row from global memory, its dO row from the tile in shared memory), so
+// the backward needs no separate pass over O and dO.
 //
-// Warp roles (320 threads): warp 0 producer, warp 1 MMA issuer, warps 2-5 and 6-9 two warpgroups
-// of row threads on alternate M-tiles; at the end warps 2-5 store dV, warps 6-9 store dK.
-// TMEM (512 columns allocated): S[2] dP[2] (64 each) | dV^T 64 | dK^T 64.
+// Work unit (one CTA): (batch, kv head, 128-key tile of the active segment); keys past the end of the
+// segment arrive as zeros, are masked by causality and are not stored.
+// Warp roles (448 threads): warp 0 producer (K, V once; Q, dO tiles through a two-stage ring),
+// warp 1 MMA issuer, warps 2-5 and 6-9 one thread per key (warpgroup w: query rows 64w .. 64w+63 of
+// the M-tile), warps 10-13 row statistics (LSE, delta).
+// TMEM (512 columns): S^T / P^T | dP^T / dS^T | dV | dK, 128 columns each.
 #include "hga_bwd_sm100.cuh"
 #include "hga_common.cuh"
 #include "hga_sm100.cuh"
@@ -32,58 +36,64 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kBandThreads = 320;
+constexpr int kBandThreads = 448;
 constexpr int kD = 128;
-constexpr int kKT = 64;                          // keys per tile
-constexpr int kQTile = 128 * kD * 2;             // bytes of one Q or dO tile
-constexpr int kKvTile = kKT * kD * 2;
-constexpr int kPdsTile = 128 * kKT * 2;
+constexpr int kKeys = 128;                       // keys per CTA
+constexpr int kTile = 128 * kD * 2;              // bytes of one K, V, Q or dO tile: [panel][128 rows][128 B]
 
 struct BandSmem {
-  alignas(1024) uint8_t q[2][kQTile];            // [panel][128 rows][128 B]
-  alignas(1024) uint8_t dO[2][kQTile];
-  alignas(1024) uint8_t k[kKvTile];              // [panel][64 keys][128 B]
-  alignas(1024) uint8_t v[kKvTile];
-  alignas(1024) uint8_t p[2][kPdsTile];          // [16 row octets][8 rows][128 B]
-  alignas(1024) uint8_t ds[2][kPdsTile];
-  uint64_t kv_full, qdo_full[2], qdo_empty[2], sdp_full[2], sdp_free[2], pds_full[2], pds_free[2], acc_done;
+  alignas(1024) uint8_t k[kTile];
+  alignas(1024) uint8_t v[kTile];
+  alignas(1024) uint8_t q[2][kTile];
+  alignas(1024) uint8_t dO[2][kTile];
+  alignas(16) float nlse[2][128];                // per query row of the M-tile in a stage: -LSE * log2(e)
+  alignas(16) float nds[2][128];                 //                                         -delta * scale
+  uint64_t kv_full, qdo_full[2], qdo_empty[2], stat_full[2];
+  uint64_t s_full, dp_full, pds_full, acc_done, drain;
   uint32_t tmem_base;
   volatile int abort;
 };
 
+// query block of step m, and the first query row (inside the item) of its M-tile
+struct Step {
+  int qb, r0;
+};
+
+}  // namespace
+
 __global__ void __launch_bounds__(kBandThreads, 1)
 k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
                       const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                      const float* __restrict__ delta_ws, const float* __restrict__ LSE, Dims dm,
+                      const uint16_t* __restrict__ O, const float* __restrict__ LSE, Dims dm,
                       float* __restrict__ dK, float* __restrict__ dV, int32_t* status_word) {
-  constexpr uint32_t kColSdP = 0;       // S[b] at 128*b, dP[b] at 128*b + 64
-  constexpr uint32_t kColDV = 256, kColDK = 320;
+  constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
   extern __shared__ uint8_t smem_raw[];
   BandSmem& sm = *reinterpret_cast<BandSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   HGA_TRACE_DECL;
-  const int tiles_per_seq = dm.S / kKT;
+  const int tiles_per_seq = (dm.S + kKeys - 1) / kKeys;
   const int kt = blockIdx.x % tiles_per_seq;
   const int bh = blockIdx.x / tiles_per_seq;
   const int h = bh % dm.Hkv, b = bh / dm.Hkv;
-  const int k0 = dm.H + kt * kKT;                 // first key position of the tile
-  // query blocks whose band [ls, p0 + Bq) holds the tile: the tile's own block and the following
-  // ones while their local window still starts at or before the tile
-  const int qb_own = (kt * kKT) / dm.Bq;
+  const int k0 = dm.H + kt * kKeys;               // first key position of the tile
+  const int k_end = min(k0 + kKeys, dm.L);        // one past its last real key
+  // query blocks whose band [ls, p0 + Bq) touches the tile: from the block that holds the tile's first
+  // key, while the local window still starts before the tile's end
+  const int qb_first = (kt * kKeys) / dm.Bq;
   int n_qb = 1;
-  while (qb_own + n_qb < dm.NQB && window_of(dm, qb_own + n_qb).ls <= k0) ++n_qb;
+  while (qb_first + n_qb < dm.NQB && window_of(dm, qb_first + n_qb).ls < k_end) ++n_qb;
   const int n_mt = dm.rows / 128;
   const int n_steps = n_qb * n_mt;
+  auto step_of = [&](int m) { return Step{qb_first + m / n_mt, (m % n_mt) * 128}; };
 
   if (tid == 0) {
     mbar_init(&sm.kv_full, 1);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.qdo_full[s], 1); mbar_init(&sm.qdo_empty[s], 1);
-      mbar_init(&sm.sdp_full[s], 1); mbar_init(&sm.sdp_free[s], 128);
-      mbar_init(&sm.pds_full[s], 128); mbar_init(&sm.pds_free[s], 1);
+      mbar_init(&sm.qdo_full[s], 1); mbar_init(&sm.qdo_empty[s], 1); mbar_init(&sm.stat_full[s], 128);
     }
-    mbar_init(&sm.acc_done, 1);
+    mbar_init(&sm.s_full, 1); mbar_init(&sm.dp_full, 1); mbar_init(&sm.pds_full, 256);
+    mbar_init(&sm.acc_done, 1); mbar_init(&sm.drain, 1);
     sm.abort = 0;
     fence_barrier_init();
   }
@@ -95,6 +105,9 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
+  // the sweep, next in the stream, may start on SMs this grid leaves idle (it waits for this grid only
+  // before it adds to dK/dV)
+  if (tid == 0) pdl_launch_dependents();
 
   const uint32_t tmem = sm.tmem_base;
   volatile int* abort = &sm.abort;
@@ -102,28 +115,30 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
-    // A copy is latency-bound per box, so a Q or dO tile travels as four boxes of 64 rows x one
-    // 64-element panel (8 KB each), issued by eight lanes at once: lanes 0-3 Q, lanes 4-7 dO.
+    // A copy is latency-bound per box, so every tile travels as four boxes of 64 rows x one 64-element
+    // panel (8 KB each), issued by eight lanes at once: lanes 0-3 K or Q, lanes 4-7 V or dO.
+    const int half = lane & 1, panel = (lane >> 1) & 1;
+    const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
     if (lane == 0) {
       prefetch_tensormap(&map_q); prefetch_tensormap(&map_do);
       prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
-      mbar_arrive_expect_tx(&sm.kv_full, 2 * kKvTile);
-      tma_load_5d(sm.k, &map_k, &sm.kv_full, 0, k0, 0, h, b);
-      tma_load_5d(sm.v, &map_v, &sm.kv_full, 0, k0, 0, h, b);
+      mbar_arrive_expect_tx(&sm.kv_full, 2 * kTile);
     }
-    const int half = lane & 1, panel = (lane >> 1) & 1;       // 64-row half of the M-tile, d panel
+    __syncwarp();
+    if (lane < 4) tma_load_5d(sm.k + off, &map_k, &sm.kv_full, 0, k0 + 64 * half, panel, h, b);
+    else if (lane < 8) tma_load_5d(sm.v + off, &map_v, &sm.kv_full, 0, k0 + 64 * half, panel, h, b);
     bool ok = true;
     int issued = 0;
     for (int m = 0; m < n_steps; ++m) {
       const int st = m & 1;
-      const int qb = qb_own + m / n_mt, r0 = (m % n_mt) * 128 + half * 64;
+      const Step sp = step_of(m);
+      const int r = sp.r0 + 64 * half;
       if (lane == 0 && m >= 2) ok = bwd_wait(&sm.qdo_empty[st], ((m >> 1) - 1) & 1, abort);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
-      if (lane == 0) mbar_arrive_expect_tx(&sm.qdo_full[st], 2 * kQTile);
+      if (lane == 0) mbar_arrive_expect_tx(&sm.qdo_full[st], 2 * kTile);
       __syncwarp();
-      const int row = qb * dm.Bq + r0 % dm.Bq, head = h * dm.G + r0 / dm.Bq;
-      const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
+      const int row = sp.qb * dm.Bq + r % dm.Bq, head = h * dm.G + r / dm.Bq;
       if (lane < 4) tma_load_5d(sm.q[st] + off, &map_q, &sm.qdo_full[st], 0, row, panel, head, b);
       else if (lane < 8) tma_load_5d(sm.dO[st] + off, &map_do, &sm.qdo_full[st], 0, row, panel, head, b);
       issued = m + 1;
@@ -137,184 +152,249 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc_sdp = idesc_bf16_f32(128, kKT, 0, 0);   // rows x keys, both K-major
-      constexpr uint32_t idesc_dkv = idesc_bf16_f32(kD, kKT, 1, 1);    // both MN-major
-      const uint64_t q_k0 = smem_desc_sw128(smem_u32(sm.q[0]), 16, 1024);       // Q  K-major A (S)
-      const uint64_t do_k0 = smem_desc_sw128(smem_u32(sm.dO[0]), 16, 1024);     // dO K-major A (dP)
-      const uint64_t q_mn0 = smem_desc_sw128(smem_u32(sm.q[0]), 16384, 1024);   // Q^T  MN-major A (dK^T)
-      const uint64_t do_mn0 = smem_desc_sw128(smem_u32(sm.dO[0]), 16384, 1024); // dO^T MN-major A (dV^T)
-      const uint64_t k_k = smem_desc_sw128(smem_u32(sm.k), 16, 1024);           // K tile K-major B (S)
-      const uint64_t v_k = smem_desc_sw128(smem_u32(sm.v), 16, 1024);           // V tile K-major B (dP)
-      const uint64_t ds0 = smem_desc_sw128(smem_u32(sm.ds[0]), 16, 1024);       // dS MN-major B (dK^T)
-      const uint64_t p0 = smem_desc_sw128(smem_u32(sm.p[0]), 16, 1024);         // P  MN-major B (dV^T)
-      auto issue_sdp = [&](int m) {
-        const uint32_t st = (uint32_t)(m & 1);
-        const uint64_t qd = desc_advance(q_k0, st * kQTile), dod = desc_advance(do_k0, st * kQTile);
-        const uint32_t s_acc = tmem + kColSdP + st * 128;
+      constexpr uint32_t idesc_t = idesc_bf16_f32(128, 128, 0, 0);     // keys x rows: A, B K-major (head_dim runs along K)
+      constexpr uint32_t idesc_g = idesc_bf16_f32(128, kD, 0, 1);      // keys x head_dim: A from TMEM, B MN-major
+      // every tile is [panel][128 rows][128 B]: K-major with 8-row groups 1024 B apart and the second
+      // panel 16 KB on; MN-major (head_dim along N, rows along K) with panels 16 KB and 8-row groups 1024 B apart
+      const uint64_t k_k = smem_desc_sw128(smem_u32(sm.k), 16, 1024);
+      const uint64_t v_k = smem_desc_sw128(smem_u32(sm.v), 16, 1024);
+      const uint64_t q_k0 = smem_desc_sw128(smem_u32(sm.q[0]), 16, 1024);
+      const uint64_t do_k0 = smem_desc_sw128(smem_u32(sm.dO[0]), 16, 1024);
+      const uint64_t q_mn0 = smem_desc_sw128(smem_u32(sm.q[0]), 16384, 1024);
+      const uint64_t do_mn0 = smem_desc_sw128(smem_u32(sm.dO[0]), 16384, 1024);
+      // acc (keys x rows) = a (K or V tile) x b^T (Q or dO tile), both K-major
+      auto issue_t = [&](uint32_t acc, uint64_t a, uint64_t bq) {
 #pragma unroll
-        for (int kk = 0; kk < kD / 16; ++kk)
-          mma_ss(s_acc, desc_advance(qd, (kk >> 2) * 16384 + (kk & 3) * 32),
-                 desc_advance(k_k, (kk >> 2) * 8192 + (kk & 3) * 32), idesc_sdp, kk > 0);
-#pragma unroll
-        for (int kk = 0; kk < kD / 16; ++kk)
-          mma_ss(s_acc + 64, desc_advance(dod, (kk >> 2) * 16384 + (kk & 3) * 32),
-                 desc_advance(v_k, (kk >> 2) * 8192 + (kk & 3) * 32), idesc_sdp, kk > 0);
-        mma_commit(&sm.sdp_full[st]);
+        for (int kk = 0; kk < kD / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;       // panel, then 32-byte K step
+          mma_ss(acc, desc_advance(a, off), desc_advance(bq, off), idesc_t, kk > 0);
+        }
       };
-      auto issue_dkv = [&](int m) {
-        const uint32_t st = (uint32_t)(m & 1);
-        const uint64_t pd = desc_advance(p0, st * kPdsTile), dsd = desc_advance(ds0, st * kPdsTile);
-        const uint64_t dom = desc_advance(do_mn0, st * kQTile), qm = desc_advance(q_mn0, st * kQTile);
-#pragma unroll
-        for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per step
-          mma_ss(tmem + kColDV, desc_advance(dom, kk * 2048), desc_advance(pd, kk * 2048), idesc_dkv,
-                 (m > 0 || kk > 0));
+      // acc (keys x head_dim) += a (keys x rows, bf16 in TMEM: rows 0-63 at columns 0-31, rows 64-127 at
+      // columns 64-95 of its region) x b (Q or dO tile: rows along K, 16 rows per instruction)
+      auto issue_g = [&](uint32_t acc, uint32_t a_tmem, uint64_t bmn, bool accumulate) {
 #pragma unroll
         for (int kk = 0; kk < 128 / 16; ++kk)
-          mma_ss(tmem + kColDK, desc_advance(qm, kk * 2048), desc_advance(dsd, kk * 2048), idesc_dkv,
-                 (m > 0 || kk > 0));
-        mma_commit(&sm.pds_free[st]);
-        mma_commit(&sm.qdo_empty[st]);
+          mma_ts(acc, a_tmem + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), desc_advance(bmn, kk * 2048), idesc_g,
+                 (accumulate || kk > 0));
       };
-      // The two ring stages form two independent chains (copy -> S,dP -> row threads -> dK,dV ->
-      // next copy); whichever GEMM group has its inputs ready is issued next, the dK/dV group
-      // first because it releases a stage.
-      bool ok = bwd_wait(&sm.kv_full, 0, abort);
-      int next_sdp = 0, next_dkv = 0;
-      uint32_t idle = 0;
-      while (ok && next_dkv < n_steps) {
-        bool did = false;
-        if (next_dkv < next_sdp && mbar_test_wait(&sm.pds_full[next_dkv & 1], (next_dkv >> 1) & 1)) {
+      bool ok = bwd_wait(&sm.kv_full, 0, abort) && bwd_wait(&sm.qdo_full[0], 0, abort);
+      if (ok) {
+        tc_fence_after_sync();
+        issue_t(tmem + kColS, k_k, q_k0);
+        mma_commit(&sm.s_full);
+        issue_t(tmem + kColDP, v_k, do_k0);
+        mma_commit(&sm.dp_full);
+      }
+      HGA_TRACE_POINT(3);
+      for (int m = 0; m < n_steps && ok; ++m) {
+        const uint32_t st = (uint32_t)(m & 1), st_n = st ^ 1u;
+        const bool more = m + 1 < n_steps;
+        ok = bwd_wait(&sm.pds_full, m & 1, abort);               // P^T and dS^T of step m are in TMEM
+        if (!ok) break;
+        tc_fence_after_sync();
+        HGA_TRACE_POINT(5);
+        issue_g(tmem + kColDV, tmem + kColS, desc_advance(do_mn0, st * kTile), m > 0);
+        if (more) {
+          // S^T of the next M-tile overwrites P^T: the in-order tensor pipe runs it after the dV GEMM above
+          ok = bwd_wait(&sm.qdo_full[st_n], ((m + 1) >> 1) & 1, abort);
+          if (!ok) break;
           tc_fence_after_sync();
-          issue_dkv(next_dkv);
-          ++next_dkv;
-          did = true;
-          HGA_TRACE_POINT(7);
+          issue_t(tmem + kColS, k_k, desc_advance(q_k0, st_n * kTile));
+          mma_commit(&sm.s_full);
         }
-        if (next_sdp < n_steps && mbar_test_wait(&sm.qdo_full[next_sdp & 1], (next_sdp >> 1) & 1) &&
-            (next_sdp < 2 || mbar_test_wait(&sm.sdp_free[next_sdp & 1], ((next_sdp >> 1) - 1) & 1))) {
-          // (a full stage implies that dK/dV of M-tile next_sdp-2 were issued, hence that its row
-          // threads are done with TMEM buffer next_sdp&1; the sdp_free test makes that visible here)
-          tc_fence_after_sync();
-          issue_sdp(next_sdp);
-          ++next_sdp;
-          did = true;
-          HGA_TRACE_POINT(6);
+        issue_g(tmem + kColDK, tmem + kColDP, desc_advance(q_mn0, st * kTile), m > 0);
+        mma_commit(&sm.qdo_empty[st]);                           // Q and dO of step m are consumed
+        if (more) {
+          issue_t(tmem + kColDP, v_k, desc_advance(do_k0, st_n * kTile));
+          mma_commit(&sm.dp_full);
         }
-        if (did) idle = 0;
-        else if (++idle >= (1u << 22) || ((idle & 255u) == 255u && *abort)) { *abort = 1; ok = false; }
+        HGA_TRACE_POINT(7);
       }
       if (ok) mma_commit(&sm.acc_done);
     }
-  } else {
-    // ------------------------------------------------------------------ one thread per query row
-    const int wg = (warp - 2) >> 2;
-    const int quarter = warp & 3;
-    const int row_in_tile = quarter * 32 + lane;
+  } else if (warp < 10) {
+    // ------------------------------------------------------------------ one thread per key
+    const int wg = (warp - 2) >> 2;                  // query rows 64*wg .. 64*wg+63 of each M-tile
+    const int quarter = warp & 3;                    // TMEM lanes this warp may touch
+    const int key = quarter * 32 + lane;
+    const int kp = k0 + key;                         // absolute position of this thread's key
     const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t s_addr = lane_base + kColS + 64 * wg, dp_addr = lane_base + kColDP + 64 * wg;
     const float sl2 = dm.scale * 1.4426950408889634f;
-    const uint32_t line = (uint32_t)(row_in_tile >> 3) * 1024 + (uint32_t)(row_in_tile & 7) * 128;
-    const uint32_t key = (uint32_t)(row_in_tile & 7);
-    const uint32_t p_line = smem_u32(sm.p[wg]) + line, ds_line = smem_u32(sm.ds[wg]) + line;
-    const uint32_t sdp_addr = lane_base + kColSdP + wg * 128;
-    // LSE, delta and the causal limit of this thread's row in M-tile m
-    auto row_of = [&](int m, float& lse, float& dl, int& vis) {
-      const int qb = qb_own + m / n_mt, r = (m % n_mt) * 128 + row_in_tile;
-      const int a = r / dm.Bq, t = r % dm.Bq;
-      const int64_t row = ((int64_t)b * dm.Hq + h * dm.G + a) * dm.S + qb * dm.Bq + t;
-      lse = LSE[row];
-      dl = delta_ws[row];
-      vis = qb * dm.Bq + t - kt * kKT + 1;       // keys of the tile at or before the query position
-    };
-    float lse = 0.f, dl = 0.f;
-    int vis = 0;
-    // This kernel is launched with programmatic serialization behind the delta pre-pass: everything up to
-    // here (set-up, the K/V tile and the first Q/dO tiles, which are inputs of the call) may have run
-    // while that kernel was still busy; delta is read from here on.  Only then is the sweep, which follows
-    // in the stream and reads delta too, allowed to start on the SMs this grid leaves idle (it waits for
-    // this grid itself only before it adds to dK/dV).
-    pdl_wait();
-    if (warp == 2 && lane == 0) pdl_launch_dependents();
-    if (wg < n_steps) row_of(wg, lse, dl, vis);
+    const uint64_t sl2_2 = pack_f32x2(sl2, sl2), scale_2 = pack_f32x2(dm.scale, dm.scale);
     bool ok = true;
-    for (int m = wg; m < n_steps; m += 2) {
-      const float neg_lse2 = -lse * 1.4426950408889634f;
-      const float neg_delta_s = -dl * dm.scale;
-      const uint64_t sl2_2 = pack_f32x2(sl2, sl2), neg_lse2_2 = pack_f32x2(neg_lse2, neg_lse2);
-      const uint64_t scale_2 = pack_f32x2(dm.scale, dm.scale), neg_delta_s_2 = pack_f32x2(neg_delta_s, neg_delta_s);
-      const int vis_m = vis;
-      if (m + 2 < n_steps) row_of(m + 2, lse, dl, vis);      // prefetch the next M-tile's row data
-      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[wg], (m >> 1) & 1, abort));
+    for (int m = 0; m < n_steps; ++m) {
+      const int st = m & 1;
+      const Step sp = step_of(m);
+      const Window w = window_of(dm, sp.qb);
+      // the warpgroup's 64 columns are 64 consecutive positions of one query head (Bq is a multiple of 64);
+      // column i is visible to this key iff the key is inside the block's band and not after the query
+      const int qp0 = w.p0 + (sp.r0 + 64 * wg) % dm.Bq;
+      const int imin = (kp < w.ls || kp >= k_end) ? 64 : kp - qp0;       // first visible column (may be <= 0)
+      const bool none = __all_sync(0xffffffffu, imin >= 64);
+      const bool masked = __any_sync(0xffffffffu, imin > 0);
+      const uint32_t nlse_a = smem_u32(&sm.nlse[st][64 * wg]), nds_a = smem_u32(&sm.nds[st][64 * wg]);
+      uint32_t pk[32];                               // P of this key against 64 query rows, packed bf16
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.s_full, m & 1, abort));
+      if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.stat_full[st], (m >> 1) & 1, abort));
       if (!ok) break;
       tc_fence_after_sync();
       HGA_TRACE_POINT(11);
-      if (m >= 2) {     // the GEMMs that read this P/dS buffer two steps ago must have finished
-        ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_free[wg], ((m >> 1) - 1) & 1, abort));
-        if (!ok) break;
+      if (none) {
+        // no key of this warp is visible to any row of the half tile: zeros, no exponentials
+#pragma unroll
+        for (int i = 0; i < 32; ++i) pk[i] = 0u;
       }
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {               // 16 keys at a time
-        uint32_t sv[16], dp[16];
-        tmem_ld16(sdp_addr + q4 * 16, sv);
-        tmem_ld16(sdp_addr + 64 + q4 * 16, dp);
-        tmem_wait_ld();
-        if (q4 == 3) {
-          tc_fence_before_sync();
-          mbar_arrive(&sm.sdp_free[wg]);
-        }
-        uint32_t pk[8], dk[8];
+      for (int c = 0; c < 2; ++c) {
+        if (!none) {
+          uint32_t x[32];
+          tmem_ld32(s_addr + 32 * c, x);
+          tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          // packed fp32 pairs: one FMA-pipe instruction for two columns
-          float a0, a1, d0, d1;
-          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), sl2_2, neg_lse2_2), a0, a1);
-          float p0 = fast_exp2(a0), p1 = fast_exp2(a1);
-          if (vis_m < kKT) {                  // the tile's own query block: causal mask
-            if (q4 * 16 + 2 * i >= vis_m) p0 = 0.f;
-            if (q4 * 16 + 2 * i + 1 >= vis_m) p1 = 0.f;
+          for (int i = 0; i < 16; i += 2) {
+            uint32_t n0, n1, n2, n3;                 // -LSE*log2e of four consecutive columns
+            ld_shared_v4(nlse_a + (32 * c + 2 * i) * 4, n0, n1, n2, n3);
+            float a0, a1, a2, a3;
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1])), sl2_2,
+                                   pack_f32x2(__uint_as_float(n0), __uint_as_float(n1))), a0, a1);
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i + 2]), __uint_as_float(x[2 * i + 3])), sl2_2,
+                                   pack_f32x2(__uint_as_float(n2), __uint_as_float(n3))), a2, a3);
+            float p0 = fast_exp2(a0), p1 = fast_exp2(a1), p2 = fast_exp2(a2), p3 = fast_exp2(a3);
+            if (masked) {
+              const int col = 32 * c + 2 * i;
+              if (col < imin) p0 = 0.f;
+              if (col + 1 < imin) p1 = 0.f;
+              if (col + 2 < imin) p2 = 0.f;
+              if (col + 3 < imin) p3 = 0.f;
+            }
+            pk[16 * c + i] = pack_bf16(p0, p1);
+            pk[16 * c + i + 1] = pack_bf16(p2, p3);
           }
-          const uint64_t g2 = fma_f32x2(pack_f32x2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])), scale_2, neg_delta_s_2);
-          unpack_f32x2(mul_f32x2(pack_f32x2(p0, p1), g2), d0, d1);
-          pk[i] = pack_bf16(p0, p1);
-          dk[i] = pack_bf16(d0, d1);
         }
+        // P^T (bf16) over the S^T columns just read: 16 columns per 32 query rows
+        uint32_t out[16];
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {      // two 16-byte chunks (8 keys each), XOR-swizzled
-          const uint32_t off = ((uint32_t)(2 * q4 + cc) ^ key) * 16;
-          st_shared_v4(p_line + off, pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-          st_shared_v4(ds_line + off, dk[4 * cc], dk[4 * cc + 1], dk[4 * cc + 2], dk[4 * cc + 3]);
-        }
+        for (int i = 0; i < 16; ++i) out[i] = pk[16 * c + i];
+        tmem_st16(s_addr + 16 * c, out);
       }
-      fence_proxy_async_smem();
-      mbar_arrive(&sm.pds_full[wg]);
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.dp_full, m & 1, abort));
+      if (!ok) break;
+      tc_fence_after_sync();
+      HGA_TRACE_POINT(13);
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t out[16];
+        if (!none) {
+          uint32_t x[32];
+          tmem_ld32(dp_addr + 32 * c, x);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 16; i += 2) {
+            uint32_t n0, n1, n2, n3;                 // -delta*scale of four consecutive columns
+            ld_shared_v4(nds_a + (32 * c + 2 * i) * 4, n0, n1, n2, n3);
+            const uint32_t pa = pk[16 * c + i], pb = pk[16 * c + i + 1];
+            const uint64_t g0 = fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1])), scale_2,
+                                          pack_f32x2(__uint_as_float(n0), __uint_as_float(n1)));
+            const uint64_t g1 = fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i + 2]), __uint_as_float(x[2 * i + 3])), scale_2,
+                                          pack_f32x2(__uint_as_float(n2), __uint_as_float(n3)));
+            float d0, d1, d2, d3;
+            unpack_f32x2(mul_f32x2(pack_f32x2(__uint_as_float(pa << 16), __uint_as_float(pa & 0xffff0000u)), g0), d0, d1);
+            unpack_f32x2(mul_f32x2(pack_f32x2(__uint_as_float(pb << 16), __uint_as_float(pb & 0xffff0000u)), g1), d2, d3);
+            out[i] = pack_bf16(d0, d1);
+            out[i + 1] = pack_bf16(d2, d3);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) out[i] = 0u;
+        }
+        tmem_st16(dp_addr + 16 * c, out);            // dS^T (bf16) over the dP^T columns just read
+      }
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(&sm.pds_full);
       HGA_TRACE_POINT(14);
     }
     if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.acc_done, 0, abort));
     HGA_TRACE_POINT(20);
     if (ok) {
-      // epilogue: thread = head_dim element (TMEM lane); a warp's store covers 128 contiguous bytes
+      // epilogue: thread = key row; warpgroup 0 stores dV, warpgroup 1 dK (512 contiguous bytes per thread)
       tc_fence_after_sync();
-      const int e = quarter * 32 + lane;
-      float* dst = (wg == 0 ? dV : dK) + ((int64_t)(b * dm.Hkv + h) * dm.S + kt * kKT) * kD + e;
+      const int srow = kt * kKeys + key;
+      float* dst = (wg == 0 ? dV : dK) + ((int64_t)(b * dm.Hkv + h) * dm.S + srow) * kD;
       const uint32_t col = wg == 0 ? kColDV : kColDK;
       const bool accumulate = dm.flags & HGA_FLAG_BWD_ACCUMULATE;
+      const bool real = srow < dm.S;
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      for (int c = 0; c < kD / 32; ++c) {
         uint32_t x[32];
-        tmem_ld32(lane_base + col + half * 32, x);
+        tmem_ld32(lane_base + col + 32 * c, x);
         tmem_wait_ld();
+        if (real) {
+          float4* d4 = reinterpret_cast<float4*>(dst + 32 * c);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float* d = dst + (int64_t)(half * 32 + i) * kD;
-          *d = accumulate ? *d + __uint_as_float(x[i]) : __uint_as_float(x[i]);
+          for (int i = 0; i < 8; ++i) {
+            float4 val = make_float4(__uint_as_float(x[4 * i]), __uint_as_float(x[4 * i + 1]),
+                                     __uint_as_float(x[4 * i + 2]), __uint_as_float(x[4 * i + 3]));
+            if (accumulate) {
+              const float4 old = d4[i];
+              val.x += old.x; val.y += old.y; val.z += old.z; val.w += old.w;
+            }
+            d4[i] = val;
+          }
         }
       }
+    }
+  } else {
+    // ------------------------------------------------------------------ row statistics, one thread per query row
+    const int j = (warp - 10) * 32 + lane;           // row of the M-tile
+    const uint32_t key7 = (uint32_t)(j & 7);
+    bool ok = true;
+    for (int m = 0; m < n_steps; ++m) {
+      const int st = m & 1;
+      const Step sp = step_of(m);
+      const int r = sp.r0 + j;
+      const int hq = h * dm.G + r / dm.Bq, srow = sp.qb * dm.Bq + r % dm.Bq;
+      // the O row (256 bytes) is requested before the tile's dO lands in shared memory
+      const uint4* orow = reinterpret_cast<const uint4*>(O + b * dm.os[0] + hq * dm.os[1] + (int64_t)srow * dm.os[2]);
+      uint4 o[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) o[i] = __ldg(orow + i);
+      const float lse = LSE[((int64_t)b * dm.Hq + hq) * dm.S + srow];
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.qdo_full[st], (m >> 1) & 1, abort));
+      if (!ok) break;
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      const uint32_t line = smem_u32(sm.dO[st]) + (uint32_t)j * 128;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {                 // 16-byte chunk i of the row: panel i / 8, chunk i % 8 (XOR-swizzled)
+        uint32_t y0, y1, y2, y3;
+        ld_shared_v4(line + (uint32_t)(i >> 3) * 16384 + (((uint32_t)(i & 7) ^ key7) * 16), y0, y1, y2, y3);
+        const uint32_t xs[4] = {o[i].x, o[i].y, o[i].z, o[i].w}, ys[4] = {y0, y1, y2, y3};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          acc[e] = fmaf(__uint_as_float(xs[e] << 16), __uint_as_float(ys[e] << 16), acc[e]);
+          acc[e] = fmaf(__uint_as_float(xs[e] & 0xffff0000u), __uint_as_float(ys[e] & 0xffff0000u), acc[e]);
+        }
+      }
+      const float delta = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+      // (stage st was last read by the key threads in step m-2, which ended before this step's tile could land)
+      sm.nlse[st][j] = -lse * 1.4426950408889634f;
+      sm.nds[st][j] = -delta * dm.scale;
+      mbar_arrive(&sm.stat_full[st]);
     }
   }
   HGA_TRACE_POINT(30);
 
   // every warp reconverges before the block barrier (a barrier reached by part of a warp would
   // count that warp as arrived)
+  __syncwarp();
+  if (warp == 1 && lane == 0 && sm.abort) {
+    // giving up: GEMMs already issued may still be writing tensor memory; wait (bounded) until the
+    // tensor pipe has run dry before the columns are given back
+    mma_commit(&sm.drain);
+    mbar_wait(&sm.drain, 0);
+  }
   __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
@@ -323,47 +403,35 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
   if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
-}  // namespace
-
 bool attn_bwd_band_sm100_supported(const Dims& dm) {
   if (dm.flags & HGA_FLAG_GENERIC_KERNELS) return false;
-  return dm.d == 128 && dm.rows % 128 == 0 && dm.Bq % 64 == 0 && dm.c % kKT == 0 && dm.H % kKT == 0 && dm.S % kKT == 0;
+  return dm.d == 128 && dm.rows % 128 == 0 && dm.Bq % 64 == 0;
 }
 
-int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const float* LSE,
-                               const void* dO, float* dK, float* dV, const float* delta_ws, int32_t* status_word,
+int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
+                               const float* LSE, const void* dO, float* dK, float* dV, int32_t* status_word,
                                cudaStream_t st) {
   CUtensorMap mq, mdo, mk, mv;
-  const uint32_t box_q[5] = {64, 64, 1, 1, 1};
-  const uint32_t box_k[5] = {64, kKT, 2, 1, 1};
+  const uint32_t box[5] = {64, 64, 1, 1, 1};
   const uint64_t dq[5] = {64, (uint64_t)dm.S, 2, (uint64_t)dm.Hq, (uint64_t)dm.B};
   const uint64_t dk[5] = {64, (uint64_t)dm.L, 2, (uint64_t)dm.Hkv, (uint64_t)dm.B};
   const uint64_t sq[4] = {(uint64_t)dm.qs[2] * 2, 128, (uint64_t)dm.qs[1] * 2, (uint64_t)dm.qs[0] * 2};
   const uint64_t so[4] = {(uint64_t)dm.os[2] * 2, 128, (uint64_t)dm.os[1] * 2, (uint64_t)dm.os[0] * 2};
   const uint64_t sk[4] = {(uint64_t)dm.ks[2] * 2, 128, (uint64_t)dm.ks[1] * 2, (uint64_t)dm.ks[0] * 2};
   const uint64_t sv[4] = {(uint64_t)dm.vs[2] * 2, 128, (uint64_t)dm.vs[1] * 2, (uint64_t)dm.vs[0] * 2};
-  if (encode_tensor_map_bf16(&mq, Q, 5, dq, sq, box_q, true) ||
-      encode_tensor_map_bf16(&mdo, dO, 5, dq, so, box_q, true) ||
-      encode_tensor_map_bf16(&mk, K, 5, dk, sk, box_k, true) ||
-      encode_tensor_map_bf16(&mv, V, 5, dk, sv, box_k, true))
+  if (encode_tensor_map_bf16(&mq, Q, 5, dq, sq, box, true) ||
+      encode_tensor_map_bf16(&mdo, dO, 5, dq, so, box, true) ||
+      encode_tensor_map_bf16(&mk, K, 5, dk, sk, box, true) ||
+      encode_tensor_map_bf16(&mv, V, 5, dk, sv, box, true))
     return HGA_ERR_UNSUPPORTED;
   const size_t smem = sizeof(BandSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(k_attn_bwd_band_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return record_cuda(e);
-  const int units = dm.B * dm.Hkv * (dm.S / kKT);
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)units);
-  cfg.blockDim = dim3(kBandThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;   // behind the delta pre-pass of the same call
-  attr.val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = (dm.flags & kFlagNoPdl) ? 0 : 1;
-  e = cudaLaunchKernelEx(&cfg, k_attn_bwd_band_sm100, mq, mdo, mk, mv, delta_ws, LSE, dm, dK, dV, status_word);
-  count_launch(1);
-  return record_cuda(e);
+  const int units = dm.B * dm.Hkv * ((dm.S + kKeys - 1) / kKeys);
+  k_attn_bwd_band_sm100<<<units, kBandThreads, smem, st>>>(mq, mdo, mk, mv, (const uint16_t*)O, LSE, dm, dK, dV,
+                                                          status_word);
+  count_launch(HGA_KERNELS_BWD_TENSOR);
+  return record_cuda(cudaGetLastError());
 }
 
 }  // namespace hga

@@ -5,8 +5,9 @@
 // TMA gathers in 64-key tiles (8 octets) exactly as in the forward kernel.  Two kinds of steps:
 //
 //  * dK/dV steps (one 64-key tile each): tiles that hold keys whose dK/dV this kernel must add,
-//    i.e. keys of the active segment that were selected through routing (the local band is written
-//    by the key-major kernel k_attn_bwd_band_sm100; without it, every active key).  They come first:
+//    i.e. keys of the active segment that lie before the local band: selected through routing, or
+//    sink keys (the local band is written by the key-major kernel k_attn_bwd_band_sm100, which
+//    runs first and stores every row of dK/dV).  They come first:
 //      S = Q K^T, dP = dO V^T -> TMEM;  P, dS by one thread per row -> shared memory;
 //      dQ += dS K;  dV^T = dO^T P, dK^T = Q^T dS (M = head_dim, N = 64 keys, K = 128 rows) -> TMEM,
 //    then four reduction warps add the transposed tiles to global memory (a warp's 32 lanes hold 32
@@ -36,6 +37,9 @@
 // TMEM (512 columns): region 0 | region 2 (aliased by dV^T, dK^T during the dK/dV steps) | dQ |
 // region 1.  Shared memory: Q, dO (32 KB each), K ring of six 16 KB stages, V ring of two, P and dS
 // (16 KB each, used by the dK/dV steps only).
+// delta = rowsum(dO o O) of the CTA's 128 rows is computed during set-up by the row threads themselves
+// (the O row from global memory, the dO row from the tile in shared memory; the two warpgroups take
+// one 64-element half each), so no pass over O and dO precedes the kernel.
 #include "hga_bwd_sm100.cuh"
 #include "hga_common.cuh"
 #include "hga_octets.cuh"
@@ -71,26 +75,20 @@ struct BwdSmem {
   uint64_t kp_full[kBwdKStages / 2], kp_empty[kBwdKStages], vp_full;       // paired steps: one barrier per pair of stages
                                                         // (kp_empty: indexed by pair number mod 6, see dp_full)
   uint64_t dq_done, dq_staged;
+  float dpart[2][128];         // halves of delta = rowsum(dO o O), one per row-thread warpgroup
   uint32_t tmem_base;
   int n_oct, dkv_lo, n_dkv;    // tiles [dkv_lo, dkv_lo + n_dkv) are processed as dK/dV steps
   volatile int abort;
   int oct_row[1];
 };
 
-__device__ __forceinline__ float dot4_bf16(uint2 x, uint2 y) {
-  float s = __uint_as_float(x.x << 16) * __uint_as_float(y.x << 16);
-  s = fmaf(__uint_as_float(x.x & 0xffff0000u), __uint_as_float(y.x & 0xffff0000u), s);
-  s = fmaf(__uint_as_float(x.y << 16), __uint_as_float(y.y << 16), s);
-  s = fmaf(__uint_as_float(x.y & 0xffff0000u), __uint_as_float(y.y & 0xffff0000u), s);
-  return s;
-}
-
 __global__ void __launch_bounds__(kBwdThreads, 1)
 k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
                  const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                 const __grid_constant__ CUtensorMap map_dq, const float* __restrict__ delta_ws, const float* __restrict__ LSE, const int32_t* __restrict__ group_idx,
+                 const __grid_constant__ CUtensorMap map_dq, const uint16_t* __restrict__ O,
+                 const float* __restrict__ LSE, const int32_t* __restrict__ group_idx,
                  const int32_t* __restrict__ n_groups, Dims dm,
-                 float* __restrict__ dK, float* __restrict__ dV, int band_done, int32_t* status_word) {
+                 float* __restrict__ dK, float* __restrict__ dV, int32_t* status_word) {
   constexpr int D = kBwdD;
   // TMEM columns.  Regions 0, 1, 2 rotate through the roles S / dP+dS of the paired steps; a dK/dV
   // step keeps S (64 columns) and dP (64) in region 0 and dV^T, dK^T in region 1.
@@ -152,9 +150,9 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     bool bad;   // invalid entries are skipped exactly as in the forward kernel (which reports them)
     const int n_oct = build_octet_table(dm, w, group_idx + (int64_t)item * dm.width, n_groups + item, sm.oct_row, &bad);
     // Keys that receive dK/dV from this kernel: positions in [H, hi), where hi is the start of the
-    // local band when the key-major band kernel has already written that part, else no limit.
+    // local band (the key-major band kernel has written that part).
     // Rows ascend, so these octets are a contiguous range [oa, ob) of the list.
-    const int hi = band_done ? w.ls : 0x7fffffff;
+    const int hi = w.ls;
     int below_h = 0, below_hi = 0;
     for (int o = lane; o < n_oct; o += 32) {
       const int row = sm.oct_row[o];
@@ -173,14 +171,19 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       sm.n_dkv = ob > oa ? (ob + 7) / 8 - oa / 8 : 0;
     }
   }
-  // Row threads: LSE and delta = rowsum(dO o O) of the thread's own row (delta comes from a
-  // coalesced pre-pass, k_bwd_delta_sm100).  Loaded here so the latency hides behind the set-up.
-  float delta = 0.f, row_lse = 0.f;
+  // Row threads: LSE of the thread's own row, and the half of its O row (64 elements: warpgroup 0 the
+  // first half, warpgroup 1 the second) that its share of delta = rowsum(dO o O) needs.  Requested here
+  // so the latency hides behind the set-up.
+  float row_lse = 0.f;
+  uint4 o_half[8];
   if (warp >= 2 && warp < 10) {
     const int r = mt * 128 + (warp & 3) * 32 + lane;
-    const int64_t row = ((int64_t)b * dm.Hq + h * dm.G + r / dm.Bq) * dm.S + qb * dm.Bq + r % dm.Bq;
-    delta = delta_ws[row];
-    row_lse = LSE[row];
+    const int hq = h * dm.G + r / dm.Bq, srow = qb * dm.Bq + r % dm.Bq;
+    row_lse = LSE[((int64_t)b * dm.Hq + hq) * dm.S + srow];
+    const uint4* op = reinterpret_cast<const uint4*>(O + b * dm.os[0] + hq * dm.os[1] + (int64_t)srow * dm.os[2]) +
+                      8 * ((warp - 2) >> 2);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o_half[i] = __ldg(op + i);
   }
   __syncwarp();
   tc_fence_before_sync();
@@ -198,7 +201,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   // one contiguous operand), so after an odd number of dK/dV steps one slot passes unused: the
   // producers complete its full barriers without a copy, the MMA thread releases it at once.
   const int n_act_even = n_pairs > 0 ? (n_act + 1) & ~1 : n_act;
-  const int red_hi = band_done ? w.ls : 0x7fffffff;
+  const int red_hi = w.ls;
   // Step order: the dK/dV tiles first (descending), so their atomics drain while the rest is
   // computed; then every other tile, descending.
   auto tile_of_step = [&](int s) {
@@ -437,9 +440,31 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
     const float sl2 = dm.scale * 1.4426950408889634f;
     const float neg_lse2 = -row_lse * 1.4426950408889634f;
-    const float neg_delta_s = -delta * dm.scale;
+    // delta: this warpgroup's 64-element half of the row's dot product (dO from the tile in shared memory:
+    // panel wg, 128-byte line of the row, 16-byte chunks XOR-swizzled), then the sum of the two halves
+    bool ok = __all_sync(0xffffffffu, bwd_wait(&sm.q_full, 0, abort));
+    {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      if (ok) {
+        const uint32_t line = smem_u32(sm.dO) + (uint32_t)wg * 16384 + (uint32_t)row_in_tile * 128;
+        const uint32_t key7 = (uint32_t)(row_in_tile & 7);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          uint32_t y0, y1, y2, y3;
+          ld_shared_v4(line + (((uint32_t)i ^ key7) * 16), y0, y1, y2, y3);
+          const uint32_t xs[4] = {o_half[i].x, o_half[i].y, o_half[i].z, o_half[i].w}, ys[4] = {y0, y1, y2, y3};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            acc[e] = fmaf(__uint_as_float(xs[e] << 16), __uint_as_float(ys[e] << 16), acc[e]);
+            acc[e] = fmaf(__uint_as_float(xs[e] & 0xffff0000u), __uint_as_float(ys[e] & 0xffff0000u), acc[e]);
+          }
+        }
+      }
+      sm.dpart[wg][row_in_tile] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    }
+    asm volatile("bar.sync 3, 256;" ::: "memory");           // the 256 row threads (reached on every path)
+    const float neg_delta_s = -(sm.dpart[0][row_in_tile] + sm.dpart[1][row_in_tile]) * dm.scale;
     HGA_TRACE_POINT(10);
-    bool ok = true;
     if (wg == 0) {
       // ---- dK/dV steps (warpgroup 0): P and dS go to shared memory as operands of dV^T / dK^T / dQ
       // this row's 128-byte line inside the P / dS buffers, and its swizzle key
@@ -633,42 +658,6 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
-// delta[row] = sum_e dO[row][e] * O[row][e]: one warp per row, 8-byte loads (a 256-byte row per
-// request), an HBM stream of O and dO at full-GPU bandwidth.
-__global__ void __launch_bounds__(256)
-k_bwd_delta_sm100(const uint16_t* __restrict__ O, const uint16_t* __restrict__ dO, Dims dm,
-                  float* __restrict__ delta) {
-  // half a warp per row (16 lanes x 16 bytes = one 256-byte row), 8 rows per warp in flight
-  const int lane = threadIdx.x & 31, sub = lane >> 4, chunk = lane & 15;
-  const int64_t n_rows = (int64_t)dm.B * dm.Hq * dm.S;
-  const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-  pdl_launch_dependents();      // the band kernel behind this one may set itself up meanwhile (it waits before reading delta)
-  for (int64_t base = warp_id * 8; base < n_rows; base += n_warps * 8) {
-    uint4 x[4], y[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int64_t row = base + 2 * u + sub;
-      x[u] = y[u] = make_uint4(0, 0, 0, 0);
-      if (row < n_rows) {
-        const int s = row % dm.S, hq = (row / dm.S) % dm.Hq, b = row / ((int64_t)dm.S * dm.Hq);
-        const int64_t off = b * dm.os[0] + hq * dm.os[1] + (int64_t)s * dm.os[2] + chunk * 8;
-        x[u] = *reinterpret_cast<const uint4*>(O + off);
-        y[u] = *reinterpret_cast<const uint4*>(dO + off);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      float part = dot4_bf16(make_uint2(x[u].x, x[u].y), make_uint2(y[u].x, y[u].y)) +
-                   dot4_bf16(make_uint2(x[u].z, x[u].w), make_uint2(y[u].z, y[u].w));
-#pragma unroll
-      for (int o = 8; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-      const int64_t row = base + 2 * u + sub;
-      if (chunk == 0 && row < n_rows) delta[row] = part;
-    }
-  }
-}
-
 bool attn_bwd_sm100_supported(const Dims& dm) {
   if (dm.flags & HGA_FLAG_GENERIC_KERNELS) return false;
   return dm.d == 128 && dm.rows % 128 == 0 && dm.g % 8 == 0 && dm.Bq % 64 == 0;
@@ -676,8 +665,9 @@ bool attn_bwd_sm100_supported(const Dims& dm) {
 
 int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
                           const float* LSE, const void* dO, const int32_t* group_idx,
-                          const int32_t* n_groups, void* dQ, float* dK, float* dV, float* delta_ws,
-                          bool zero_grads, int32_t* status_word, cudaStream_t st) {
+                          const int32_t* n_groups, void* dQ, float* dK, float* dV, int32_t* status_word,
+                          cudaStream_t st) {
+  if (!attn_bwd_band_sm100_supported(dm)) return HGA_ERR_UNSUPPORTED;
   CUtensorMap mq, mdo, mk, mv, mdq;
   const uint32_t box[5] = {64, 8, 2, 1, 1};
   const uint32_t box_q[5] = {64, 64, 1, 1, 1};
@@ -698,30 +688,14 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
   if (smem > 227 * 1024) return HGA_ERR_UNSUPPORTED;
   cudaError_t e = cudaFuncSetAttribute(k_attn_bwd_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return record_cuda(e);
-  const int64_t n_rows = (int64_t)dm.B * dm.Hq * dm.S;
-  // one block = 8 warps x 8 rows; a multiple of the SM count when there is enough work
-  const int64_t want_blocks = (n_rows + 63) / 64;
-  const int delta_blocks = (int)(want_blocks < 148 * 8 ? want_blocks : 148 * 8);
-  k_bwd_delta_sm100<<<delta_blocks, 256, 0, st>>>((const uint16_t*)O, (const uint16_t*)dO, dm, delta_ws);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return record_cuda(e);
-  // dK/dV of the local band: written once per key tile by the key-major kernel (plain stores that
-  // cover every row of the active segment), which also makes zero-filling unnecessary.  Where that
-  // kernel does not apply, this kernel adds every contribution atomically onto zeroed buffers.
-  int band_done = 0;
-  if (attn_bwd_band_sm100_supported(dm)) {
-    const int rc = launch_attn_bwd_band_sm100(dm, Q, K, V, LSE, dO, dK, dV, delta_ws, status_word, st);
-    if (rc == HGA_OK) band_done = 1;
-    else if (rc != HGA_ERR_UNSUPPORTED) return rc;
-  }
-  if (!band_done && zero_grads) {
-    const size_t bytes = (size_t)dm.B * dm.Hkv * dm.S * dm.d * sizeof(float);
-    if ((e = cudaMemsetAsync(dK, 0, bytes, st)) != cudaSuccess) return record_cuda(e);
-    if ((e = cudaMemsetAsync(dV, 0, bytes, st)) != cudaSuccess) return record_cuda(e);
-  }
+  // dK/dV of the local band: written once per key tile by the key-major kernel, with plain stores that
+  // cover every row of the active segment (so nothing has to be zero-filled); this kernel then adds the
+  // contributions of the keys before the band atomically.
+  const int rc = launch_attn_bwd_band_sm100(dm, Q, K, V, O, LSE, dO, dK, dV, status_word, st);
+  if (rc != HGA_OK) return rc;
   const int units = dm.B * dm.Hkv * dm.NQB * (dm.rows / 128);
-  // After the band kernel the sweep is launched with programmatic serialization: its CTAs may start on
-  // SMs the band kernel's last wave leaves idle (they wait for it only before adding to dK/dV).
+  // The sweep is launched with programmatic serialization behind the band kernel: its CTAs may start on
+  // SMs the band kernel leaves idle (they wait for it only before adding to dK/dV).
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)units);
   cfg.blockDim = dim3(kBwdThreads);
@@ -731,10 +705,10 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
-  cfg.numAttrs = (band_done && !(dm.flags & kFlagNoPdl)) ? 1 : 0;
-  e = cudaLaunchKernelEx(&cfg, k_attn_bwd_sm100, mq, mdo, mk, mv, mdq, (const float*)delta_ws, LSE, group_idx, n_groups,
-                         dm, dK, dV, band_done, status_word);
-  count_launch(2);
+  cfg.numAttrs = (dm.flags & kFlagNoPdl) ? 0 : 1;
+  e = cudaLaunchKernelEx(&cfg, k_attn_bwd_sm100, mq, mdo, mk, mv, mdq, (const uint16_t*)O, LSE, group_idx, n_groups,
+                         dm, dK, dV, status_word);
+  count_launch(HGA_KERNELS_BWD_TENSOR);
   return record_cuda(e);
 }
 

@@ -434,7 +434,7 @@ static int launch_fwd(const Dims& dm, const void* Q, const void* K, const void* 
   const int units = dm.B * dm.Hkv * dm.NQB * ((rows_padded(dm) + 127) / 128);
   k_attn_fwd_sm100<D><<<units, kFwdThreads, smem, st>>>(mq, mk, mv, group_idx, n_groups, dm, (uint16_t*)O, LSE,
                                                        status_word);
-  count_launch();
+  count_launch(HGA_KERNELS_FWD_TENSOR);
   return record_cuda(cudaGetLastError());
 }
 

@@ -312,7 +312,7 @@ __global__ void __launch_bounds__(256) k_grads_to_bf16(const float4* __restrict_
 int launch_grads_to_bf16(const float* src, void* dst, size_t n, cudaStream_t st) {
   const size_t n8 = n / 8;
   k_grads_to_bf16<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>((const float4*)src, (uint4*)dst, n8);
-  count_launch();
+  count_launch(HGA_KERNELS_AUX);
   return record_cuda(cudaGetLastError());
 }
 
@@ -336,7 +336,7 @@ int launch_attn_fwd_generic(const Dims& dm, const void* Q, const void* K, const 
         (const uint16_t*)Q, (const uint16_t*)K, (const uint16_t*)V, group_idx, n_groups, dm,
         (uint16_t*)O, LSE, status_word);
   }
-  count_launch();
+  count_launch(HGA_KERNELS_FWD_GENERIC);
   return record_cuda(cudaGetLastError());
 }
 
@@ -353,15 +353,15 @@ static int bwd_generic(const Dims& dm, const uint16_t* Q, const uint16_t* K, con
   if (e != cudaSuccess) return record_cuda(e);
   const int64_t n_rows = (int64_t)dm.B * dm.Hq * dm.S;
   k_bwd_delta<D><<<(unsigned)((n_rows + kAttnWarps - 1) / kAttnWarps), kAttnThreads, 0, st>>>(O, dO, dm, delta);
-  count_launch();
+  count_launch(HGA_KERNELS_BWD_GENERIC);
   int rc = record_cuda(cudaGetLastError());
   if (rc) return rc;
   k_bwd_dq_generic<D><<<items, kAttnThreads, smem, st>>>(Q, K, V, dO, LSE, delta, group_idx, n_groups, dm, dQ, status_word);
-  count_launch();
+  count_launch(HGA_KERNELS_BWD_GENERIC);
   rc = record_cuda(cudaGetLastError());
   if (rc) return rc;
   k_bwd_dkv_generic<D><<<items, kAttnThreads, smem, st>>>(Q, K, V, dO, LSE, delta, group_idx, n_groups, dm, dK, dV);
-  count_launch();
+  count_launch(HGA_KERNELS_BWD_GENERIC);
   return record_cuda(cudaGetLastError());
 }
 

@@ -14,9 +14,10 @@ __host__ __device__ inline int score_agg_of(int flags) {
   return (flags & HGA_FLAG_SCORE_MEAN) ? 1 : (flags & HGA_FLAG_SCORE_LSE) ? 2 : 0;
 }
 
-// Internal flag (a bit of hga_params.flags that hga.h does not define): launch the backward's kernels
-// without programmatic serialization.  Set by hga_step_host, whose steps are bound by the host link: there
-// the early-started CTAs only get in the way of the next (batch, kv head) pair's kernels.
+// Internal flag (a bit of Dims.flags that hga.h does not define and the exported calls reject): launch
+// the backward's kernels without programmatic serialization.  Set by hga_step_host, whose steps are bound
+// by the host link: there the early-started CTAs only get in the way of the next (batch, kv head) pair's
+// kernels.
 constexpr int kFlagNoPdl = 1 << 30;
 
 // Resolved problem description handed to kernels by value.
@@ -69,7 +70,7 @@ __host__ __device__ inline int max_routed_tokens(const Dims& dm) {
 }
 
 // Launch bookkeeping (hga_api.cu).
-void count_launch(int n = 1);
+void count_launch(int family, int n = 1);   // family: HGA_KERNELS_*
 int record_cuda(cudaError_t e);  // returns HGA_OK or HGA_ERR_CUDA and remembers the code
 
 // Kernel launchers, one per translation unit.  All return an HGA status.
@@ -100,12 +101,12 @@ int launch_route_sm100(const Dims& dm, const void* Q, const void* chunk_sum, con
 bool attn_bwd_sm100_supported(const Dims& dm);
 int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
                           const float* LSE, const void* dO, const int32_t* group_idx,
-                          const int32_t* n_groups, void* dQ, float* dK, float* dV, float* delta_ws,
-                          bool zero_grads, int32_t* status_word, cudaStream_t st);
-// Key-major dK/dV of the local band (plain stores covering every active-segment row).
+                          const int32_t* n_groups, void* dQ, float* dK, float* dV, int32_t* status_word,
+                          cudaStream_t st);
+// Key-major dK/dV of the local band (plain stores covering every active-segment row); launched by the above.
 bool attn_bwd_band_sm100_supported(const Dims& dm);
-int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const float* LSE,
-                               const void* dO, float* dK, float* dV, const float* delta_ws, int32_t* status_word,
+int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
+                               const float* LSE, const void* dO, float* dK, float* dV, int32_t* status_word,
                                cudaStream_t st);
 
 // Validates an hga_params block and fills the resolved description (hga_api.cu).

@@ -325,21 +325,21 @@ int launch_route_generic(const Dims& dm, const void* Q, const void* chunk_sum,
       k_chunk_scores<128><<<grid, kScoreThreads, smem, st>>>(Qp, cs, dm, scores);
     else
       k_chunk_scores<64><<<grid, kScoreThreads, smem, st>>>(Qp, cs, dm, scores);
-    count_launch();
+    count_launch(HGA_KERNELS_ROUTE_GENERIC);
     int rc = record_cuda(cudaGetLastError());
     if (rc) return rc;
   } else if (chunk_scores) {
     // nothing to score: the optional output is still defined (-inf everywhere) by k_select_chunks
   }
   k_select_chunks<<<items, 256, 0, st>>>(scores, dm, chunk_idx, chunk_scores);
-  count_launch();
+  count_launch(HGA_KERNELS_ROUTE_GENERIC);
   int rc = record_cuda(cudaGetLastError());
   if (rc) return rc;
   if (dm.d == 128)
     k_route_groups<128><<<items, kScoreThreads, smem, st>>>(Qp, gs, dm, chunk_idx, group_idx, n_groups, group_scores, gscratch);
   else
     k_route_groups<64><<<items, kScoreThreads, smem, st>>>(Qp, gs, dm, chunk_idx, group_idx, n_groups, group_scores, gscratch);
-  count_launch();
+  count_launch(HGA_KERNELS_ROUTE_GENERIC);
   return record_cuda(cudaGetLastError());
 }
 

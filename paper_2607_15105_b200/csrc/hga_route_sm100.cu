@@ -40,6 +40,7 @@ struct RouteSmem {
   static constexpr int kTile = 128 * D * 2;
   alignas(1024) uint8_t a[STAGES][kTile];   // summary tiles (A operand)
   uint64_t q_full, a_full[STAGES], a_empty[STAGES], acc_full[ACCS], acc_free[ACCS];
+  uint64_t drain;              // give-up path only: completes when the tensor pipe has run dry
   uint32_t tmem_base;
   volatile int abort;
   int n_sel;
@@ -125,6 +126,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       mbar_init(&sm.q_full, 1);
       for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.a_full[s], 1); mbar_init(&sm.a_empty[s], 1); }
       for (int s = 0; s < ACCS; ++s) { mbar_init(&sm.acc_full[s], 1); mbar_init(&sm.acc_free[s], 128); }
+      mbar_init(&sm.drain, 1);
       sm.abort = 0;
       sm.n_sel = 0;
       fence_barrier_init();
@@ -454,10 +456,16 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     // count and use no routed groups for that item), and the copies still in flight get a bounded time to land
     // before the CTA's shared memory is released.
     if (tid == 0) n_groups[item] = -1;
-    if (warp == 0 && lane == 0) {
+    if (warp == 0 && lane == 0) {        // (tiles_issued is warp 0's own count)
       if (k_sel > 0) mbar_wait(&sm.q_full, 0);
       for (int tg = tiles_issued > STAGES ? tiles_issued - STAGES : 0; tg < tiles_issued; ++tg)
         mbar_wait(&sm.a_full[tg % STAGES], (tg / STAGES) & 1);
+    }
+    if (warp == 1 && lane == 0) {
+      // GEMMs this thread issued may still be writing tensor memory: a commit completes once every
+      // earlier MMA of the thread has, so wait for one (bounded) before the columns are given back
+      mma_commit(&sm.drain);
+      mbar_wait(&sm.drain, 0);
     }
   }
   __syncwarp();
@@ -522,7 +530,7 @@ static int launch_route(const Dims& dm, const void* Q, const void* chunk_sum, co
   const int items = dm.B * dm.Hkv * dm.NQB;
   k_route_sm100<D, STAGES, ACCS><<<items, kRtThreads, smem, st>>>(mq, mc, mg, dm, chunk_idx, group_idx, n_groups, chunk_scores,
                                                    group_scores, ((rows_padded(dm) + 31) & ~31) * D * 2, max_cand);
-  count_launch();
+  count_launch(HGA_KERNELS_ROUTE_TENSOR);
   return record_cuda(cudaGetLastError());
 }
 

@@ -5,8 +5,11 @@
 // framework's allocator is locked or has handed out all device memory, a latency-critical
 // loop that must never enter cudaMalloc (it synchronises the whole device), a process whose
 // device memory was budgeted to the last byte at start-up.  For them the scratch lives here,
-// in a fixed array that is part of the library image: every GPU on which the library is
-// loaded holds HGA_ROUTE_STATIC_SCRATCH_BYTES of it until the process exits.
+// in a fixed array that is part of the library image: every GPU that has run this entry point
+// holds HGA_ROUTE_STATIC_SCRATCH_BYTES of it until the process exits.  (CUDA loads a module's
+// device data when something in the module is first used, so the array becomes resident with
+// the address look-up of the first call on a device -- that first call is the one moment at
+// which this entry point makes the driver reserve device memory.)
 #include <mutex>
 
 #include "hga_common.cuh"
@@ -53,11 +56,19 @@ extern "C" int hga_route_static(const hga_params* p, const void* Q, const void* 
   if (dm.kc > 0 && (!chunk_idx || !group_idx)) return HGA_ERR_NULL;
   auto misaligned = [](const void* x) { return (reinterpret_cast<uintptr_t>(x) & 15) != 0; };
   if (misaligned(Q) || misaligned(chunk_sum) || misaligned(group_sum)) return HGA_ERR_ALIGN;
-  // the fixed array bounds the problem size: refuse anything larger, launch nothing
+  // the fixed array bounds the problem size: refuse anything larger, launch nothing (also where the
+  // fused router below would not need the array, so that the limit does not depend on the shape)
   if (route_workspace_bytes(dm) > (size_t)HGA_ROUTE_STATIC_SCRATCH_BYTES) return HGA_ERR_WORKSPACE;
   void* scratch = nullptr;
   rc = scratch_on_current_device(&scratch);
   if (rc) return rc;
+  // Shapes the fused tensor-core router takes keep every score on chip: it runs first, as in
+  // hga_route, and the array stays untouched.  Other shapes go to the CUDA-core router below.
+  if (route_sm100_supported(dm)) {
+    rc = launch_route_sm100(dm, Q, chunk_sum, group_sum, chunk_idx, group_idx, n_groups, nullptr, nullptr,
+                            (cudaStream_t)stream);
+    if (rc != HGA_ERR_UNSUPPORTED) return rc;
+  }
   // Every score the selection kernels read is written earlier in the same call, so nothing in
   // the array has to start at zero and the previous call's contents are simply overwritten.
   return launch_route_generic(dm, Q, chunk_sum, group_sum, chunk_idx, group_idx, n_groups, nullptr,

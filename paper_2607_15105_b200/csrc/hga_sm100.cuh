@@ -69,14 +69,16 @@ constexpr long long kWaitCycles = 1ll << 30;
 
 // One bounded wait shared by the kernels: polls until the phase completes, the CTA's abort flag is
 // seen (checked every 64 polls), or the time limit runs out (then sets the flag).  abort may be null.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort) {
+// limit_cycles: the kernels use the default; the self-test kernel passes a short one.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort,
+                                                  long long limit_cycles = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t i = 0; i < kWaitLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 63u) {
       if (abort && *abort) return false;
-      if (clock64() - t0 > kWaitCycles) break;
+      if (clock64() - t0 > limit_cycles) break;
     }
   }
   if (abort) *abort = 1;

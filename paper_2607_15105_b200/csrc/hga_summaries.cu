@@ -95,7 +95,7 @@ int launch_build_summaries(const Dims& dm, const void* K, int tok_begin, int tok
     k_build_summaries<128><<<grid, block, smem, st>>>(Kp, dm, tok_begin / dm.c, cs, gs);
   else
     k_build_summaries<64><<<grid, block, smem, st>>>(Kp, dm, tok_begin / dm.c, cs, gs);
-  count_launch();
+  count_launch(HGA_KERNELS_SUMMARIES);
   return record_cuda(cudaGetLastError());
 }
 

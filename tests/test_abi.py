@@ -107,6 +107,8 @@ def test_flag_rules_on_the_host(lib):
     assert ok(binding.HGA_FLAG_SCORE_MEAN) == 0 and ok(binding.HGA_FLAG_SCORE_LSE) == 0
     assert ok(binding.HGA_FLAG_SCORE_MEAN | binding.HGA_FLAG_SCORE_LSE) == -4      # at most one aggregator
     assert ok(1 << 9) == -4                                                          # unknown flag bit
+    for bit in range(7, 32):                                                         # every bit hga.h does not define
+        assert ok(1 << bit if bit < 31 else -(1 << 31)) == -4, bit
     # generation shapes need their flag: q_block below the chunk, unaligned history and length
     dec = replace(cfg, total_len=1003, seg_len=3, q_block=3)
     assert ok(0, dec) == -2

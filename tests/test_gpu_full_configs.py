@@ -9,8 +9,8 @@ import oracle
 from paper_2607_15105_b200 import binding
 from paper_2607_15105_b200.workloads import CONFIGS, make_inputs
 
-from hga_testlib import (TOL_GRAD, TOL_LSE, TOL_O, bf16_to_f64, bits_of, check_routing, item_rows,
-                         rel_fro, to_dev)
+from hga_testlib import (TOL_GRAD, TOL_GRAD_ROW, TOL_LSE, TOL_O, bf16_to_f64, bits_of, check_routing,
+                         item_rows, rel_fro, row_err_ratio, to_dev)
 
 pytestmark = pytest.mark.gpu
 
@@ -27,6 +27,8 @@ def sample_items(cfg, full_head, extra, seed):
 
 # routed keys per item (a data-independent count) for the last query block of each config
 ROUTED_KEYS_LAST_BLOCK = {1: 320, 2: 512, 3: 768, 4: 768, 5: 2560, 6: 768}
+# per configuration: (items that may carry an excused chunk, chunks that may carry an excused group)
+EXCUSED_BOUNDS = {1: (1, 1), 2: (2, 2), 3: (2, 2), 4: (2, 2), 5: (8, 8), 6: (2, 2)}
 
 
 @pytest.mark.parametrize("n,full_head,extra", [(1, (0, 0), 4), (2, (0, 5), 12), (3, (0, 3), 12),
@@ -39,9 +41,19 @@ def test_config_against_oracle(n, full_head, extra):
     buf = binding.HgaLayerBuffers(cfg, backward=cfg.backward)
     # history summaries come from earlier segments; the step itself adds the active range
     buf.build_summaries(K, 0, cfg.history)
+    before = binding.hga_kernel_launch_counts()
     buf.step(Q, K, V, dO)
     torch.cuda.synchronize()
     assert int(buf.status.item()) == 0
+    # which kernels ran: the tensor-core router and forward on every configuration, the tensor-core
+    # backward wherever head_dim is 128 (configuration 1 has head_dim 64: its backward is the CUDA-core one)
+    ran = [b - a for a, b in zip(before, binding.hga_kernel_launch_counts())]
+    T = binding
+    assert ran[T.HGA_KERNELS_ROUTE_TENSOR] == 1 and ran[T.HGA_KERNELS_ROUTE_GENERIC] == 0, ran
+    assert ran[T.HGA_KERNELS_FWD_TENSOR] == 1 and ran[T.HGA_KERNELS_FWD_GENERIC] == 0, ran
+    if cfg.backward:
+        tensor_bwd = cfg.head_dim == 128
+        assert (ran[T.HGA_KERNELS_BWD_TENSOR] >= 2) == tensor_bwd and (ran[T.HGA_KERNELS_BWD_GENERIC] == 0) == tensor_bwd, ran
     head, items = sample_items(cfg, full_head, extra, seed=n)
     if n == 4:
         head, items = [], head[::2]          # forward only: 16 items are plenty
@@ -55,7 +67,11 @@ def test_config_against_oracle(n, full_head, extra):
     ref = oracle.route(cfg, x["Q"], cs, gs, items=items, want_scores=True)
     gi, ng = buf.group_idx.cpu().numpy(), buf.n_groups.cpu().numpy()
     checked, ec, eg = check_routing(cfg, ref, buf.chunk_idx.cpu().numpy(), gi, ng, items=items)
-    assert ec <= max(2, checked // 4), (checked, ec, eg)
+    print("config %d: %d items checked, %d with an excused chunk, %d chunks with an excused group" % (n, checked, ec, eg))
+    # near ties (score gap < 1e-3 at the k-th place) are rare where keys have topic structure; the i.i.d.
+    # configuration 5 is the near-tie-heavy one (about one block in ten has such a gap at the chunk level)
+    max_ec, max_eg = EXCUSED_BOUNDS[n]
+    assert ec <= max_ec and eg <= max_eg, (checked, ec, eg)
     # data-independent counts, everywhere
     keys = cfg.sink + ng[:, :, -1] * cfg.group + cfg.local + cfg.q_block
     assert np.all(keys == ROUTED_KEYS_LAST_BLOCK[n])
@@ -73,9 +89,12 @@ def test_config_against_oracle(n, full_head, extra):
     rest = sorted(set(items) - set(head))
     if rest:
         dQ += oracle.attn_bwd(cfg, x["Q"], x["K"], x["V"], x["dO"], gi, ng, items=rest)[0]   # disjoint rows
-    assert rel_fro(bf16_to_f64(buf.dQ)[bi, hi, si], dQ[bi, hi, si]) <= TOL_GRAD
-    assert rel_fro(buf.dK[b, h].cpu().numpy().astype(np.float64), dKo[b, h]) <= TOL_GRAD
-    assert rel_fro(buf.dV[b, h].cpu().numpy().astype(np.float64), dVo[b, h]) <= TOL_GRAD
+    for name, got, want in (("dQ", bf16_to_f64(buf.dQ)[bi, hi, si], dQ[bi, hi, si]),
+                            ("dK", buf.dK[b, h].cpu().numpy().astype(np.float64), dKo[b, h]),
+                            ("dV", buf.dV[b, h].cpu().numpy().astype(np.float64), dVo[b, h])):
+        fro, row = rel_fro(got, want), row_err_ratio(got, want)
+        print("config %d %s: rel. Frobenius %.2e, row ratio %.2f" % (n, name, fro, row))
+        assert fro <= TOL_GRAD and row <= TOL_GRAD_ROW, (name, fro, row)
     # rows of the active segment that no query block routes to get exactly zero
     H = cfg.history
     touched = np.zeros(cfg.seg_len, bool)

@@ -9,8 +9,8 @@ import oracle
 from paper_2607_15105_b200 import binding
 from paper_2607_15105_b200.workloads import CONFIGS, HgaConfig, bf16_bits_to_f64, make_inputs
 
-from hga_testlib import (TOL_GRAD, TOL_LSE, TOL_O, bf16_to_f64, bits_of, check_routing, item_rows,
-                         rel_fro, to_dev)
+from hga_testlib import (TOL_GRAD, TOL_LSE, TOL_O, bf16_to_f64, bits_of, check_grads, check_routing,
+                         item_rows, rel_fro, to_dev)
 
 pytestmark = pytest.mark.gpu
 
@@ -126,9 +126,8 @@ def test_attention_fwd_bwd_on_oracle_indices(name, flags):
     dQ, dK, dV = oracle.attn_bwd(cfg, x["Q"], x["K"], x["V"], x["dO"], c.ref["group_idx"], c.ref["n_groups"])
     assert np.max(np.abs(bf16_to_f64(buf.O) - O)) <= TOL_O
     assert np.max(np.abs(buf.LSE.cpu().numpy().astype(np.float64) - LSE)) <= TOL_LSE
-    assert rel_fro(bf16_to_f64(buf.dQ), dQ) <= TOL_GRAD
-    assert rel_fro(buf.dK.cpu().numpy().astype(np.float64), dK) <= TOL_GRAD
-    assert rel_fro(buf.dV.cpu().numpy().astype(np.float64), dV) <= TOL_GRAD
+    check_grads((bf16_to_f64(buf.dQ), buf.dK.cpu().numpy().astype(np.float64),
+                 buf.dV.cpu().numpy().astype(np.float64)), (dQ, dK, dV), name)
 
 
 @pytest.mark.parametrize("flags", FLAG_SETS)

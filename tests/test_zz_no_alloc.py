@@ -78,6 +78,40 @@ def _same_up_to_near_ties(cfg, ref, ci, gi, gap=1e-3):
                 assert all(abs(s[m - j * per] - kth) < gap for m in ca ^ cb), (it, j, ca ^ cb)
 
 
+def test_static_route_allocates_nothing_after_its_first_call():
+    """The first call on a device makes CUDA place the library's fixed array in device memory; from the
+    second call on, the free device memory is the same before and after a call (no allocation, no free),
+    on a shape the fused router takes and on one that needs the array."""
+    small = HgaConfig("static_small", 2, 4, 2, 128, 1536, 512, 64, 8, 64, 5, 3, 64, 128,
+                      topics=16, needles=4, backward=False, seed=23)
+    odd = HgaConfig("static_g16", 1, 2, 1, 64, 1024, 256, 64, 16, 64, 4, 2, 64, 64,
+                    topics=8, needles=0, backward=False, seed=24)     # 4 groups per chunk: CUDA-core router + the array
+    for cfg in (small, odd):
+        x = make_inputs(cfg, with_dO=False)
+        Q, K = _dev(x["Q"]), _dev(x["K"])
+        buf = binding.HgaLayerBuffers(cfg, backward=False)
+        buf.build_summaries(K, 0, cfg.total_len)
+        call = lambda: binding.hga_route_static(buf.p, Q, buf.chunk_sum, buf.group_sum, buf.chunk_idx,
+                                                buf.group_idx, buf.n_groups)
+        before = binding.hga_kernel_launch_counts()
+        call()                                   # may be the device's first call: set-up happens here
+        torch.cuda.synchronize()
+        ran = [b - a for a, b in zip(before, binding.hga_kernel_launch_counts())]
+        tensor = cfg is small
+        assert (ran[binding.HGA_KERNELS_ROUTE_TENSOR] == 1) == tensor, ran
+        assert (ran[binding.HGA_KERNELS_ROUTE_GENERIC] > 0) == (not tensor), ran
+        free0 = torch.cuda.mem_get_info()[0]
+        for _ in range(3):
+            call()
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free0
+        buf.route(Q)                             # hga_route with a caller workspace selects the same
+        ref = (buf.chunk_idx.clone(), buf.group_idx.clone(), buf.n_groups.clone())
+        call()
+        torch.cuda.synchronize()
+        assert all(torch.equal(a, b) for a, b in zip(ref, (buf.chunk_idx, buf.group_idx, buf.n_groups)))
+
+
 def test_static_route_refuses_problems_beyond_its_array():
     # 8 sequences of the 128K evaluation shape need 16 MiB of scores: more than the fixed array
     big = CONFIGS[4].scaled(batch=8)
