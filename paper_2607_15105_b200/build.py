@@ -61,4 +61,6 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--debug-waits" in sys.argv:      # diagnostic build: see csrc/hga_bwd_sm100.cuh
+        NVCC_FLAGS.append("-DHGA_DEBUG_WAIT")
+    print(build_library(force="--force" in sys.argv or "--debug-waits" in sys.argv, verbose="-v" in sys.argv))

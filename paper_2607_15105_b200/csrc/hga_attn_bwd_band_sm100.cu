@@ -17,12 +17,12 @@
 //   dV  += P^T dO,  dK += dS^T Q         (M = 128 keys, N = head_dim, K = 128 query rows)  A from TMEM
 // All of them are M = 128, N = 128 instructions (full tensor-pipe rate).
 // delta = rowsum(dO o O) of the M-tile's rows is computed here, by four otherwise idle warps (one
-// thread per query row: its O row from global memory, its dO row from the tile in shared memory), so
-// the backward needs no separate pass over O and dO.
+// thread per query row, from the O and dO tiles in shared memory; the O tile arrives by TMA one step
+// ahead), so the backward needs no separate pass over O and dO.
 //
 // Work unit (one CTA): (batch, kv head, 128-key tile of the active segment); keys past the end of the
 // segment arrive as zeros, are masked by causality and are not stored.
-// Warp roles (448 threads): warp 0 producer (K, V once; Q, dO tiles through a two-stage ring),
+// Warp roles (448 threads): warp 0 producer (K, V once; Q, dO tiles through a two-stage ring, O tiles one at a time),
 // warp 1 MMA issuer, warps 2-5 and 6-9 one thread per key (warpgroup w: query rows 64w .. 64w+63 of
 // the M-tile), warps 10-13 row statistics (LSE, delta).
 // TMEM (512 columns): S^T / P^T | dP^T / dS^T | dV | dK, 128 columns each.
@@ -46,9 +46,10 @@ struct BandSmem {
   alignas(1024) uint8_t v[kTile];
   alignas(1024) uint8_t q[2][kTile];
   alignas(1024) uint8_t dO[2][kTile];
-  alignas(16) float nlse[2][128];                // per query row of the M-tile in a stage: -LSE * log2(e)
-  alignas(16) float nds[2][128];                 //                                         -delta * scale
-  uint64_t kv_full, qdo_full[2], qdo_empty[2], stat_full[2];
+  alignas(1024) uint8_t o[kTile];                // (q, dO and o, contiguous, also stage the dV / dK tiles on their way out)
+  alignas(16) float nlse[128];                   // per query row of the current M-tile: -LSE * log2(e)
+  alignas(16) float nds[128];                    //                                      -delta * scale
+  uint64_t kv_full, qdo_full[2], qdo_empty[2], o_full, o_empty, stat_full;
   uint64_t s_full, dp_full, pds_full, acc_done, drain;
   uint32_t tmem_base;
   volatile int abort;
@@ -64,7 +65,7 @@ struct Step {
 __global__ void __launch_bounds__(kBandThreads, 1)
 k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
                       const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                      const uint16_t* __restrict__ O, const float* __restrict__ LSE, Dims dm,
+                      const __grid_constant__ CUtensorMap map_o, const float* __restrict__ LSE, Dims dm,
                       float* __restrict__ dK, float* __restrict__ dV, int32_t* status_word) {
   constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
   extern __shared__ uint8_t smem_raw[];
@@ -90,8 +91,9 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
   if (tid == 0) {
     mbar_init(&sm.kv_full, 1);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.qdo_full[s], 1); mbar_init(&sm.qdo_empty[s], 1); mbar_init(&sm.stat_full[s], 128);
+      mbar_init(&sm.qdo_full[s], 1); mbar_init(&sm.qdo_empty[s], 1);
     }
+    mbar_init(&sm.o_full, 1); mbar_init(&sm.o_empty, 128); mbar_init(&sm.stat_full, 128);
     mbar_init(&sm.s_full, 1); mbar_init(&sm.dp_full, 1); mbar_init(&sm.pds_full, 256);
     mbar_init(&sm.acc_done, 1); mbar_init(&sm.drain, 1);
     sm.abort = 0;
@@ -116,29 +118,37 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
     // A copy is latency-bound per box, so every tile travels as four boxes of 64 rows x one 64-element
-    // panel (8 KB each), issued by eight lanes at once: lanes 0-3 K or Q, lanes 4-7 V or dO.
+    // panel (8 KB each), issued by up to twelve lanes at once: lanes 0-3 K or Q, lanes 4-7 V or dO, lanes 8-11 O.
     const int half = lane & 1, panel = (lane >> 1) & 1;
     const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
     if (lane == 0) {
       prefetch_tensormap(&map_q); prefetch_tensormap(&map_do);
-      prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
+      prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); prefetch_tensormap(&map_o);
       mbar_arrive_expect_tx(&sm.kv_full, 2 * kTile);
     }
     __syncwarp();
     if (lane < 4) tma_load_5d(sm.k + off, &map_k, &sm.kv_full, 0, k0 + 64 * half, panel, h, b);
     else if (lane < 8) tma_load_5d(sm.v + off, &map_v, &sm.kv_full, 0, k0 + 64 * half, panel, h, b);
     bool ok = true;
-    int issued = 0;
+    int issued = 0, o_issued = 0;
     for (int m = 0; m < n_steps; ++m) {
       const int st = m & 1;
       const Step sp = step_of(m);
       const int r = sp.r0 + 64 * half;
+      const int row = sp.qb * dm.Bq + r % dm.Bq, head = h * dm.G + r / dm.Bq;
+      // the O tile of step m: its single buffer is free once the statistics warps have read step m-1's
+      if (lane == 0 && m >= 1) ok = bwd_wait(&sm.o_empty, (m - 1) & 1, abort);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane == 0) mbar_arrive_expect_tx(&sm.o_full, kTile);
+      __syncwarp();
+      if (lane >= 8 && lane < 12) tma_load_5d(sm.o + off, &map_o, &sm.o_full, 0, row, panel, head, b);
+      o_issued = m + 1;
       if (lane == 0 && m >= 2) ok = bwd_wait(&sm.qdo_empty[st], ((m >> 1) - 1) & 1, abort);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       if (lane == 0) mbar_arrive_expect_tx(&sm.qdo_full[st], 2 * kTile);
       __syncwarp();
-      const int row = sp.qb * dm.Bq + r % dm.Bq, head = h * dm.G + r / dm.Bq;
       if (lane < 4) tma_load_5d(sm.q[st] + off, &map_q, &sm.qdo_full[st], 0, row, panel, head, b);
       else if (lane < 8) tma_load_5d(sm.dO[st] + off, &map_do, &sm.qdo_full[st], 0, row, panel, head, b);
       issued = m + 1;
@@ -148,10 +158,15 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
       // giving up: let the copies still in flight land before shared memory is released
       mbar_wait(&sm.kv_full, 0);
       for (int m = issued > 2 ? issued - 2 : 0; m < issued; ++m) mbar_wait(&sm.qdo_full[m & 1], (m >> 1) & 1);
+      if (o_issued > 0) mbar_wait(&sm.o_full, (o_issued - 1) & 1);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp runs this branch converged (waits included) and one elected lane issues: see mma_ss_w.
+    {
+      auto mma_wait = [&](uint64_t* bar, uint32_t parity, volatile int* ab) {
+        return __all_sync(0xffffffffu, bwd_wait(bar, parity, ab));
+      };
       constexpr uint32_t idesc_t = idesc_bf16_f32(128, 128, 0, 0);     // keys x rows: A, B K-major (head_dim runs along K)
       constexpr uint32_t idesc_g = idesc_bf16_f32(128, kD, 0, 1);      // keys x head_dim: A from TMEM, B MN-major
       // every tile is [panel][128 rows][128 B]: K-major with 8-row groups 1024 B apart and the second
@@ -167,7 +182,7 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
           const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;       // panel, then 32-byte K step
-          mma_ss(acc, desc_advance(a, off), desc_advance(bq, off), idesc_t, kk > 0);
+          mma_ss_w(acc, desc_advance(a, off), desc_advance(bq, off), idesc_t, kk > 0);
         }
       };
       // acc (keys x head_dim) += a (keys x rows, bf16 in TMEM: rows 0-63 at columns 0-31, rows 64-127 at
@@ -175,43 +190,43 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
       auto issue_g = [&](uint32_t acc, uint32_t a_tmem, uint64_t bmn, bool accumulate) {
 #pragma unroll
         for (int kk = 0; kk < 128 / 16; ++kk)
-          mma_ts(acc, a_tmem + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), desc_advance(bmn, kk * 2048), idesc_g,
+          mma_ts_w(acc, a_tmem + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), desc_advance(bmn, kk * 2048), idesc_g,
                  (accumulate || kk > 0));
       };
-      bool ok = bwd_wait(&sm.kv_full, 0, abort) && bwd_wait(&sm.qdo_full[0], 0, abort);
+      bool ok = mma_wait(&sm.kv_full, 0, abort) && mma_wait(&sm.qdo_full[0], 0, abort);
       if (ok) {
         tc_fence_after_sync();
         issue_t(tmem + kColS, k_k, q_k0);
-        mma_commit(&sm.s_full);
+        mma_commit_w(&sm.s_full);
         issue_t(tmem + kColDP, v_k, do_k0);
-        mma_commit(&sm.dp_full);
+        mma_commit_w(&sm.dp_full);
       }
       HGA_TRACE_POINT(3);
       for (int m = 0; m < n_steps && ok; ++m) {
         const uint32_t st = (uint32_t)(m & 1), st_n = st ^ 1u;
         const bool more = m + 1 < n_steps;
-        ok = bwd_wait(&sm.pds_full, m & 1, abort);               // P^T and dS^T of step m are in TMEM
+        ok = mma_wait(&sm.pds_full, m & 1, abort);               // P^T and dS^T of step m are in TMEM
         if (!ok) break;
         tc_fence_after_sync();
         HGA_TRACE_POINT(5);
         issue_g(tmem + kColDV, tmem + kColS, desc_advance(do_mn0, st * kTile), m > 0);
         if (more) {
           // S^T of the next M-tile overwrites P^T: the in-order tensor pipe runs it after the dV GEMM above
-          ok = bwd_wait(&sm.qdo_full[st_n], ((m + 1) >> 1) & 1, abort);
+          ok = mma_wait(&sm.qdo_full[st_n], ((m + 1) >> 1) & 1, abort);
           if (!ok) break;
           tc_fence_after_sync();
           issue_t(tmem + kColS, k_k, desc_advance(q_k0, st_n * kTile));
-          mma_commit(&sm.s_full);
+          mma_commit_w(&sm.s_full);
         }
         issue_g(tmem + kColDK, tmem + kColDP, desc_advance(q_mn0, st * kTile), m > 0);
-        mma_commit(&sm.qdo_empty[st]);                           // Q and dO of step m are consumed
+        mma_commit_w(&sm.qdo_empty[st]);                           // Q and dO of step m are consumed
         if (more) {
           issue_t(tmem + kColDP, v_k, desc_advance(do_k0, st_n * kTile));
-          mma_commit(&sm.dp_full);
+          mma_commit_w(&sm.dp_full);
         }
         HGA_TRACE_POINT(7);
       }
-      if (ok) mma_commit(&sm.acc_done);
+      if (ok) mma_commit_w(&sm.acc_done);
     }
   } else if (warp < 10) {
     // ------------------------------------------------------------------ one thread per key
@@ -225,7 +240,6 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
     const uint64_t sl2_2 = pack_f32x2(sl2, sl2), scale_2 = pack_f32x2(dm.scale, dm.scale);
     bool ok = true;
     for (int m = 0; m < n_steps; ++m) {
-      const int st = m & 1;
       const Step sp = step_of(m);
       const Window w = window_of(dm, sp.qb);
       // the warpgroup's 64 columns are 64 consecutive positions of one query head (Bq is a multiple of 64);
@@ -234,10 +248,10 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
       const int imin = (kp < w.ls || kp >= k_end) ? 64 : kp - qp0;       // first visible column (may be <= 0)
       const bool none = __all_sync(0xffffffffu, imin >= 64);
       const bool masked = __any_sync(0xffffffffu, imin > 0);
-      const uint32_t nlse_a = smem_u32(&sm.nlse[st][64 * wg]), nds_a = smem_u32(&sm.nds[st][64 * wg]);
+      const uint32_t nlse_a = smem_u32(&sm.nlse[64 * wg]), nds_a = smem_u32(&sm.nds[64 * wg]);
       uint32_t pk[32];                               // P of this key against 64 query rows, packed bf16
       ok = __all_sync(0xffffffffu, bwd_wait(&sm.s_full, m & 1, abort));
-      if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.stat_full[st], (m >> 1) & 1, abort));
+      if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.stat_full, m & 1, abort));
       if (!ok) break;
       tc_fence_after_sync();
       HGA_TRACE_POINT(11);
@@ -319,69 +333,73 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
     if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.acc_done, 0, abort));
     HGA_TRACE_POINT(20);
     if (ok) {
-      // epilogue: thread = key row; warpgroup 0 stores dV, warpgroup 1 dK (512 contiguous bytes per thread)
+      // epilogue: thread = key row; warpgroup 0 sends dV, warpgroup 1 dK.  A row (512 bytes) goes through
+      // shared memory (the Q / dO / O tiles, free now: every GEMM and every copy into them is complete) and
+      // leaves as one bulk copy, or one bulk add with the accumulate flag; rows are 528 bytes apart so that
+      // the 16-byte stores of a quarter warp fall into different banks
       tc_fence_after_sync();
+      constexpr uint32_t kRowPitch = kD * 4 + 16;
+      static_assert(2 * 128 * kRowPitch <= 5 * kTile, "staging area: q, dO and o tiles");
       const int srow = kt * kKeys + key;
       float* dst = (wg == 0 ? dV : dK) + ((int64_t)(b * dm.Hkv + h) * dm.S + srow) * kD;
       const uint32_t col = wg == 0 ? kColDV : kColDK;
-      const bool accumulate = dm.flags & HGA_FLAG_BWD_ACCUMULATE;
-      const bool real = srow < dm.S;
+      const uint32_t stage = smem_u32(sm.q[0]) + (uint32_t)(wg * 128 + key) * kRowPitch;
 #pragma unroll
       for (int c = 0; c < kD / 32; ++c) {
         uint32_t x[32];
         tmem_ld32(lane_base + col + 32 * c, x);
         tmem_wait_ld();
-        if (real) {
-          float4* d4 = reinterpret_cast<float4*>(dst + 32 * c);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            float4 val = make_float4(__uint_as_float(x[4 * i]), __uint_as_float(x[4 * i + 1]),
-                                     __uint_as_float(x[4 * i + 2]), __uint_as_float(x[4 * i + 3]));
-            if (accumulate) {
-              const float4 old = d4[i];
-              val.x += old.x; val.y += old.y; val.z += old.z; val.w += old.w;
-            }
-            d4[i] = val;
-          }
-        }
+        for (int i = 0; i < 8; ++i) st_shared_v4(stage + (uint32_t)(32 * c + 4 * i) * 4, x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
+      }
+      fence_proxy_async_smem();
+      if (srow < dm.S) {
+        if (dm.flags & HGA_FLAG_BWD_ACCUMULATE) bulk_reduce_add_f32(dst, stage, kD * 4);
+        else bulk_store(dst, stage, kD * 4);
+        tma_store_commit();
+        tma_store_wait_read();
       }
     }
   } else {
     // ------------------------------------------------------------------ row statistics, one thread per query row
     const int j = (warp - 10) * 32 + lane;           // row of the M-tile
     const uint32_t key7 = (uint32_t)(j & 7);
+    auto lse_of = [&](int m) {
+      const Step sp = step_of(m);
+      const int r = sp.r0 + j;
+      return LSE[((int64_t)b * dm.Hq + h * dm.G + r / dm.Bq) * dm.S + sp.qb * dm.Bq + r % dm.Bq];
+    };
+    float lse_next = lse_of(0);
     bool ok = true;
     for (int m = 0; m < n_steps; ++m) {
       const int st = m & 1;
-      const Step sp = step_of(m);
-      const int r = sp.r0 + j;
-      const int hq = h * dm.G + r / dm.Bq, srow = sp.qb * dm.Bq + r % dm.Bq;
-      // the O row (256 bytes) is requested before the tile's dO lands in shared memory
-      const uint4* orow = reinterpret_cast<const uint4*>(O + b * dm.os[0] + hq * dm.os[1] + (int64_t)srow * dm.os[2]);
-      uint4 o[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) o[i] = __ldg(orow + i);
-      const float lse = LSE[((int64_t)b * dm.Hq + hq) * dm.S + srow];
+      const float lse = lse_next;
+      if (m + 1 < n_steps) lse_next = lse_of(m + 1);
       ok = __all_sync(0xffffffffu, bwd_wait(&sm.qdo_full[st], (m >> 1) & 1, abort));
+      if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.o_full, m & 1, abort));
       if (!ok) break;
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
-      const uint32_t line = smem_u32(sm.dO[st]) + (uint32_t)j * 128;
+      const uint32_t do_line = smem_u32(sm.dO[st]) + (uint32_t)j * 128, o_line = smem_u32(sm.o) + (uint32_t)j * 128;
 #pragma unroll
       for (int i = 0; i < 16; ++i) {                 // 16-byte chunk i of the row: panel i / 8, chunk i % 8 (XOR-swizzled)
-        uint32_t y0, y1, y2, y3;
-        ld_shared_v4(line + (uint32_t)(i >> 3) * 16384 + (((uint32_t)(i & 7) ^ key7) * 16), y0, y1, y2, y3);
-        const uint32_t xs[4] = {o[i].x, o[i].y, o[i].z, o[i].w}, ys[4] = {y0, y1, y2, y3};
+        const uint32_t off = (uint32_t)(i >> 3) * 16384 + (((uint32_t)(i & 7) ^ key7) * 16);
+        uint32_t xs[4], ys[4];
+        ld_shared_v4(o_line + off, xs[0], xs[1], xs[2], xs[3]);
+        ld_shared_v4(do_line + off, ys[0], ys[1], ys[2], ys[3]);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           acc[e] = fmaf(__uint_as_float(xs[e] << 16), __uint_as_float(ys[e] << 16), acc[e]);
           acc[e] = fmaf(__uint_as_float(xs[e] & 0xffff0000u), __uint_as_float(ys[e] & 0xffff0000u), acc[e]);
         }
       }
+      mbar_arrive(&sm.o_empty);                      // the O tile may be overwritten by the next step's
       const float delta = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-      // (stage st was last read by the key threads in step m-2, which ended before this step's tile could land)
-      sm.nlse[st][j] = -lse * 1.4426950408889634f;
-      sm.nds[st][j] = -delta * dm.scale;
-      mbar_arrive(&sm.stat_full[st]);
+      // the key threads read the previous step's statistics until they hand its P^T and dS^T over
+      if (m > 0) ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_full, (m - 1) & 1, abort));
+      if (!ok) break;
+      sm.nlse[j] = -lse * 1.4426950408889634f;
+      sm.nds[j] = -delta * dm.scale;
+      mbar_arrive(&sm.stat_full);
     }
   }
   HGA_TRACE_POINT(30);
@@ -389,17 +407,17 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
   // every warp reconverges before the block barrier (a barrier reached by part of a warp would
   // count that warp as arrived)
   __syncwarp();
-  if (warp == 1 && lane == 0 && sm.abort) {
+  if (warp == 1 && sm.abort) {
     // giving up: GEMMs already issued may still be writing tensor memory; wait (bounded) until the
     // tensor pipe has run dry before the columns are given back
-    mma_commit(&sm.drain);
+    mma_commit_w(&sm.drain);
     mbar_wait(&sm.drain, 0);
   }
   __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
   HGA_TRACE_DUMP;
-  if (tid == 0 && sm.abort && status_word) atomicOr(status_word, HGA_STATUS_WAIT_TIMEOUT);
+  if (tid == 0 && sm.abort && status_word) atomicOr(status_word, HGA_ABORT_CODE(2, sm.abort));
   if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
@@ -411,7 +429,7 @@ bool attn_bwd_band_sm100_supported(const Dims& dm) {
 int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* O,
                                const float* LSE, const void* dO, float* dK, float* dV, int32_t* status_word,
                                cudaStream_t st) {
-  CUtensorMap mq, mdo, mk, mv;
+  CUtensorMap mq, mdo, mk, mv, mo;
   const uint32_t box[5] = {64, 64, 1, 1, 1};
   const uint64_t dq[5] = {64, (uint64_t)dm.S, 2, (uint64_t)dm.Hq, (uint64_t)dm.B};
   const uint64_t dk[5] = {64, (uint64_t)dm.L, 2, (uint64_t)dm.Hkv, (uint64_t)dm.B};
@@ -421,6 +439,7 @@ int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, con
   const uint64_t sv[4] = {(uint64_t)dm.vs[2] * 2, 128, (uint64_t)dm.vs[1] * 2, (uint64_t)dm.vs[0] * 2};
   if (encode_tensor_map_bf16(&mq, Q, 5, dq, sq, box, true) ||
       encode_tensor_map_bf16(&mdo, dO, 5, dq, so, box, true) ||
+      encode_tensor_map_bf16(&mo, O, 5, dq, so, box, true) ||
       encode_tensor_map_bf16(&mk, K, 5, dk, sk, box, true) ||
       encode_tensor_map_bf16(&mv, V, 5, dk, sv, box, true))
     return HGA_ERR_UNSUPPORTED;
@@ -428,8 +447,7 @@ int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, con
   cudaError_t e = cudaFuncSetAttribute(k_attn_bwd_band_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return record_cuda(e);
   const int units = dm.B * dm.Hkv * ((dm.S + kKeys - 1) / kKeys);
-  k_attn_bwd_band_sm100<<<units, kBandThreads, smem, st>>>(mq, mdo, mk, mv, (const uint16_t*)O, LSE, dm, dK, dV,
-                                                          status_word);
+  k_attn_bwd_band_sm100<<<units, kBandThreads, smem, st>>>(mq, mdo, mk, mv, mo, LSE, dm, dK, dV, status_word);
   count_launch(HGA_KERNELS_BWD_TENSOR);
   return record_cuda(cudaGetLastError());
 }

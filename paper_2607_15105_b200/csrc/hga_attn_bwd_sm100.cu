@@ -27,8 +27,9 @@
 //    (dQ(u) reads dS before S(u+2) overwrites it) free of barriers.
 //
 // Warp roles (512 threads): warp 0 copies K tiles and runs up to three pairs ahead, warps 14 and 15
-// copy V tiles (half of each tile; V has room for one pair only, refilled as soon as the dP GEMM of
-// the previous pair is done, so their issue time matters), warp 1 MMA issuer, warps 2-5 and 6-9
+// copy V tiles (half of each tile; in the paired steps V has room for two pairs -- its own two stages and
+// the P / dS tiles, idle by then -- each refilled as soon as the dP GEMM that read it is done: with one
+// pair only, the copy's latency sat between consecutive dP GEMMs), warp 1 MMA issuer, warps 2-5 and 6-9
 // one thread per query row (warpgroup 0: first tile of a pair and all dK/dV steps; warpgroup 1:
 // second tile of a pair; both write the dQ epilogue), warps 10-13 dK/dV reduction.
 // Every barrier hand-off costs the MMA thread a few hundred cycles and every tcgen05.commit about a
@@ -53,7 +54,7 @@ using namespace sm100;
 
 constexpr int kBwdThreads = 512;                // 16 warps: 128 registers per thread
 constexpr int kBwdKStages = 6;                  // K ring: three pairs (a K tile is held until its dQ GEMM)
-constexpr int kBwdVStages = 2;                  // V ring: one pair (a V tile is free once dP is done)
+constexpr int kBwdVStages = 2;                  // V ring of the dK/dV steps; the paired steps add the P / dS tiles as a second pair
 constexpr int kBwdD = 128;
 constexpr int kKT = 64;                         // keys per tile
 constexpr int kOct = 8 * kBwdD * 2;             // bytes of one octet of K/V/Q/dO rows (2 panels)
@@ -69,18 +70,20 @@ struct BwdSmem {
   alignas(1024) uint8_t ds[kPdsTile];           // (P and dS pass through shared memory only for dK/dV tiles)
   uint64_t q_full, k_full[kBwdKStages], k_empty[kBwdKStages], v_full[kBwdVStages], v_empty[kBwdVStages];
   uint64_t sdp_full, pds_full, dkv_full, dkv_free;      // dK/dV steps
-  uint64_t s_full[2], dp_full[4], ds_full;              // paired steps (S(u+1) is committed before step u is over: two barriers;
+  uint64_t s_full[2], dp_full[4], ds_full[2], s_read[2];   // paired steps (S(u+1) is committed before step u is over: two barriers;
                                                         // dP: four, so that a copy item taken ahead of time cannot mistake an older phase)
   uint64_t phase_a_done;                                // every GEMM of the dK/dV steps is complete
-  uint64_t kp_full[kBwdKStages / 2], kp_empty[kBwdKStages], vp_full;       // paired steps: one barrier per pair of stages
+  uint64_t kp_full[kBwdKStages / 2], kp_empty[kBwdKStages], vp_full[2];    // paired steps: one barrier per pair of stages
                                                         // (kp_empty: indexed by pair number mod 6, see dp_full)
   uint64_t dq_done, dq_staged;
-  float dpart[2][128];         // halves of delta = rowsum(dO o O), one per row-thread warpgroup
   uint32_t tmem_base;
   int n_oct, dkv_lo, n_dkv;    // tiles [dkv_lo, dkv_lo + n_dkv) are processed as dK/dV steps
   volatile int abort;
   int oct_row[1];
 };
+
+static_assert(kPdsTile == kKvTile && offsetof(BwdSmem, ds) == offsetof(BwdSmem, p) + kKvTile,
+              "the P and dS tiles double as one pair of V stages");
 
 __global__ void __launch_bounds__(kBwdThreads, 1)
 k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
@@ -114,12 +117,16 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     for (int s = 0; s < kBwdVStages; ++s) { mbar_init(&sm.v_full[s], 2); mbar_init(&sm.v_empty[s], 1); }   // two V producers
     mbar_init(&sm.sdp_full, 1); mbar_init(&sm.pds_full, 128);
     mbar_init(&sm.dkv_full, 1); mbar_init(&sm.dkv_free, 128);
-    mbar_init(&sm.s_full[0], 1); mbar_init(&sm.s_full[1], 1); mbar_init(&sm.ds_full, 256);
+    mbar_init(&sm.s_full[0], 1); mbar_init(&sm.s_full[1], 1);
+    // (two barriers each, used alternately: S(u+1) and dP(u+1) are issued before the MMA warp waits for the row
+    // threads' arrivals of pair u, so the row threads may finish pair u+1 -- and arrive again -- before that wait
+    // has observed pair u; with one barrier its phase would then be missed.  Pair u+2 cannot start before.)
+    for (int s = 0; s < 2; ++s) { mbar_init(&sm.ds_full[s], 256); mbar_init(&sm.s_read[s], 256); }
     for (int s = 0; s < 4; ++s) mbar_init(&sm.dp_full[s], 1);
     mbar_init(&sm.phase_a_done, 1);
     for (int s = 0; s < kBwdKStages / 2; ++s) mbar_init(&sm.kp_full[s], 1);
     for (int s = 0; s < kBwdKStages; ++s) mbar_init(&sm.kp_empty[s], 1);
-    mbar_init(&sm.vp_full, 2);
+    mbar_init(&sm.vp_full[0], 2); mbar_init(&sm.vp_full[1], 2);
     mbar_init(&sm.dq_done, 1); mbar_init(&sm.dq_staged, 256);
     sm.abort = 0;
     fence_barrier_init();
@@ -253,13 +260,16 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // completes ONE barrier per operand, so the MMA thread observes one barrier per operand and
     // pair.  Lanes 0-7 (K) / 0-3 (V): first tile, lanes 8-15 / 4-7: second tile.
     {
-      const int n_ps = n_stages / 2;
+      const int n_ps = kBwdKStages / 2;
       const int which = is_v ? lane >> 2 : lane >> 3;                     // tile of the pair
       const int oct_in_tile = is_v ? (warp == 14 ? 0 : 4) + (lane & 3) : lane & 7;
       const bool copy_lane = is_v ? lane < 8 : lane < 16;
       for (int p = 0; p < n_pairs && ok; ++p) {
-        const int ps = (n_act_even / 2 + p) % n_ps;
-        uint64_t* full = is_v ? &sm.vp_full : &sm.kp_full[ps];
+        // K: three pairs of stages, continuing the slot numbering.  V: two pairs, pair p in slot p & 1; slot 0
+        // is the V ring, slot 1 the P and dS tiles (adjacent, one K/V tile each), which only the dK/dV steps
+        // use otherwise.  A V pair is free once its dP GEMM is done, a K pair only after its dQ GEMM.
+        const int ps = is_v ? (p & 1) : (n_act_even / 2 + p) % n_ps;
+        uint64_t* full = is_v ? &sm.vp_full[ps] : &sm.kp_full[ps];
         const int s = n_act + 2 * p + which;                              // step (tile order)
         int row = dm.L;
         if (s < n_tiles) {
@@ -267,11 +277,13 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (o < n_oct) row = sm.oct_row[o];
         }
         if (lane == 0) {
-          if (p < n_ps) {
+          if (is_v) {
+            // first use: the dK/dV steps (which read V stages, P and dS) must be over; later: dP of pair p-2 is done
+            if (p < 2) { if (n_act > 0) ok = bwd_wait(&sm.phase_a_done, 0, abort); }
+            else ok = bwd_wait(&sm.dp_full[(p - 2) & 3], (uint32_t)((p - 2) >> 2) & 1, abort);
+          } else if (p < n_ps) {
             // first paired use of these stages: if a dK/dV step used them, those steps must be over
             if (2 * ps < n_act_even) ok = bwd_wait(&sm.phase_a_done, 0, abort);
-          } else if (is_v) {
-            ok = bwd_wait(&sm.dp_full[(p - 1) & 3], (uint32_t)((p - 1) >> 2) & 1, abort);   // dP of the previous pair has read the V stages
           } else {
             ok = bwd_wait(&sm.kp_empty[(n_act_even / 2 + p - 3) % kBwdKStages], (uint32_t)((p - 3) / kBwdKStages) & 1, abort);   // dQ of pair p-3 is done
           }
@@ -281,7 +293,8 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)(is_v ? 8 : 16) * kOct);
         __syncwarp();
         if (copy_lane)
-          tma_load_5d((is_v ? sm.v[2 * ps + which] : sm.k[2 * ps + which]) + oct_in_tile * kOct, map, full, 0, row, 0, h, b);
+          tma_load_5d((is_v ? (ps == 0 ? sm.v[0] : sm.p) + which * kKvTile : sm.k[2 * ps + which]) + oct_in_tile * kOct, map, full,
+                      0, row, 0, h, b);
         HGA_TRACE_POINT(2);
       }
     }
@@ -293,7 +306,11 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp runs this branch converged (waits included) and one elected lane issues: see mma_ss_w.
+    {
+      auto mma_wait = [&](uint64_t* bar, uint32_t parity, volatile int* ab) {
+        return __all_sync(0xffffffffu, bwd_wait(bar, parity, ab));
+      };
       constexpr uint32_t idesc_sdp = idesc_bf16_f32(128, kKT, 0, 0);       // rows x 64 keys, both K-major
       constexpr uint32_t idesc_sdp2 = idesc_bf16_f32(128, 2 * kKT, 0, 0);  // rows x 128 keys
       constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);          // dS K-major, K tile MN-major
@@ -306,22 +323,23 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const uint64_t do_mn = smem_desc_sw128(smem_u32(sm.dO), 16384, 1024);  // dO^T as MN-major A (dV^T)
       const uint64_t k_k0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, kOct);    // K tile(s), K-major B  (S)
       const uint64_t v_k0 = smem_desc_sw128(smem_u32(sm.v[0]), 16, kOct);    // V tile(s), K-major B  (dP)
+      const uint64_t v_k1 = smem_desc_sw128(smem_u32(sm.p), 16, kOct);       // second V pair of the paired steps (P, dS tiles)
       const uint64_t k_mn0 = smem_desc_sw128(smem_u32(sm.k[0]), 1024, kOct); // K tile(s), MN-major B (dQ)
       const uint64_t dsd = smem_desc_sw128(smem_u32(sm.ds), 16, 1024);       // dS: K-major A (dQ) and MN-major B (dK^T)
       const uint64_t pd = smem_desc_sw128(smem_u32(sm.p), 16, 1024);         // P : MN-major B (dV^T)
       // (arguments are ring slots)
-      auto wait_k = [&](int s) { return bwd_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1, abort); };
-      auto wait_v = [&](int s) { return bwd_wait(&sm.v_full[s % kBwdVStages], (s / kBwdVStages) & 1, abort); };
+      auto wait_k = [&](int s) { return mma_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1, abort); };
+      auto wait_v = [&](int s) { return mma_wait(&sm.v_full[s % kBwdVStages], (s / kBwdVStages) & 1, abort); };
       // acc (128 rows x N keys) = a (Q or dO, K-major) x b^T (key tiles at ring stage st, K-major)
       auto issue_qk = [&](uint32_t acc, uint64_t a, uint64_t b0, int st, uint32_t idesc) {   // st: ring stage
         const uint64_t bd = desc_advance(b0, (uint32_t)st * kKvTile);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t a_off = (kk >> 2) * 16384 + (kk & 3) * 32, b_off = (kk >> 2) * 1024 + (kk & 3) * 32;
-          mma_ss(acc, desc_advance(a, a_off), desc_advance(bd, b_off), idesc, kk > 0);
+          mma_ss_w(acc, desc_advance(a, a_off), desc_advance(bd, b_off), idesc, kk > 0);
         }
       };
-      bool ok = bwd_wait(&sm.q_full, 0, abort);
+      bool ok = mma_wait(&sm.q_full, 0, abort);
       bool dq_started = false;
       // ---- dK/dV steps: one at a time, every operand from shared memory.  The tensor pipe runs in
       // issue order and a commit covers everything issued before it, so sdp_full of step s+1 also
@@ -333,30 +351,30 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tc_fence_after_sync();
         issue_qk(tmem + region(0), q_k, k_k0, st, idesc_sdp);
         issue_qk(tmem + region(0) + 64, do_k, v_k0, vst, idesc_sdp);
-        mma_commit(&sm.sdp_full);
-        mma_commit(&sm.v_empty[vst]);
-        ok = bwd_wait(&sm.pds_full, s & 1, abort);
+        mma_commit_w(&sm.sdp_full);
+        mma_commit_w(&sm.v_empty[vst]);
+        ok = mma_wait(&sm.pds_full, s & 1, abort);
         if (!ok) break;
         tc_fence_after_sync();
         const uint64_t kmn = desc_advance(k_mn0, (uint32_t)st * kKvTile);
 #pragma unroll
         for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per MMA
-          mma_ss(tmem + kColDQ, desc_advance(dsd, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
+          mma_ss_w(tmem + kColDQ, desc_advance(dsd, kk * 32), desc_advance(kmn, kk * 2 * kOct), idesc_dq,
                  (dq_started || kk > 0));
         dq_started = true;
         if (s > 0) {
-          ok = bwd_wait(&sm.dkv_free, (s - 1) & 1, abort);
+          ok = mma_wait(&sm.dkv_free, (s - 1) & 1, abort);
           if (!ok) break;
           tc_fence_after_sync();
         }
 #pragma unroll
         for (int kk = 0; kk < 128 / 16; ++kk)    // 16 query rows per MMA (2 row octets)
-          mma_ss(tmem + kColDV, desc_advance(do_mn, kk * 2048), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
+          mma_ss_w(tmem + kColDV, desc_advance(do_mn, kk * 2048), desc_advance(pd, kk * 2048), idesc_dkv, kk > 0);
 #pragma unroll
         for (int kk = 0; kk < 128 / 16; ++kk)
-          mma_ss(tmem + kColDK, desc_advance(q_mn, kk * 2048), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
-        mma_commit(&sm.dkv_full);
-        mma_commit(&sm.k_empty[st]);
+          mma_ss_w(tmem + kColDK, desc_advance(q_mn, kk * 2048), desc_advance(dsd, kk * 2048), idesc_dkv, kk > 0);
+        mma_commit_w(&sm.dkv_full);
+        mma_commit_w(&sm.k_empty[st]);
         HGA_TRACE_POINT(4);
       }
       // ---- paired steps.  Step u covers ring stages st, st+1 (contiguous); S(u) lives in region
@@ -366,23 +384,23 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           // the unused slot: observe its (copy-less) full barriers and release it
           ok = wait_k(n_act) && wait_v(n_act);
           if (ok) {
-            mma_commit(&sm.k_empty[n_act % kBwdKStages]);
-            mma_commit(&sm.v_empty[n_act % kBwdVStages]);
+            mma_commit_w(&sm.k_empty[n_act % kBwdKStages]);
+            mma_commit_w(&sm.v_empty[n_act % kBwdVStages]);
           }
         }
-        if (ok && n_act_even > 0) mma_commit(&sm.phase_a_done);
+        if (ok && n_act_even > 0) mma_commit_w(&sm.phase_a_done);
         const int ps0 = (n_act_even / 2) % (kBwdKStages / 2);
-        if (ok) ok = bwd_wait(&sm.kp_full[ps0], 0, abort);
+        if (ok) ok = mma_wait(&sm.kp_full[ps0], 0, abort);
         if (ok) {
           tc_fence_after_sync();
           issue_qk(tmem + region(0), q_k, k_k0, 2 * ps0, idesc_sdp2);
-          mma_commit(&sm.s_full[0]);
+          mma_commit_w(&sm.s_full[0]);
         }
-        if (ok) ok = bwd_wait(&sm.vp_full, 0, abort);
+        if (ok) ok = mma_wait(&sm.vp_full[0], 0, abort);
         if (ok) {
           tc_fence_after_sync();
           issue_qk(tmem + region(1), do_k, v_k0, 0, idesc_sdp2);
-          mma_commit(&sm.dp_full[0]);    // also tells the V producers that the V stages are free
+          mma_commit_w(&sm.dp_full[0]);    // also tells the V producers that the V pair is free
         }
         HGA_TRACE_POINT(3);
       }
@@ -393,42 +411,43 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const int rp = rs == 2 ? 0 : rs + 1;          // region of dP(u), dS(u)
         const int rs_n = rp == 2 ? 0 : rp + 1;        // region of S(u+1): two steps ago it held dP(u-1)
         if (u + 1 < n_pairs) {
-          ok = bwd_wait(&sm.kp_full[ps_n], (uint32_t)((u + 1) / kPs) & 1, abort);
+          ok = mma_wait(&sm.kp_full[ps_n], (uint32_t)((u + 1) / kPs) & 1, abort);
           // S(1) is the first to use the region that aliases the dK^T/dV^T accumulators: the
           // reduction warps must have read the last ones
-          if (ok && u == 0 && n_act > 0) ok = bwd_wait(&sm.dkv_free, (n_act - 1) & 1, abort);
+          if (ok && u == 0 && n_act > 0) ok = mma_wait(&sm.dkv_free, (n_act - 1) & 1, abort);
           if (!ok) break;
           tc_fence_after_sync();
           issue_qk(tmem + region(rs_n), q_k, k_k0, 2 * ps_n, idesc_sdp2);
-          mma_commit(&sm.s_full[(u + 1) & 1]);
+          mma_commit_w(&sm.s_full[(u + 1) & 1]);
           HGA_TRACE_POINT(6);
+          // dP(u+1) goes into the region of S(u) as soon as the row threads have read S(u) (they keep P in
+          // registers): it is then complete long before they finish dS(u) and P(u+1) and ask for it
+          ok = mma_wait(&sm.s_read[u & 1], (uint32_t)(u >> 1) & 1, abort) &&
+               mma_wait(&sm.vp_full[(u + 1) & 1], (uint32_t)((u + 1) >> 1) & 1, abort);
+          if (!ok) break;
+          tc_fence_after_sync();
+          issue_qk(tmem + region(rs), do_k, ((u + 1) & 1) ? v_k1 : v_k0, 0, idesc_sdp2);
+          mma_commit_w(&sm.dp_full[(u + 1) & 3]);
+          HGA_TRACE_POINT(8);
         }
-        ok = bwd_wait(&sm.ds_full, u & 1, abort);     // the row threads are done with S(u) and dP(u)
+        ok = mma_wait(&sm.ds_full[u & 1], (uint32_t)(u >> 1) & 1, abort);     // the row threads are done with dP(u): dS(u) is in its place
         if (!ok) break;
         tc_fence_after_sync();
         HGA_TRACE_POINT(5);
-        if (u + 1 < n_pairs) {
-          ok = bwd_wait(&sm.vp_full, (uint32_t)(u + 1) & 1, abort);
-          if (!ok) break;
-          tc_fence_after_sync();
-          issue_qk(tmem + region(rs), do_k, v_k0, 0, idesc_sdp2);       // dP(u+1) into the region of S(u)
-          mma_commit(&sm.dp_full[(u + 1) & 3]);
-          HGA_TRACE_POINT(8);
-        }
         // dQ += dS K over 128 keys: bf16 dS from TMEM (first tile at columns 0-31 of its region,
         // second tile at 64-95), the two K stages as one MN-major B operand
         const uint64_t kmn = desc_advance(k_mn0, (uint32_t)(2 * ps) * kKvTile);
         const uint32_t ds_base = tmem + region(rp);
 #pragma unroll
         for (int kk = 0; kk < 2 * kKT / 16; ++kk)
-          mma_ts(tmem + kColDQ, ds_base + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), desc_advance(kmn, kk * 2 * kOct),
+          mma_ts_w(tmem + kColDQ, ds_base + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), desc_advance(kmn, kk * 2 * kOct),
                  idesc_dq, (dq_started || kk > 0));
         dq_started = true;
-        mma_commit(&sm.kp_empty[(n_act_even / 2 + u) % kBwdKStages]);
+        mma_commit_w(&sm.kp_empty[(n_act_even / 2 + u) % kBwdKStages]);
         HGA_TRACE_POINT(7);
         rs = rs_n;
       }
-      if (ok) mma_commit(&sm.dq_done);
+      if (ok) mma_commit_w(&sm.dq_done);
     }
   } else if (warp < 10) {
     // ------------------------------------------------------------------ one thread per query row
@@ -460,10 +479,22 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
       }
-      sm.dpart[wg][row_in_tile] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+      // the two halves meet in tensor memory: columns 0 and 1 of the dQ accumulator, which no GEMM writes
+      // before the first dS exists (every shared-memory buffer may already be receiving copies)
+      tmem_st1(lane_base + kColDQ + wg, __float_as_uint((acc[0] + acc[1]) + (acc[2] + acc[3])));
+      tmem_wait_st();
     }
+    tc_fence_before_sync();
     asm volatile("bar.sync 3, 256;" ::: "memory");           // the 256 row threads (reached on every path)
-    const float neg_delta_s = -(sm.dpart[0][row_in_tile] + sm.dpart[1][row_in_tile]) * dm.scale;
+    tc_fence_after_sync();
+    uint32_t d_lo, d_hi;
+    tmem_ld2(lane_base + kColDQ, d_lo, d_hi);
+    tmem_wait_ld();
+    // (the first dQ GEMM of a dK/dV step follows the arrivals of warpgroup 0 alone: it must not overwrite
+    // these two columns before warpgroup 1 has read them)
+    tc_fence_before_sync();
+    asm volatile("bar.sync 3, 256;" ::: "memory");
+    const float neg_delta_s = -(__uint_as_float(d_lo) + __uint_as_float(d_hi)) * dm.scale;
     HGA_TRACE_POINT(10);
     if (wg == 0) {
       // ---- dK/dV steps (warpgroup 0): P and dS go to shared memory as operands of dV^T / dK^T / dQ
@@ -541,6 +572,8 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           pk[8 * q4 + i] = pack_bf16(p0, p1);
         }
       }
+      tc_fence_before_sync();
+      mbar_arrive(&sm.s_read[u & 1]);                 // S(u) has been read: its region may take dP(u+1)
       ok = __all_sync(0xffffffffu, bwd_wait(&sm.dp_full[u & 3], (u >> 2) & 1, abort));
       if (!ok) break;
       tc_fence_after_sync();
@@ -563,7 +596,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(&sm.ds_full);
+      mbar_arrive(&sm.ds_full[u & 1]);
       HGA_TRACE_POINT(14);
       rs = rp == 2 ? 0 : rp + 1;
     }
@@ -654,7 +687,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   __syncthreads();
   HGA_TRACE_POINT(31);
   HGA_TRACE_DUMP;
-  if (tid == 0 && sm.abort && status_word) atomicOr(status_word, HGA_STATUS_WAIT_TIMEOUT);
+  if (tid == 0 && sm.abort && status_word) atomicOr(status_word, HGA_ABORT_CODE(3, sm.abort));
   if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
@@ -713,3 +746,12 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
 }
 
 }  // namespace hga
+
+#ifdef HGA_DEBUG_WAIT
+extern "C" __attribute__((visibility("default"))) int hga_debug_dump(int* out64) {
+  cudaMemcpyFromSymbol(out64, hga::g_dbg_fail, sizeof(int) * 64);
+  int zero[64] = {0};
+  cudaMemcpyToSymbol(hga::g_dbg_fail, zero, sizeof(zero));
+  return 0;
+}
+#endif

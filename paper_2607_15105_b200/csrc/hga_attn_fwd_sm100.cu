@@ -42,7 +42,7 @@ using namespace sm100;
 constexpr int kFwdThreads = 256;
 constexpr int kStages = 2;
 constexpr int kFT = 64;                      // keys per tile
-constexpr float kRescaleThreshold = 8.0f;   // log2 units
+constexpr float kRescaleThreshold = 8.0f;   // log2 units: the reference is raised when the maximum outgrows it by this much
 
 template <int D>
 struct FwdSmem {
@@ -60,9 +60,16 @@ struct FwdSmem {
   int oct_row[1];   // really max_routed_tokens/8 entries (dynamic shared memory follows)
 };
 
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort) {
-  return mbar_wait_bounded(bar, parity, abort);
+__device__ __forceinline__ bool wait_or_abort_(uint64_t* bar, uint32_t parity, volatile int* abort, int code) {
+  return mbar_wait_bounded(bar, parity, abort, kWaitCycles, code);
 }
+#ifdef HGA_DEBUG_WAIT
+#define wait_or_abort(bar, parity, abort) wait_or_abort_((bar), (parity), (abort), __LINE__)
+#define HGA_FWD_ABORT_CODE(flag) (HGA_STATUS_WAIT_TIMEOUT | ((flag) << 8) | (1 << 28))
+#else
+#define wait_or_abort(bar, parity, abort) wait_or_abort_((bar), (parity), (abort), 1)
+#define HGA_FWD_ABORT_CODE(flag) HGA_STATUS_WAIT_TIMEOUT
+#endif
 
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 2)
@@ -177,7 +184,11 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp runs this branch converged (waits included) and one elected lane issues: see mma_ss_w.
+    {
+      auto mma_wait = [&](uint64_t* bar, uint32_t parity, volatile int* ab) {
+        return __all_sync(0xffffffffu, wait_or_abort(bar, parity, ab));
+      };
       constexpr uint32_t idesc_s = idesc_bf16_f32(128, kFT, 0, 0);
       constexpr uint32_t idesc_o = idesc_bf16_f32(128, D, 0, 1);
       // Descriptors are built once; inside the loops an MMA costs two integer adds (the lone
@@ -193,13 +204,13 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;   // panel, then 32-byte K step
-          mma_ss(d_addr, desc_advance(q_desc, off), desc_advance(kd, off), idesc_s, kk > 0);
+          mma_ss_w(d_addr, desc_advance(q_desc, off), desc_advance(kd, off), idesc_s, kk > 0);
         }
-        mma_commit(&sm.s_full[j & 1]);           // also releases the K stage (see the K producer)
+        mma_commit_w(&sm.s_full[j & 1]);           // also releases the K stage (see the K producer)
       };
-      bool ok = wait_or_abort(&sm.q_full, 0, abort);
+      bool ok = mma_wait(&sm.q_full, 0, abort);
       for (int j = 0; j < 2 && j < n_tiles && ok; ++j) {      // prologue: S two tiles ahead
-        ok = wait_or_abort(&sm.k_full[j % kStages], (j / kStages) & 1, abort);
+        ok = mma_wait(&sm.k_full[j % kStages], (j / kStages) & 1, abort);
         if (!ok) break;
         tc_fence_after_sync();
         issue_s(j);
@@ -208,9 +219,9 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       for (int j = 0; j < n_tiles && ok; ++j) {
         const int sv = j % kStages;
         const bool more = j + 2 < n_tiles;
-        ok = wait_or_abort(&sm.v_full[sv], (j / kStages) & 1, abort);
+        ok = mma_wait(&sm.v_full[sv], (j / kStages) & 1, abort);
         HGA_TRACE_POINT(6);
-        if (ok) ok = wait_or_abort(&sm.p_full[j & 1], (j >> 1) & 1, abort);
+        if (ok) ok = mma_wait(&sm.p_full[j & 1], (j >> 1) & 1, abort);
         if (!ok) break;
         tc_fence_after_sync();
         HGA_TRACE_POINT(5);
@@ -218,13 +229,13 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t p_addr = tmem + (j & 1) * 64;
 #pragma unroll
         for (int kk = 0; kk < kFT / 16; ++kk)     // 16 keys per step: 2 octets in smem, 8 TMEM columns of P
-          mma_ts(o_acc, p_addr + kk * 8, desc_advance(vd, kk * 2 * kOctBytes), idesc_o, (j > 0 || kk > 0));
-        mma_commit(&sm.v_empty[sv]);
-        if (j + 2 == n_tiles) mma_commit(&sm.tail_done);   // PV of the last-but-one tile (see rescale)
-        if (j + 1 == n_tiles) mma_commit(&sm.o_done);
+          mma_ts_w(o_acc, p_addr + kk * 8, desc_advance(vd, kk * 2 * kOctBytes), idesc_o, (j > 0 || kk > 0));
+        mma_commit_w(&sm.v_empty[sv]);
+        if (j + 2 == n_tiles) mma_commit_w(&sm.tail_done);   // PV of the last-but-one tile (see rescale)
+        if (j + 1 == n_tiles) mma_commit_w(&sm.o_done);
         HGA_TRACE_POINT(7);
         if (more) {                                // S(j+2) reuses the buffer P(j) sat in: ordered after PV(j)
-          ok = wait_or_abort(&sm.k_full[(j + 2) % kStages], ((j + 2) / kStages) & 1, abort);
+          ok = mma_wait(&sm.k_full[(j + 2) % kStages], ((j + 2) / kStages) & 1, abort);
           if (!ok) break;
           tc_fence_after_sync();
           issue_s(j + 2);
@@ -246,8 +257,38 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
       const uint32_t o_addr = lane_base + kColO;
       const float sl2 = dm.scale * 1.4426950408889634f;   // softmax scale in log2 units
+      // m_used: the reference the exponentials of a row are taken against (log2 units).  Only the FIRST tile
+      // is read twice (true maximum, then exponentials).  Later tiles are read once: p = 2^(x - m_used) with
+      // the reference as it stands, the tile's own maximum being found in the same pass.  A tile whose maximum
+      // outgrows the reference by more than the threshold (rare after the first tiles) raises the reference to
+      // that maximum (O, l rescaled) and takes its exponentials again -- S is still intact then, because P is
+      // only written once the tile is known to be in range.  The result is the one a maximum pass per tile
+      // would give: the reference is raised at the same tiles to the same values.
       float m_used = -INFINITY, l = 0.f, l_mma = 0.f;
+      const uint64_t sl2_2 = pack_f32x2(sl2, sl2);
       bool ok = true;
+      // O *= corr (per row); O must hold exactly the sum up to tile j-1, i.e. PV(j-1) must have completed.
+      // The issuer queues S(j+1) directly behind PV(j-1), so that S being ready proves it; the last tile
+      // has no S(j+1) and uses a barrier committed behind PV(n-2) instead.
+      auto rescale_o = [&](int j, float corr) {
+        bool fine;
+        if (j + 1 < n_tiles)
+          fine = __all_sync(0xffffffffu, wait_or_abort(&sm.s_full[(j + 1) & 1], ((j + 1) >> 1) & 1, abort));
+        else
+          fine = __all_sync(0xffffffffu, wait_or_abort(&sm.tail_done, 0, abort));
+        if (!fine) return false;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t y[32];
+          tmem_ld32(o_addr + c * 32, y);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) y[i] = __float_as_uint(__uint_as_float(y[i]) * corr);
+          tmem_st32(o_addr + c * 32, y);
+        }
+        return true;
+      };
       for (int j = 0; j < n_tiles; ++j) {
         const uint32_t s_addr = lane_base + (j & 1) * 64;
         ok = __all_sync(0xffffffffu, wait_or_abort(&sm.s_full[j & 1], (j >> 1) & 1, abort));
@@ -260,89 +301,99 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tc_fence_after_sync();
         HGA_TRACE_POINT(11);     // waiting for S
         const int vis = limit - kFT * j;                  // visible columns of this tile (may be <= 0)
-        // S is read from TMEM twice (row maximum, then exponentials), 32 columns at a time: holding
-        // all 64 values across both passes costs more registers than the budget of two CTAs per SM allows
-        float mxs[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        // scaled maximum of the tile's visible columns (a pass of its own: first tile and fall-back only)
+        auto tile_max = [&]() {
+          float mxs[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t x[32];
-          tmem_ld32(s_addr + 32 * c, x);
-          tmem_wait_ld();
-          if (vis >= kFT) {
+          for (int c = 0; c < 2; ++c) {
+            uint32_t x[32];
+            tmem_ld32(s_addr + 32 * c, x);
+            tmem_wait_ld();
+            if (vis >= kFT) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mxs[i & 3] = fmaxf(mxs[i & 3], __uint_as_float(x[i]));
-          } else {
+              for (int i = 0; i < 32; ++i) mxs[i & 3] = fmaxf(mxs[i & 3], __uint_as_float(x[i]));
+            } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (32 * c + i < vis) mxs[i & 3] = fmaxf(mxs[i & 3], __uint_as_float(x[i]));
+              for (int i = 0; i < 32; ++i)
+                if (32 * c + i < vis) mxs[i & 3] = fmaxf(mxs[i & 3], __uint_as_float(x[i]));
+            }
           }
-        }
-        const float mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])) * sl2;
-        HGA_TRACE_POINT(12);
-        float corr = 1.f;
-        bool raise = real_row && mx > m_used + kRescaleThreshold;   // also true for the first visible tile
-        if (raise) {
-          corr = fast_exp2(m_used - mx);                  // 0 when m_used is -inf
-          m_used = mx;
-          l *= corr;
-          l_mma *= corr;
-        }
-        if (j > 0 && __any_sync(0xffffffffu, raise)) {
-          // O must hold exactly the sum up to tile j-1, i.e. PV(j-1) must have completed.  The
-          // issuer queues S(j+1) directly behind PV(j-1), so that S being ready proves it; the last
-          // tile has no S(j+1) and uses a barrier committed behind PV(n-2) instead.
-          if (j + 1 < n_tiles)
-            ok = __all_sync(0xffffffffu, wait_or_abort(&sm.s_full[(j + 1) & 1], ((j + 1) >> 1) & 1, abort));
-          else
-            ok = __all_sync(0xffffffffu, wait_or_abort(&sm.tail_done, 0, abort));
+          return fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])) * sl2;
+        };
+        // raises the reference of the rows that ask for it to `to` and rescales their sums and O
+        auto raise_to = [&](bool raise, float to) {
+          float corr = 1.f;
+          if (raise) {
+            corr = fast_exp2(m_used - to);                // 0 when m_used is -inf
+            m_used = to;
+            l *= corr;
+            l_mma *= corr;
+          }
+          if (j > 0 && __any_sync(0xffffffffu, raise)) return rescale_o(j, corr);
+          return true;
+        };
+        if (j == 0) {
+          ok = raise_to(true, tile_max());
           if (!ok) break;
-          tc_fence_after_sync();
+        }
+        HGA_TRACE_POINT(13);
+        // p = 2^(x - m); P (bf16) is written over S once the whole tile is known to be in range.  l sums the
+        // exact probabilities (for LSE), l_mma the rounded ones the MMA really applies: normalising O by THEIR
+        // sum makes the rounding of a dominant weight cancel.  Two columns per step on packed fp32 pairs.
+        uint32_t pk[32];
+        float t_l, t_r, t_max;
+        auto exp_pass = [&]() {
+          const float neg_m = -m_used;
+          const uint64_t neg_m2 = pack_f32x2(neg_m, neg_m);
+          uint64_t lsum = pack_f32x2(0.f, 0.f), rsum = pack_f32x2(0.f, 0.f);
+          float mxa = -INFINITY, mxb = -INFINITY;
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t y[32];
-            tmem_ld32(o_addr + c * 32, y);
+          for (int c = 0; c < 2; ++c) {
+            uint32_t x[32];
+            tmem_ld32(s_addr + 32 * c, x);
             tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) y[i] = __float_as_uint(__uint_as_float(y[i]) * corr);
-            tmem_st32(o_addr + c * 32, y);
-          }
-        }
-        // p = 2^(x - m); P (bf16) is written over S.  l sums the exact probabilities (for LSE),
-        // l_mma the rounded ones the MMA really applies: normalising O by THEIR sum makes the
-        // rounding of a dominant weight cancel.
-        HGA_TRACE_POINT(13);
-        const float neg_m = -m_used;
-        // two columns per step on packed fp32 pairs: one FMA for both arguments, one add each for the
-        // exact and the rounded sums (the row threads are issue-bound when two CTAs share the SM)
-        const uint64_t sl2_2 = pack_f32x2(sl2, sl2), neg_m2 = pack_f32x2(neg_m, neg_m);
-        uint64_t lsum = pack_f32x2(0.f, 0.f), rsum = pack_f32x2(0.f, 0.f);
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t x[32], pk[16];
-          tmem_ld32(s_addr + 32 * c, x);       // (P of the first half lands in columns 0-15: already consumed)
-          tmem_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float a0, a1;
-            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1])), sl2_2, neg_m2),
-                         a0, a1);
-            float p0 = fast_exp2(a0), p1 = fast_exp2(a1);
-            if (vis < kFT) {                              // diagonal / ragged tile only
-              if (32 * c + 2 * i >= vis) p0 = 0.f;
-              if (32 * c + 2 * i + 1 >= vis) p1 = 0.f;
+            for (int i = 0; i < 16; ++i) {
+              const float x0 = __uint_as_float(x[2 * i]), x1 = __uint_as_float(x[2 * i + 1]);
+              float a0, a1;
+              unpack_f32x2(fma_f32x2(pack_f32x2(x0, x1), sl2_2, neg_m2), a0, a1);
+              float p0 = fast_exp2(a0), p1 = fast_exp2(a1);
+              if (vis < kFT) {                            // diagonal / ragged tile only
+                if (32 * c + 2 * i >= vis) { p0 = 0.f; a0 = -INFINITY; }
+                if (32 * c + 2 * i + 1 >= vis) { p1 = 0.f; a1 = -INFINITY; }
+              }
+              if (i & 1) mxb = fmaxf(mxb, fmaxf(a0, a1)); else mxa = fmaxf(mxa, fmaxf(a0, a1));
+              lsum = add_f32x2(lsum, pack_f32x2(p0, p1));
+              const __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
+              pk[16 * c + i] = *reinterpret_cast<const uint32_t*>(&hh);
+              rsum = add_f32x2(rsum, pack_f32x2(__uint_as_float(pk[16 * c + i] << 16), __uint_as_float(pk[16 * c + i] & 0xffff0000u)));
             }
-            lsum = add_f32x2(lsum, pack_f32x2(p0, p1));
-            const __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
-            pk[i] = *reinterpret_cast<const uint32_t*>(&hh);
-            rsum = add_f32x2(rsum, pack_f32x2(__uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u)));
           }
-          tmem_st16(s_addr + c * 16, pk);
+          float la, lb, ra, rb;
+          unpack_f32x2(lsum, la, lb);
+          unpack_f32x2(rsum, ra, rb);
+          t_l = la + lb;
+          t_r = ra + rb;
+          t_max = fmaxf(mxa, mxb);                        // largest exponent argument = tile maximum - m_used
+        };
+        exp_pass();
+        if (__any_sync(0xffffffffu, t_max > kRescaleThreshold)) {
+          // the tile's maximum outgrows the reference: raise it to that maximum and take the exponentials again
+          ok = raise_to(t_max > kRescaleThreshold, m_used + t_max);
+          if (!ok) break;
+          exp_pass();
         }
-        float la, lb, ra, rb;
-        unpack_f32x2(lsum, la, lb);
-        unpack_f32x2(rsum, ra, rb);
-        l += la + lb;
-        l_mma += ra + rb;
+        {
+          uint32_t out[16];
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) out[i] = pk[16 * c + i];
+            tmem_st16(s_addr + c * 16, out);
+          }
+        }
+        l += t_l;
+        l_mma += t_r;
         HGA_TRACE_POINT(14);
         tmem_wait_st();
         tc_fence_before_sync();
@@ -392,7 +443,7 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   __syncthreads();
   HGA_TRACE_POINT(31);
   HGA_TRACE_DUMP;
-  if (tid == 0 && sm.abort && status_word) atomicOr(status_word, HGA_STATUS_WAIT_TIMEOUT);
+  if (tid == 0 && sm.abort && status_word) atomicOr(status_word, HGA_FWD_ABORT_CODE(sm.abort));
   if (warp == 1) {
     __syncwarp();
     tmem_dealloc(tmem, kTmemCols);

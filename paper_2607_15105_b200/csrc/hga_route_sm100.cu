@@ -187,17 +187,21 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       }
     } else if (warp == 1) {
       // ---------------------------------------------------------------- MMA issuer
-      if (lane == 0) {
+      // The whole warp runs this branch converged (waits included) and one elected lane issues: see mma_ss_w.
+      {
+        auto mma_wait = [&](uint64_t* bar, uint32_t parity, volatile int* ab) {
+          return __all_sync(0xffffffffu, rt_wait(bar, parity, ab));
+        };
         const uint32_t idesc = idesc_bf16_f32(128, rows_half, 0, 0);
-        bool ok = phase2 ? true : rt_wait(&sm.q_full, 0, abort);
+        bool ok = phase2 ? true : mma_wait(&sm.q_full, 0, abort);
         if (!phase2) HGA_RT_STAMP(2);
         for (int t = 0; t < n_tiles && ok; ++t) {
           const int tg = t_begin + t, s = tg % STAGES;
-          ok = rt_wait(&sm.a_full[s], (tg / STAGES) & 1, abort);
+          ok = mma_wait(&sm.a_full[s], (tg / STAGES) & 1, abort);
           HGA_RT_STAMP(3 + tg);
           for (int hf = 0; hf < n_halves && ok; ++hf) {
             const int step = tg * n_halves + hf, buf = step % ACCS, use = step / ACCS;
-            if (use > 0) ok = rt_wait(&sm.acc_free[buf], (use - 1) & 1, abort);
+            if (use > 0) ok = mma_wait(&sm.acc_free[buf], (use - 1) & 1, abort);
             if (!ok) break;
             tc_fence_after_sync();
             const uint64_t ad = smem_desc_sw128(smem_u32(sm.a[s]), 16, kOctBytes);
@@ -206,11 +210,11 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
               const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-              mma_ss(tmem + buf * kAccCols, desc_advance(ad, off), desc_advance(bd, off), idesc, kk > 0);
+              mma_ss_w(tmem + buf * kAccCols, desc_advance(ad, off), desc_advance(bd, off), idesc, kk > 0);
             }
-            mma_commit(&sm.acc_full[buf]);
+            mma_commit_w(&sm.acc_full[buf]);
           }
-          if (ok) mma_commit(&sm.a_empty[s]);
+          if (ok) mma_commit_w(&sm.a_empty[s]);
           HGA_RT_STAMP(12 + tg);
         }
       }
@@ -461,10 +465,10 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       for (int tg = tiles_issued > STAGES ? tiles_issued - STAGES : 0; tg < tiles_issued; ++tg)
         mbar_wait(&sm.a_full[tg % STAGES], (tg / STAGES) & 1);
     }
-    if (warp == 1 && lane == 0) {
-      // GEMMs this thread issued may still be writing tensor memory: a commit completes once every
-      // earlier MMA of the thread has, so wait for one (bounded) before the columns are given back
-      mma_commit(&sm.drain);
+    if (warp == 1) {
+      // GEMMs the warp's issuing lane started may still be writing tensor memory: a commit completes once
+      // every earlier MMA of that lane has, so wait for one (bounded) before the columns are given back
+      mma_commit_w(&sm.drain);
       mbar_wait(&sm.drain, 0);
     }
   }

@@ -139,6 +139,73 @@ def test_item_the_router_gave_up_on_gets_sink_and_local_only(flags):
     check_grads(grads_of(buf), ref_grads, "n_groups = -1")
 
 
+@pytest.mark.parametrize("flags", FAMILY_FLAGS)
+def test_late_dominant_key_raises_the_softmax_reference_mid_sweep(flags):
+    """A key late in the routed order (the last position of the local window before the block) whose
+    logit lies ~98 binary orders above every other key's: the forward kernel, which takes the exponentials
+    of later tiles against the reference of earlier ones, must notice that this tile alone would leave
+    the exponent range and fall back to the tile's own maximum.  Exact answer: O ~ that key's value row."""
+    cfg = cfg_of(seed=41, batch=1)
+    x = make_inputs(cfg)
+    from paper_2607_15105_b200.workloads import f32_to_bf16_bits
+    H, Bq = cfg.history, cfg.q_block
+    K = x["K"].copy()
+    Q = x["Q"].copy()
+    one = lambda v: f32_to_bf16_bits(np.array([v], np.float32))[0]
+    for h in range(cfg.n_kv_heads):
+        K[0, h, :, 0] = 0                                   # component 0 belongs to the planted pair alone
+    qb = cfg.n_q_blocks - 1                                 # the last block, both kv heads: no later block sees the key
+    kpos = H + qb * Bq - 1
+    K[0, :, kpos, 0] = one(48.0)
+    Q[0, :, qb * Bq:(qb + 1) * Bq, 0] = one(16.0)           # 16 * 48 / sqrt(128) = 67.9 nats = 98 in log2
+    x = dict(x, K=K, Q=Q)
+    cs, gs = oracle.build_summaries(cfg, K)
+    ref = oracle.route(cfg, Q, cs, gs)
+    gi, ng = ref["group_idx"], ref["n_groups"]
+    O, LSE = oracle.attn_fwd(cfg, Q, K, x["V"], gi, ng)
+    buf = binding.HgaLayerBuffers(cfg, backward=False, flags=flags)
+    buf.attn_fwd(to_dev(Q), to_dev(K), to_dev(x["V"]), torch.from_numpy(gi).cuda(), torch.from_numpy(ng).cuda())
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    assert float(LSE.max()) > 60.0                          # the planted logit is really there
+    assert np.max(np.abs(bf16_to_f64(buf.O) - O)) <= TOL_O
+    assert np.max(np.abs(buf.LSE.cpu().numpy().astype(np.float64) - LSE)) <= TOL_LSE
+
+
+def test_backward_next_to_another_stream_never_misses_a_barrier_phase():
+    """The backward kernels hand tiles over through mbarrier phases; a waiter that is late must still
+    find the phase it waits for.  Running the backward while another stream keeps the GPU busy (the
+    way hga_tbptt_walk overlaps one segment's backward with the next segment's forward) stretches those
+    delays: every call must finish in its usual time with a clean status word, and with the same dQ."""
+    import time
+    pr = Problem(cfg_of(batch=1, n_q_heads=32, n_kv_heads=8, total_len=4096, seg_len=2048, topk_chunks=16,
+                        topk_groups=4, topics=64, needles=8, seed=43))
+    cfg = pr.cfg
+    a, b = binding.HgaLayerBuffers(cfg), binding.HgaLayerBuffers(cfg)
+    for buf in (a, b):
+        buf.build_summaries(pr.K, 0, cfg.total_len)
+        buf.route(pr.Q)
+        buf.attn_fwd(pr.Q, pr.K, pr.V)
+    a.attn_bwd(pr.Q, pr.K, pr.V, pr.dO)
+    torch.cuda.synchronize()
+    first = a.dQ.clone()
+    side = torch.cuda.Stream()
+    for it in range(25):
+        t0 = time.time()
+        for _ in range(8):
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                a.attn_bwd(pr.Q, pr.K, pr.V, pr.dO)
+            b.build_summaries(pr.K)
+            b.route(pr.Q)
+            b.attn_fwd(pr.Q, pr.K, pr.V)
+            torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        assert time.time() - t0 < 0.25, "a bounded wait ran out (each takes about half a second)"
+        assert int(a.status.item()) == 0 and int(b.status.item()) == 0
+    assert torch.equal(a.dQ, first)
+
+
 def test_kernel_families_are_counted_per_call():
     pr = Problem(cfg_of())
     cfg = pr.cfg
