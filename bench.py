@@ -82,10 +82,39 @@ def active_group_pairs(cfg, group_idx, n_groups):
     return n * cfg.group * cfg.gqa * cfg.q_block
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per call, summed over the call's kernels, from the
-# ncu captures summarised under profiles/ (forward: k_attn_fwd_sm100; backward: k_bwd_delta_sm100
-# 33.58 MB + k_attn_bwd_band_sm100 42.88 MB + k_attn_bwd_sm100 88.73 MB).
-NCU_TRAFFIC_BYTES = {3: {"hga_attn_fwd": 63.34e6, "hga_attn_bwd": 165.19e6}}
+def load_traffic(config):
+    """DRAM bytes per call (dram__bytes_read.sum + dram__bytes_write.sum, summed over the call's kernels)
+    from the ncu captures summarised under profiles/: profiles/traffic.json says which commit and which
+    kernels the figures belong to.  Returns ({call: bytes}, provenance) or ({}, None)."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as f:
+            t = json.load(f)
+    except (OSError, ValueError):
+        return {}, None
+    entry = t.get("configs", {}).get(str(config))
+    if not entry:
+        return {}, None
+    return entry.get("calls", {}), {"commit": t.get("commit"), "captured": t.get("captured"),
+                                    "kernels": entry.get("kernels")}
+
+
+def route_work(cfg):
+    """Algorithmic work of hga_route: 2*d*(G*Bq)*(candidates + opened groups) flops per item; bytes = the
+    candidate chunk summaries and the opened chunks' group summaries read once per item, Q once, lists out."""
+    d, rows = cfg.head_dim, cfg.gqa * cfg.q_block
+    per = cfg.chunk // cfg.group
+    flops = nbytes = 0.0
+    for qb in range(cfg.n_q_blocks):
+        p0 = cfg.history + qb * cfg.q_block
+        ls = max(0, ((p0 - cfg.local) // cfg.chunk) * cfg.chunk) if p0 - cfg.local > 0 else 0
+        se = min(cfg.sink, ls)
+        n_cand = (ls - se) // cfg.chunk
+        k_sel = min(cfg.topk_chunks, n_cand)
+        flops += 2.0 * d * rows * (n_cand + k_sel * per)
+        nbytes += (n_cand + k_sel * per) * d * 2 + rows * d * 2 + (cfg.topk_chunks * (1 + min(cfg.topk_groups, per)) + 1) * 4
+    n = cfg.batch * cfg.n_kv_heads
+    return flops * n, nbytes * n
 
 
 def roofline_entry(name, flops, nbytes, seconds, peaks, sustained=False):
@@ -276,6 +305,143 @@ def time_tbptt_walk(cfg, args, stream):
             "note": "one layer, forward+backward of every segment (history 0 .. L-S); inputs larger than L2"}
 
 
+def time_varlen(args, stream):
+    """hga_varlen_step on 16 short packed sequences of the headline layer shape (512 new tokens behind
+    1536 resident ones each): the packed call against the same sequences run one after another on the
+    caller's stream through the four calls, both as eager launches with L2 flushed before each step."""
+    import torch
+    from paper_2607_15105_b200 import binding
+    n_seq, L, S = 16, 2048, 512
+    base = CONFIGS[3].scaled(total_len=L, seg_len=S, topics=64, needles=0)
+    xs = [make_inputs(base.scaled(seed=base.seed + 200 + i)) for i in range(n_seq)]
+    pack = lambda k: np.ascontiguousarray(np.concatenate([x[k][0].transpose(1, 0, 2) for x in xs], axis=0))
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    Q, K, V, dO = (dev(pack(k)) for k in ("Q", "K", "V", "dO"))
+    del xs
+    Hq, Hkv, d, kc, kge = base.n_q_heads, base.n_kv_heads, base.head_dim, base.topk_chunks, base.kg_eff
+    cu_q = np.arange(n_seq + 1, dtype=np.int32) * S
+    cu_k = np.arange(n_seq + 1, dtype=np.int32) * L
+    n_q, n_k = n_seq * S, n_seq * L
+    p = binding.make_params(base)
+    cs = torch.zeros(Hkv, n_k // base.chunk, d, dtype=torch.bfloat16, device="cuda")
+    gs = torch.zeros(Hkv, n_k // base.group, d, dtype=torch.bfloat16, device="cuda")
+    items = Hkv * n_q // base.q_block
+    ci = torch.zeros(items, kc, dtype=torch.int32, device="cuda")
+    gi = torch.zeros(items, kc * kge, dtype=torch.int32, device="cuda")
+    ng = torch.zeros(items, dtype=torch.int32, device="cuda")
+    O, dQ = torch.zeros(n_q, Hq, d, dtype=torch.bfloat16, device="cuda"), torch.zeros(n_q, Hq, d, dtype=torch.bfloat16, device="cuda")
+    LSE = torch.zeros(Hq * n_q, dtype=torch.float32, device="cuda")
+    dK = torch.zeros(Hkv * n_q * d, dtype=torch.float32, device="cuda")
+    dV = torch.zeros_like(dK)
+    ws = torch.empty(binding.hga_varlen_workspace_bytes(p, cu_q, cu_k) + 256, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # resident state: the history summaries of every sequence (token-major keys, packed summary buffers)
+    ph = binding.make_params(base, k_stride=(L * Hkv * d, d, Hkv * d), summary_len=n_k)
+    for i in range(n_seq):
+        binding.hga_build_summaries(ph, K[i * L:], 0, L - S, cs[:, i * L // base.chunk:], gs[:, i * L // base.group:])
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+
+    def packed():
+        binding.hga_varlen_step(p, cu_q, cu_k, Q, K, V, dO, cs, gs, ci, gi, ng, O, LSE, dQ, dK, dV, ws, status)
+
+    reps = max(3, min(args.steps, 7))
+    for _ in range(3):
+        packed()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in ev:
+        flush.zero_()
+        a.record(stream)
+        packed()
+        b.record(stream)
+    torch.cuda.synchronize()
+    ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+    return {"sequences": n_seq, "tokens": n_q, "resident_tokens": n_k, "ms_per_step": round(ms, 4),
+            "tokens_per_s": round(n_q / (ms * 1e-3), 1), "launch": "eager, two library streams",
+            "device_status_word": int(status.item()),
+            "note": "16 packed sequences, 512 new tokens behind 1536 resident ones each; summaries of the active "
+                    "ranges + route + attention fwd + bwd per sequence"}
+
+
+def time_config(n, args, peaks):
+    """One benchmark configuration other than the headline one: per-call medians (eager launches, CUDA
+    events around each call, L2 flushed before every step), the CUDA-graph step, and each call's roofline."""
+    import torch
+    from paper_2607_15105_b200 import binding
+    cfg = CONFIGS[n]
+    x = make_inputs(cfg)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    Q, K, V = dev(x["Q"]), dev(x["K"]), dev(x["V"])
+    dO = dev(x["dO"]) if cfg.backward else None
+    del x
+    buf = binding.HgaLayerBuffers(cfg, backward=cfg.backward, flags=args.flags)
+    buf.build_summaries(K, 0, cfg.history)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    names = ["build_summaries", "route", "attn_fwd"] + (["attn_bwd"] if cfg.backward else [])
+    calls = [lambda: buf.build_summaries(K), lambda: buf.route(Q), lambda: buf.attn_fwd(Q, K, V)]
+    if cfg.backward:
+        calls.append(lambda: buf.attn_bwd(Q, K, V, dO))
+    steps = max(3, min(args.steps, 7))
+    for _ in range(3):
+        for c in calls:
+            c()
+    torch.cuda.synchronize()
+    launches0 = binding.hga_kernel_launch_counts()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)] for _ in range(steps)]
+    for e in ev:
+        flush.zero_()
+        e[0].record(stream)
+        for i, c in enumerate(calls):
+            c()
+            e[i + 1].record(stream)
+    torch.cuda.synchronize()
+    ran = [b - a for a, b in zip(launches0, binding.hga_kernel_launch_counts())]
+    per_call = np.array([[e[j].elapsed_time(e[j + 1]) for j in range(len(calls))] for e in ev])
+    med = np.median(per_call, axis=0) * 1e-3
+    graph_ms = None
+    try:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for c in calls:
+                c()
+        gev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in gev:
+            flush.zero_()
+            a.record(stream)
+            g.replay()
+            b.record(stream)
+        torch.cuda.synchronize()
+        graph_ms = float(np.median([a.elapsed_time(b) for a, b in gev]))
+    except Exception:      # capture unavailable: the eager numbers stand
+        pass
+    gi, ng = buf.group_idx.cpu().numpy(), buf.n_groups.cpu().numpy()
+    wc = work_counts(cfg, ng)
+    wc["bwd_flops"] += 4.0 * cfg.head_dim * active_group_pairs(cfg, gi, ng)
+    rf, rb = route_work(cfg)
+    roofs = {"route": roofline_entry("hga_route", rf, rb, med[1], peaks),
+             "attn_fwd": roofline_entry("hga_attn_fwd", wc["fwd_flops"], wc["fwd_bytes"], med[2], peaks)}
+    if cfg.backward:
+        roofs["attn_bwd"] = roofline_entry("hga_attn_bwd", wc["bwd_flops"], wc["bwd_bytes"], med[3], peaks)
+    attn = [roofs[k] for k in ("attn_fwd", "attn_bwd") if k in roofs]
+    step_us = graph_ms * 1e3 if graph_ms is not None else float(med.sum()) * 1e6
+    fam = ("summaries", "route_tensor", "route_generic", "fwd_tensor", "fwd_generic", "bwd_tensor", "bwd_generic", "aux")
+    out = {"workload": cfg.name, "pass": "fwd+bwd" if cfg.backward else "fwd", "steps": steps,
+           "per_call_us_median": {k: round(float(m) * 1e6, 2) for k, m in zip(names, med)},
+           "step_us": round(step_us, 2), "launch": "cuda_graph" if graph_ms is not None else "eager",
+           "tokens_per_s": round(cfg.tokens_per_step / (step_us * 1e-6), 1),
+           "roofline": {k: {f: v[f] for f in ("bound", "achieved", "peak", "unit", "frac", "roofline_us", "measured_us")}
+                        for k, v in roofs.items()},
+           "attention": {"us": round(sum(r["measured_us"] for r in attn), 2),
+                         "roofline_us": round(sum(r["roofline_us"] for r in attn), 2),
+                         "frac_of_roofline": round(sum(r["roofline_us"] for r in attn) / sum(r["measured_us"] for r in attn), 4)},
+           "kernel_launches_by_family": {f: int(c) for f, c in zip(fam, ran) if c},
+           "device_status_word": int(buf.status.item())}
+    del Q, K, V, dO, buf, flush
+    torch.cuda.empty_cache()
+    return out
+
+
 # ----------------------------------------------------------------------------- main arm
 
 def time_decode(args, stream, peaks):
@@ -396,6 +562,8 @@ def main():
                     help="run only the generation-shaped step and print its object (profiling captures)")
     ap.add_argument("--decode-batch", type=int, default=0,
                     help="sequences in the generation-shaped step (default: configuration 7's 32)")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the per-configuration timings (configurations 2, 4, 5 and 6 beside the headline one)")
     ap.add_argument("--no-walk", action="store_true",
                     help="skip the whole-sequence TBPTT walk (every segment of the sequence, one layer)")
     args = ap.parse_args()
@@ -574,8 +742,10 @@ def main():
         roofs = {"attn_fwd": roofline_entry("hga_attn_fwd", wc["fwd_flops"], wc["fwd_bytes"], med[2], peaks)}
         if cfg.backward:
             roofs["attn_bwd"] = roofline_entry("hga_attn_bwd", wc["bwd_flops"], wc["bwd_bytes"], med[3], peaks)
+        traffic, provenance = load_traffic(args.config)
         for r in roofs.values():
-            r["traffic"] = NCU_TRAFFIC_BYTES.get(args.config, {}).get(r["kernel"])
+            r["traffic"] = traffic.get(r["kernel"])
+            r["traffic_source"] = provenance
             r["algorithmic_bytes"] = wc["fwd_bytes"] if r["kernel"] == "hga_attn_fwd" else wc["bwd_bytes"]
             r["algorithmic_flops"] = wc["fwd_flops"] if r["kernel"] == "hga_attn_fwd" else wc["bwd_flops"]
         dominant = max(roofs.values(), key=lambda r: r["measured_us"])
@@ -607,6 +777,13 @@ def main():
             "paper_context": "217.75 (HGA) / 207.02 (dense) tokens/s: whole-model QLoRA step at 2K on a "
                              "Quadro RTX 5000 (Table 2); another machine and scope, not the target",
         }
+        if world == 1 and args.config == 3 and not args.no_configs:
+            # the other benchmark configurations, each a few milliseconds of GPU time
+            del Q, K, V, dO, arena
+            torch.cuda.empty_cache()
+            line["configs"] = {str(n): time_config(n, args, peaks) for n in (2, 4, 5, 6)}
+        if world == 1 and args.config == 3 and not args.no_configs:
+            line["varlen"] = time_varlen(args, stream)
         if walk is not None:
             line["tbptt_walk"] = walk
         if decode is not None:

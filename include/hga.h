@@ -263,8 +263,11 @@ HGA_API int hga_tbptt_walk(const hga_params* p, const void* Q, const void* K, co
  * p gives the head counts, head_dim, chunk/group/q_block, budgets, windows, scale and flags; its
  * batch, total_len, seg_len, summary_len and strides are ignored.  dO == NULL runs the forward half
  * only.  Every sequence runs build_summaries(active range) -> route -> attn_fwd -> attn_bwd as a
- * batch-1 problem on `stream`, one after the other (host logic only: the kernels are the ones
- * above).  workspace: device scratch of hga_varlen_workspace_bytes() bytes. */
+ * batch-1 problem (host logic only: the kernels are the ones above).  The sequences are independent, so
+ * they go alternately to two streams the library creates once per device, and the kernels of two
+ * sequences run side by side; both streams start behind the work already queued on `stream` and are
+ * joined back into it before the call returns.  workspace: device scratch of
+ * hga_varlen_workspace_bytes() bytes (one half per stream). */
 HGA_API int hga_varlen_step(const hga_params* p, int32_t n_seq, const int32_t* cu_q, const int32_t* cu_k,
                     const void* Q, const void* K, const void* V, const void* dO, void* chunk_sum,
                     void* group_sum, int32_t* chunk_idx, int32_t* group_idx, int32_t* n_groups, void* O,

@@ -528,7 +528,8 @@ int hga_varlen_workspace_bytes(const hga_params* p, int32_t n_seq, const int32_t
     route_max = std::max(route_max, route_workspace_bytes(dm));
     bwd_max = std::max(bwd_max, bwd_workspace_bytes(dm));
   }
-  *bytes = ((route_max + 255) & ~(size_t)255) + bwd_max;
+  // two lanes (see hga_varlen_step): each has its own routing and backward scratch
+  *bytes = 2 * (((route_max + 255) & ~(size_t)255) + ((bwd_max + 255) & ~(size_t)255));
   return HGA_OK;
 }
 
@@ -550,12 +551,32 @@ int hga_varlen_step(const hga_params* p, int32_t n_seq, const int32_t* cu_q, con
   const int per = p->chunk / p->group;
   const int kge = p->topk_groups < per ? p->topk_groups : per;
   const size_t grad_bytes = (p->flags & HGA_FLAG_BWD_BF16_GRADS) ? 2 : 4;
+  // The sequences are independent problems.  A short sequence fills only part of the GPU (its kernels are
+  // one or two CTAs per SM wide and a few waves deep at most), so the sequences go alternately to two
+  // library-owned streams ("lanes"), each with its own half of the workspace: the kernels of two sequences
+  // run side by side.  Both lanes start behind the work already queued on `stream` and are joined back into
+  // it before the call returns.
+  cudaStream_t st = (cudaStream_t)stream;
+  StepPipe* pipe = n_seq > 1 ? step_pipe(1) : nullptr;
+  if (n_seq > 1 && !pipe) return HGA_ERR_CUDA;
+  cudaStream_t lanes[2] = {pipe ? pipe->in : st, pipe ? pipe->out : st};
+  if (pipe) {
+    rc = record_cuda(cudaEventRecord(pipe->fork, st));
+    if (rc) return rc;
+    for (int l = 0; l < 2; ++l) {
+      rc = record_cuda(cudaStreamWaitEvent(lanes[l], pipe->fork, 0));
+      if (rc) return rc;
+    }
+  }
+  const size_t lane_bytes = need / 2;
   for (int i = 0; i < n_seq; ++i) {
     hga_params ps;
     varlen_params(p, n_seq, cu_q, cu_k, i, ps);
     Dims dm;
     rc = resolve(&ps, dm);
     if (rc) return rc;
+    void* lane_stream = (void*)lanes[i & 1];
+    char* ws = (char*)workspace + (size_t)(i & 1) * lane_bytes;
     const int64_t q0 = cu_q[i], k0 = cu_k[i];
     const char* Qi = (const char*)Q + q0 * Hq * d * 2;
     const char* Ki = (const char*)K + k0 * Hkv * d * 2;
@@ -569,17 +590,26 @@ int hga_varlen_step(const hga_params* p, int32_t n_seq, const int32_t* cu_q, con
     int32_t* ng = n_groups + item0;
     float* lse = LSE + Hq * q0;
     const size_t route_ws = route_workspace_bytes(dm), bwd_ws = bwd_workspace_bytes(dm);
-    rc = hga_build_summaries(&ps, Ki, dm.H, dm.L, csi, gsi, stream);
+    rc = hga_build_summaries(&ps, Ki, dm.H, dm.L, csi, gsi, lane_stream);
     if (rc) return rc;
-    rc = hga_route(&ps, Qi, csi, gsi, ci, gi, ng, nullptr, nullptr, workspace, route_ws, stream);
+    rc = hga_route(&ps, Qi, csi, gsi, ci, gi, ng, nullptr, nullptr, ws, route_ws, lane_stream);
     if (rc) return rc;
-    rc = hga_attn_fwd(&ps, Qi, Ki, Vi, gi, ng, Oi, lse, status_word, stream);
+    rc = hga_attn_fwd(&ps, Qi, Ki, Vi, gi, ng, Oi, lse, status_word, lane_stream);
     if (rc) return rc;
     if (bwd) {
       rc = hga_attn_bwd(&ps, Qi, Ki, Vi, Oi, lse, (const char*)dO + q0 * Hq * d * 2, gi, ng,
                         (char*)dQ + q0 * Hq * d * 2, (char*)dK + Hkv * d * q0 * grad_bytes,
                         (char*)dV + Hkv * d * q0 * grad_bytes,
-                        (char*)workspace + ((route_ws + 255) & ~(size_t)255), bwd_ws, status_word, stream);
+                        ws + ((route_ws + 255) & ~(size_t)255), bwd_ws, status_word, lane_stream);
+      if (rc) return rc;
+    }
+  }
+  if (pipe) {
+    // `stream` waits for both lanes (one event each; recorded and waited on in turn)
+    for (int l = 0; l < 2; ++l) {
+      rc = record_cuda(cudaEventRecord(pipe->join, lanes[l]));
+      if (rc) return rc;
+      rc = record_cuda(cudaStreamWaitEvent(st, pipe->join, 0));
       if (rc) return rc;
     }
   }

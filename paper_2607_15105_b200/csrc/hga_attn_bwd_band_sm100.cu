@@ -444,8 +444,8 @@ int launch_attn_bwd_band_sm100(const Dims& dm, const void* Q, const void* K, con
       encode_tensor_map_bf16(&mv, V, 5, dk, sv, box, true))
     return HGA_ERR_UNSUPPORTED;
   const size_t smem = sizeof(BandSmem) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(k_attn_bwd_band_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return record_cuda(e);
+  const int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(&k_attn_bwd_band_sm100), smem);
+  if (rc) return rc;
   const int units = dm.B * dm.Hkv * ((dm.S + kKeys - 1) / kKeys);
   k_attn_bwd_band_sm100<<<units, kBandThreads, smem, st>>>(mq, mdo, mk, mv, mo, LSE, dm, dK, dV, status_word);
   count_launch(HGA_KERNELS_BWD_TENSOR);

@@ -719,12 +719,13 @@ int launch_attn_bwd_sm100(const Dims& dm, const void* Q, const void* K, const vo
   // the octet table starts inside the struct's tail padding; 1024 bytes of slack for the manual alignment
   const size_t smem = offsetof(BwdSmem, oct_row) + sizeof(int) * (max_routed_tokens(dm) / 8 + 8) + 1024;
   if (smem > 227 * 1024) return HGA_ERR_UNSUPPORTED;
-  cudaError_t e = cudaFuncSetAttribute(k_attn_bwd_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return record_cuda(e);
+  int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(&k_attn_bwd_sm100), smem);
+  if (rc) return rc;
+  cudaError_t e;
   // dK/dV of the local band: written once per key tile by the key-major kernel, with plain stores that
   // cover every row of the active segment (so nothing has to be zero-filled); this kernel then adds the
   // contributions of the keys before the band atomically.
-  const int rc = launch_attn_bwd_band_sm100(dm, Q, K, V, O, LSE, dO, dK, dV, status_word, st);
+  rc = launch_attn_bwd_band_sm100(dm, Q, K, V, O, LSE, dO, dK, dV, status_word, st);
   if (rc != HGA_OK) return rc;
   const int units = dm.B * dm.Hkv * dm.NQB * (dm.rows / 128);
   // The sweep is launched with programmatic serialization behind the band kernel: its CTAs may start on

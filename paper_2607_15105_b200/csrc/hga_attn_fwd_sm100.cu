@@ -476,12 +476,9 @@ static int launch_fwd(const Dims& dm, const void* Q, const void* K, const void* 
     return HGA_ERR_UNSUPPORTED;
   const size_t smem = sizeof(FwdSmem<D>) + sizeof(int) * (max_routed_tokens(dm) / 8 + 8) + 1024;
   if (smem > 113 * 1024) return HGA_ERR_UNSUPPORTED;      // two CTAs per SM
-  cudaError_t e = cudaFuncSetAttribute(k_attn_fwd_sm100<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   // two CTAs per SM need the largest shared-memory carve-out
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_attn_fwd_sm100<D>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             (int)cudaSharedmemCarveoutMaxShared);
-  if (e != cudaSuccess) return record_cuda(e);
+  const int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(&k_attn_fwd_sm100<D>), smem, true);
+  if (rc) return rc;
   const int units = dm.B * dm.Hkv * dm.NQB * ((rows_padded(dm) + 127) / 128);
   k_attn_fwd_sm100<D><<<units, kFwdThreads, smem, st>>>(mq, mk, mv, group_idx, n_groups, dm, (uint16_t*)O, LSE,
                                                        status_word);

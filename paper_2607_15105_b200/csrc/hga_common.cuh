@@ -69,6 +69,9 @@ __host__ __device__ inline int max_routed_tokens(const Dims& dm) {
   return dm.sink + dm.width * dm.g + dm.local + dm.Bq + dm.c;
 }
 
+// cudaFuncSetAttribute(max dynamic shared memory [, maximal carve-out]) for `func`, cached per device (hga_tma.cu)
+int ensure_dynamic_smem(const void* func, size_t bytes, bool max_carveout = false);
+
 // Launch bookkeeping (hga_api.cu).
 void count_launch(int family, int n = 1);   // family: HGA_KERNELS_*
 int record_cuda(cudaError_t e);  // returns HGA_OK or HGA_ERR_CUDA and remembers the code

@@ -526,11 +526,9 @@ static int launch_route(const Dims& dm, const void* Q, const void* chunk_sum, co
     return HGA_ERR_UNSUPPORTED;
   const int max_cand = route_max_cand(dm);
   const size_t smem = route_sm100_smem(dm, max_cand);
-  cudaError_t e = cudaFuncSetAttribute(k_route_sm100<D, STAGES, ACCS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return record_cuda(e);
   // two CTAs per SM need the largest shared-memory carve-out
-  e = cudaFuncSetAttribute(k_route_sm100<D, STAGES, ACCS>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-  if (e != cudaSuccess) return record_cuda(e);
+  const int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(&k_route_sm100<D, STAGES, ACCS>), smem, true);
+  if (rc) return rc;
   const int items = dm.B * dm.Hkv * dm.NQB;
   k_route_sm100<D, STAGES, ACCS><<<items, kRtThreads, smem, st>>>(mq, mc, mg, dm, chunk_idx, group_idx, n_groups, chunk_scores,
                                                    group_scores, ((rows_padded(dm) + 31) & ~31) * D * 2, max_cand);
