@@ -60,7 +60,20 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_trace_harness() -> str:
+    """The timeline harness (trace/hga_trace_harness.cu, -DHGA_TRACE): a stand-alone program, not part of the library."""
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    out = os.path.join(HERE, "hga_trace")
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "--expt-relaxed-constexpr",
+                           "-DHGA_TRACE", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", out,
+                           os.path.join(HERE, "trace", "hga_trace_harness.cu")])
+    return out
+
+
 if __name__ == "__main__":
+    if "--trace" in sys.argv:
+        print(build_trace_harness())
+        sys.exit(0)
     if "--debug-waits" in sys.argv:      # diagnostic build: see csrc/hga_bwd_sm100.cuh
         NVCC_FLAGS.append("-DHGA_DEBUG_WAIT")
     print(build_library(force="--force" in sys.argv or "--debug-waits" in sys.argv, verbose="-v" in sys.argv))

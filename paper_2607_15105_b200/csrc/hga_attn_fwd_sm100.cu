@@ -26,14 +26,7 @@
 #include "hga_common.cuh"
 #include "hga_octets.cuh"
 #include "hga_sm100.cuh"
-
-// Optional phase timers: a profiling harness defines these three macros; otherwise no-ops.
-// HGA_TRACE_POINT(tag) charges the cycles since the previous point to bucket `tag`.
-#ifndef HGA_TRACE_POINT
-#define HGA_TRACE_DECL
-#define HGA_TRACE_POINT(tag)
-#define HGA_TRACE_DUMP
-#endif
+#include "hga_trace.cuh"
 
 namespace hga {
 

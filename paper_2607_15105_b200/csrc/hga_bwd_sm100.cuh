@@ -4,13 +4,7 @@
 #include <cuda_bf16.h>
 
 #include "hga_sm100.cuh"
-
-// Optional phase timers: a profiling harness defines these three macros; otherwise no-ops.
-#ifndef HGA_TRACE_POINT
-#define HGA_TRACE_DECL
-#define HGA_TRACE_POINT(tag)
-#define HGA_TRACE_DUMP
-#endif
+#include "hga_trace.cuh"
 
 namespace hga {
 

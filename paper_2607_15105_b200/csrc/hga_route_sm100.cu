@@ -16,12 +16,6 @@
 #include "hga_common.cuh"
 #include "hga_sm100.cuh"
 
-// Optional phase stamps: a profiling harness defines these macros; otherwise no-ops.
-#ifndef HGA_RT_STAMP
-#define HGA_RT_DECL
-#define HGA_RT_STAMP(k)
-#endif
-
 namespace hga {
 
 using namespace sm100;
@@ -77,7 +71,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   uint32_t* okeys = reinterpret_cast<uint32_t*>(sm.sel) + 64;   // orderable scores alone, when candidates <= 640
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  HGA_RT_DECL;
   const int item = blockIdx.x;
   int b, h, qb;
   item_coords(dm, item, b, h, qb);
@@ -117,7 +110,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         tma_load_5d(sm.a[s] + lane * kOctBytes, &map_gs, &sm.a_full[s], 0, row, 0, h, b);
       }
     }
-    HGA_RT_STAMP(3 + tg);
   };
   const int n_pre = k_sel > 0 ? (n_ct < STAGES ? n_ct : STAGES) : 0;   // chunk tiles copied ahead of the CTA barrier
 
@@ -146,7 +138,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sm.tmem_base;
-  HGA_RT_STAMP(1);
 
   // One GEMM phase: tiles [t_begin, t_begin + n_tiles) in the global tile numbering (which
   // drives barrier parities); `phase2` selects the octet source.
@@ -158,7 +149,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const int r = 8 * o, a = r / bq_pad, t = r % bq_pad;    // rows past the segment arrive as zeros
         tma_load_5d(q_smem + o * kOctBytes, &map_q, &sm.q_full, 0, qb * dm.Bq + t, 0, h * dm.G + a, b);
       }
-      HGA_RT_STAMP(2);
     }
     if (phase2 && warp >= 2 && lane < 2) {
       // First tile of the opened chunks' group summaries, again spread over the eight warps (two
@@ -176,7 +166,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       if (phase2) {
         tiles_issued = t_begin + 1;        // (its boxes come from the other warps, see above)
         if (lane == 0) mbar_arrive_expect_tx(&sm.a_full[t_begin % STAGES], Smem::kTile);
-        HGA_RT_STAMP(3 + t_begin);
       }
       for (int t = phase2 ? 1 : n_pre; t < n_tiles; ++t) {
         const int tg = t_begin + t, s = tg % STAGES, use = tg / STAGES;
@@ -194,11 +183,9 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         };
         const uint32_t idesc = idesc_bf16_f32(128, rows_half, 0, 0);
         bool ok = phase2 ? true : mma_wait(&sm.q_full, 0, abort);
-        if (!phase2) HGA_RT_STAMP(2);
         for (int t = 0; t < n_tiles && ok; ++t) {
           const int tg = t_begin + t, s = tg % STAGES;
           ok = mma_wait(&sm.a_full[s], (tg / STAGES) & 1, abort);
-          HGA_RT_STAMP(3 + tg);
           for (int hf = 0; hf < n_halves && ok; ++hf) {
             const int step = tg * n_halves + hf, buf = step % ACCS, use = step / ACCS;
             if (use > 0) ok = mma_wait(&sm.acc_free[buf], (use - 1) & 1, abort);
@@ -215,7 +202,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             mma_commit_w(&sm.acc_full[buf]);
           }
           if (ok) mma_commit_w(&sm.a_empty[s]);
-          HGA_RT_STAMP(12 + tg);
         }
       }
     } else if (warp < 6) {
@@ -232,7 +218,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
           ok = __all_sync(0xffffffffu, rt_wait(&sm.acc_full[buf], (step / ACCS) & 1, abort));
           if (!ok) break;
           tc_fence_after_sync();
-          HGA_RT_STAMP(3 + tg);
           for (int c = 0; c < rows_half; c += 32) {
             uint32_t x[32];
             tmem_ld32(lane_base + buf * kAccCols + c, x);
@@ -264,7 +249,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
           }
           tc_fence_before_sync();
           mbar_arrive(&sm.acc_free[buf]);
-          HGA_RT_STAMP(12 + tg);
         }
         if (!ok) break;
         if (agg == 1) best = sum * (1.f / (float)dm.rows);
@@ -294,7 +278,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   if (k_sel > 0) run_phase(0, n_ct, false);
   __syncwarp();          // the roles diverge inside a warp: reconverge before the block barrier
   __syncthreads();
-  HGA_RT_STAMP(20);
 
   // ---------------------------------------------------------------------- chunk top-k
   if (!sm.abort) {
@@ -338,9 +321,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
           if (lane == 0 && base + warp * 32 < n_cand) flags[(base + warp * 32) >> 5] = word;
         }
       };
-      HGA_RT_STAMP(24);
       rank_select(false);
-      HGA_RT_STAMP(25);
       __syncthreads();
       int n_picked = 0;
       for (int q = 0; q < (n_cand + 31) / 32; ++q) n_picked += __popc(flags[q]);
@@ -349,7 +330,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         rank_select(true);
         __syncthreads();
       }
-      HGA_RT_STAMP(26);
       for (int i = tid; i < n_cand; i += kRtThreads) {
         if ((flags[i >> 5] >> (i & 31)) & 1u) {
           int pos = __popc(flags[i >> 5] & ((1u << (i & 31)) - 1u));
@@ -392,11 +372,9 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   __syncthreads();
 
   // ---------------------------------------------------------------------- groups of the opened chunks
-  HGA_RT_STAMP(21);
   if (k_sel > 0 && !sm.abort) run_phase(n_ct, n_gt, true);
   __syncwarp();
   __syncthreads();
-  HGA_RT_STAMP(22);
   if (!sm.abort) {
     int32_t* gi = group_idx + (int64_t)item * dm.width;
     const bool global_budget = (dm.flags & HGA_FLAG_GLOBAL_GROUP_BUDGET) != 0;
@@ -454,7 +432,6 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     if (tid == 0) n_groups[item] = k_sel * dm.kge;
   }
 
-  HGA_RT_STAMP(23);
   if (sm.abort) {
     // A bounded wait gave up: the item's routing is marked invalid (the attention calls report a negative
     // count and use no routed groups for that item), and the copies still in flight get a bounded time to land
