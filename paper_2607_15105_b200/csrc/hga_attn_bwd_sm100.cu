@@ -632,7 +632,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tma_store_5d(&map_dq, sm.q + panel * 16384 + half * 8192, 0, qb * dm.Bq + r0 % dm.Bq, panel,
                      h * dm.G + r0 / dm.Bq, b);
         tma_store_commit();
-        tma_store_wait_all();
+        tma_store_wait_read();      // (the source tile has been read; the writes complete before the grid does)
       }
     }
   } else {
