@@ -91,8 +91,9 @@ extern "C" {
                                   [B,Hkv,S,d] (the dtype of K and V, so the call is a drop-in autograd
                                   node) instead of fp32.  The sums over query blocks still run in fp32,
                                   in the workspace (hga_workspace_bytes grows accordingly), and are
-                                  rounded once at the end.  Not with HGA_FLAG_BWD_ACCUMULATE, not in
-                                  hga_step_host (HGA_ERR_UNSUPPORTED). */
+                                  rounded once at the end (one conversion launch for both tensors,
+                                  released early by the last attention kernel).  Not with
+                                  HGA_FLAG_BWD_ACCUMULATE, not in hga_step_host (HGA_ERR_UNSUPPORTED). */
 
 /* bits OR-ed into *status_word by the attention kernels */
 #define HGA_STATUS_BAD_INDEX 1     /* a group_idx entry was out of range, inside the sink or

@@ -261,14 +261,17 @@ int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* 
   const bool zero_grads = !(dm.flags & HGA_FLAG_BWD_ACCUMULATE);
   const size_t n_kv = (size_t)dm.B * dm.Hkv * dm.S * dm.d;
   if (bf16_grads) {
-    // the sums over query blocks run in fp32 in the workspace and are rounded once at the end
+    // the sums over query blocks run in fp32 in the workspace and are rounded once at the end, by one
+    // conversion launch for both tensors
     dK = (float*)((char*)workspace + bwd_delta_bytes(dm));
     dV = dK + n_kv;
   }
   rc = HGA_ERR_UNSUPPORTED;
+  bool tensor_path = false;
   if (attn_bwd_sm100_supported(dm)) {
     // its band kernel stores every row of dK/dV (or adds to it); UNSUPPORTED is returned before any launch
     rc = launch_attn_bwd_sm100(dm, Q, K, V, O, LSE, dO, group_idx, n_groups, dQ, dK, dV, status_word, st);
+    tensor_path = rc == HGA_OK;
   }
   if (rc == HGA_ERR_UNSUPPORTED) {
     if (zero_grads) {
@@ -281,9 +284,7 @@ int hga_attn_bwd(const hga_params* p, const void* Q, const void* K, const void* 
                                  (float*)workspace, status_word, st);
   }
   if (rc || !bf16_grads) return rc;
-  rc = launch_grads_to_bf16(dK, dK_out, n_kv, st);
-  if (rc) return rc;
-  return launch_grads_to_bf16(dV, dV_out, n_kv, st);
+  return launch_grads_to_bf16(dK, dK_out, dV_out, n_kv, tensor_path && !(dm.flags & kFlagNoPdl), st);
 }
 
 int hga_step_arena_bytes(const hga_params* p, size_t* bytes) {

@@ -151,6 +151,8 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   if (warp == 1) {
     tmem_alloc(&sm.tmem_base, 512);
     tmem_relinquish();
+    // with bf16 outputs the conversion kernel follows this grid: let its launch overlap this grid's tail
+    if (lane == 0 && (dm.flags & HGA_FLAG_BWD_BF16_GRADS)) pdl_launch_dependents();
   }
   if (warp == 0) {
     if (lane == 0) { prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); }

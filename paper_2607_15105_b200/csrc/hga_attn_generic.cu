@@ -298,22 +298,35 @@ static size_t token_smem_bytes(const Dims& dm) {
   return sizeof(int) * ((size_t)max_routed_tokens(dm) + dm.width + 4);
 }
 
-// dK/dV accumulators (fp32) -> bf16 output, eight elements per thread
-__global__ void __launch_bounds__(256) k_grads_to_bf16(const float4* __restrict__ src, uint4* __restrict__ dst, size_t n8) {
+// dK/dV accumulators (fp32, adjacent: dV's follow dK's) -> the two bf16 outputs, eight elements per thread
+__global__ void __launch_bounds__(256) k_grads_to_bf16(const float4* __restrict__ src, uint4* __restrict__ dst_k,
+                                                       uint4* __restrict__ dst_v, size_t n8) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n8) return;
+  // (a no-op unless launched with programmatic serialization: then the sums are complete only from here on)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (i >= 2 * n8) return;
   const float4 a = src[2 * i], b = src[2 * i + 1];
   const __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x, a.y), h1 = __floats2bfloat162_rn(a.z, a.w);
   const __nv_bfloat162 h2 = __floats2bfloat162_rn(b.x, b.y), h3 = __floats2bfloat162_rn(b.z, b.w);
-  dst[i] = make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
-                      *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
+  uint4* dst = i < n8 ? dst_k + i : dst_v + (i - n8);
+  *dst = make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
+                    *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
 }
 
-int launch_grads_to_bf16(const float* src, void* dst, size_t n, cudaStream_t st) {
+int launch_grads_to_bf16(const float* src, void* dst_k, void* dst_v, size_t n, bool after_sweep, cudaStream_t st) {
   const size_t n8 = n / 8;
-  k_grads_to_bf16<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>((const float4*)src, (uint4*)dst, n8);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((2 * n8 + 255) / 256));
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = after_sweep ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, k_grads_to_bf16, (const float4*)src, (uint4*)dst_k, (uint4*)dst_v, n8);
   count_launch(HGA_KERNELS_AUX);
-  return record_cuda(cudaGetLastError());
+  return record_cuda(e);
 }
 
 int launch_attn_fwd_generic(const Dims& dm, const void* Q, const void* K, const void* V,

@@ -118,7 +118,9 @@ int resolve_params(const hga_params* p, Dims& dm);
 size_t route_workspace_bytes(const Dims& dm);
 size_t bwd_workspace_bytes(const Dims& dm);
 
-// fp32 -> bf16 (round to nearest even) of n elements, n a multiple of 8 (hga_attn_generic.cu)
-int launch_grads_to_bf16(const float* src, void* dst, size_t n, cudaStream_t st);
+// fp32 -> bf16 (round to nearest even): src holds n dK sums followed by n dV sums, n a multiple of 8; one
+// launch for both tensors.  after_sweep: launched with programmatic serialization behind the tensor-core sweep
+// (which releases it early in that mode), so that its launch overlaps the sweep's tail (hga_attn_generic.cu)
+int launch_grads_to_bf16(const float* src, void* dst_k, void* dst_v, size_t n, bool after_sweep, cudaStream_t st);
 
 }  // namespace hga

@@ -103,3 +103,33 @@ def test_config_against_oracle(n, full_head, extra):
         touched[tok[tok >= H] - H] = True
     if (~touched).any():
         assert float(buf.dK[b, h][torch.from_numpy(~touched).cuda()].abs().max()) == 0.0
+
+
+def test_config3_bf16_gradient_outputs_at_full_size():
+    """HGA_FLAG_BWD_BF16_GRADS at configuration 3, in the launch configuration bench.py times: the two
+    tensor-core kernels sum in fp32 in the workspace and ONE conversion launch (released early by the sweep)
+    rounds both tensors, so dK/dV must equal the fp32 call's result rounded once."""
+    cfg = CONFIGS[3]
+    x = make_inputs(cfg)
+    Q, K, V, dO = (to_dev(x[k]) for k in ("Q", "K", "V", "dO"))
+    res = {}
+    for extra in (0, binding.HGA_FLAG_BWD_BF16_GRADS):
+        buf = binding.HgaLayerBuffers(cfg, flags=extra)
+        buf.build_summaries(K, 0, cfg.history)
+        buf.step(Q, K, V, None)
+        before = binding.hga_kernel_launch_counts()
+        buf.attn_bwd(Q, K, V, dO, buf.group_idx, buf.n_groups)
+        torch.cuda.synchronize()
+        assert int(buf.status.item()) == 0
+        ran = [b - a for a, b in zip(before, binding.hga_kernel_launch_counts())]
+        assert ran[binding.HGA_KERNELS_BWD_TENSOR] == 2 and ran[binding.HGA_KERNELS_AUX] == (1 if extra else 0), ran
+        res[extra] = (buf.dQ.clone(), buf.dK.clone(), buf.dV.clone())
+    (dQ32, dK32, dV32), (dQ16, dK16, dV16) = res[0], res[binding.HGA_FLAG_BWD_BF16_GRADS]
+    assert dK16.dtype == torch.bfloat16 and dV16.dtype == torch.bfloat16
+    assert torch.equal(dQ32, dQ16)
+    for a32, a16 in ((dK32, dK16), (dV32, dV16)):
+        ref = a32.double()
+        err = (a16.double() - ref).abs()
+        # one rounding to 8 significant bits, plus the run-to-run wobble of the fp32 atomics
+        assert bool((err <= ref.abs() * 2.0 ** -8 + 1e-5).all())
+        assert float(a16.double().abs().max()) > 0.0

@@ -336,9 +336,15 @@ def test_bf16_gradient_outputs(name, flags):
     for extra in (0, binding.HGA_FLAG_BWD_BF16_GRADS):
         buf = binding.HgaLayerBuffers(cfg, flags=flags | extra)
         buf.attn_fwd(c.Q, c.K, c.V, c.gi, c.ng)
+        before = binding.hga_kernel_launch_counts()
         buf.attn_bwd(c.Q, c.K, c.V, c.dO, c.gi, c.ng)
         torch.cuda.synchronize()
         assert int(buf.status.item()) == 0
+        ran = [b - a for a, b in zip(before, binding.hga_kernel_launch_counts())]
+        # one conversion launch for both tensors, behind either kernel family
+        tensor = flags == 0 and cfg.head_dim == 128
+        assert ran[binding.HGA_KERNELS_AUX] == (1 if extra else 0), ran
+        assert (ran[binding.HGA_KERNELS_BWD_TENSOR] == 2) == tensor, ran
         outs[extra] = (buf.dQ.clone(), buf.dK.clone(), buf.dV.clone())
     (dQ32, dK32, dV32), (dQ16, dK16, dV16) = outs[0], outs[binding.HGA_FLAG_BWD_BF16_GRADS]
     assert dK16.dtype == torch.bfloat16 and dV16.dtype == torch.bfloat16
