@@ -11,11 +11,13 @@
 // selected through routing (and of sink keys inside the active segment), and computes dQ.
 //
 // The GEMMs are the TRANSPOSED ones, so that P and dS never pass through shared memory:
-//   S^T  = K Q^T,  dP^T = V dO^T         (M = 128 keys, N = 128 query rows, K = head_dim)  smem x smem
+//   S^T  = K Q^T,  dP^T = V dO^T         (M = 128 keys, N = 64 query rows, K = head_dim)   smem x smem
 //   P^T  = 2^(S^T*c - LSE*log2e),  dS^T = scale * P^T o (dP^T - delta)    one thread per KEY (TMEM lane),
 //          written back as bf16 over the columns just read
-//   dV  += P^T dO,  dK += dS^T Q         (M = 128 keys, N = head_dim, K = 128 query rows)  A from TMEM
-// All of them are M = 128, N = 128 instructions (full tensor-pipe rate).
+//   dV  += P^T dO,  dK += dS^T Q         (M = 128 keys, N = head_dim, K = 64 query rows)   A from TMEM
+// An M-tile (128 query rows) is taken in two HALF-STEPS of 64 rows that alternate between two 128-column
+// regions of tensor memory, so that the GEMMs of one half-step run while the key threads work on the other
+// (with one 256-column region per M-tile the tensor pipe idled through the key threads' work and vice versa).
 // delta = rowsum(dO o O) of the M-tile's rows is computed here, by four otherwise idle warps (one
 // thread per query row, from the O and dO tiles in shared memory; the O tile arrives by TMA one step
 // ahead), so the backward needs no separate pass over O and dO.
@@ -23,9 +25,9 @@
 // Work unit (one CTA): (batch, kv head, 128-key tile of the active segment); keys past the end of the
 // segment arrive as zeros, are masked by causality and are not stored.
 // Warp roles (448 threads): warp 0 producer (K, V once; Q, dO tiles through a two-stage ring, O tiles one at a time),
-// warp 1 MMA issuer, warps 2-5 and 6-9 one thread per key (warpgroup w: query rows 64w .. 64w+63 of
-// the M-tile), warps 10-13 row statistics (LSE, delta).
-// TMEM (512 columns): S^T / P^T | dP^T / dS^T | dV | dK, 128 columns each.
+// warp 1 MMA issuer, warps 2-5 and 6-9 one thread per key (warpgroup w: query rows 32w .. 32w+31 of
+// every half-step), warps 10-13 row statistics (LSE, delta).
+// TMEM (512 columns): two regions of [S^T / P^T (64) | dP^T / dS^T (64)], then dV and dK, 128 columns each.
 #include "hga_bwd_sm100.cuh"
 #include "hga_common.cuh"
 #include "hga_sm100.cuh"
@@ -49,8 +51,10 @@ struct BandSmem {
   alignas(1024) uint8_t o[kTile];                // (q, dO and o, contiguous, also stage the dV / dK tiles on their way out)
   alignas(16) float nlse[128];                   // per query row of the current M-tile: -LSE * log2(e)
   alignas(16) float nds[128];                    //                                      -delta * scale
-  uint64_t kv_full, qdo_full[2], qdo_empty[2], o_full, o_empty, stat_full;
-  uint64_t s_full, dp_full, pds_full, acc_done, drain;
+  uint64_t kv_full, qdo_full[2][2], qdo_empty[2][2], o_full, o_empty;   // Q/dO: [ring stage][half of the M-tile's rows]
+  // per half of the M-tile (= per region of tensor memory), so that every barrier completes once per step and
+  // each completion depends on its waiter having seen the previous one
+  uint64_t stat_full[2], sdp_full[2], pds_full[2], acc_done, drain;
   uint32_t tmem_base;
   volatile int abort;
 };
@@ -67,7 +71,7 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
                       const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                       const __grid_constant__ CUtensorMap map_o, const float* __restrict__ LSE, Dims dm,
                       float* __restrict__ dK, float* __restrict__ dV, int32_t* status_word) {
-  constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
+  constexpr uint32_t kColS = 0, kColDP = 64, kRegion = 128, kColDV = 256, kColDK = 384;   // (S^T, dP^T: inside a region)
   extern __shared__ uint8_t smem_raw[];
   BandSmem& sm = *reinterpret_cast<BandSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
@@ -90,14 +94,21 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
 
   if (tid == 0) {
     mbar_init(&sm.kv_full, 1);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.qdo_full[s], 1); mbar_init(&sm.qdo_empty[s], 1);
+    for (int s = 0; s < 4; ++s) {
+      mbar_init(&sm.qdo_full[s >> 1][s & 1], 1); mbar_init(&sm.qdo_empty[s >> 1][s & 1], 1);
     }
-    mbar_init(&sm.o_full, 1); mbar_init(&sm.o_empty, 128); mbar_init(&sm.stat_full, 128);
-    mbar_init(&sm.s_full, 1); mbar_init(&sm.dp_full, 1); mbar_init(&sm.pds_full, 256);
+    mbar_init(&sm.o_full, 1); mbar_init(&sm.o_empty, 128);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sm.stat_full[s], 64); mbar_init(&sm.sdp_full[s], 1); mbar_init(&sm.pds_full[s], 256);
+    }
     mbar_init(&sm.acc_done, 1); mbar_init(&sm.drain, 1);
     sm.abort = 0;
     fence_barrier_init();
+    // the copies of the K and V tile, of the first two steps' Q and dO and of the first O tile are issued by
+    // twelve warps at once right after the block barrier below; their byte counts are announced here
+    mbar_arrive_expect_tx(&sm.kv_full, 2 * kTile);
+    mbar_arrive_expect_tx(&sm.o_full, kTile);
+    for (int s = 0; s < (n_steps > 1 ? 4 : 2); ++s) mbar_arrive_expect_tx(&sm.qdo_full[s >> 1][s & 1], kTile);
   }
   if (warp == 1) {
     tmem_alloc(&sm.tmem_base, 512);
@@ -115,50 +126,79 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
   volatile int* abort = &sm.abort;
   HGA_TRACE_POINT(1);
 
+  // A copy is latency-bound per box and costs its issuing warp a few hundred cycles, so every tile travels as
+  // four boxes of 64 rows x one 64-element panel (8 KB each); the 28 boxes a CTA starts with go out from
+  // twelve warps in parallel, in the order they are needed: K, V, the first half-step's Q and dO rows, the
+  // second half-step's, the first O tile, then the second step's Q and dO.
+  auto qdo_coords = [&](int m, int half, int& row, int& head) {
+    const Step sp = step_of(m);
+    const int r = sp.r0 + 64 * half;
+    row = sp.qb * dm.Bq + r % dm.Bq;
+    head = h * dm.G + r / dm.Bq;
+  };
+  if (warp >= 2 && lane == 0) {
+    for (int i = warp - 2; i < (n_steps > 1 ? 28 : 20); i += 12) {
+      int row, head;
+      // All CTAs start at once and HBM is the bottleneck of these first microseconds: what the first
+      // half-step needs (the first twelve boxes) goes out alone, the rest once that has arrived
+      if (i >= 12 && !(bwd_wait(&sm.kv_full, 0, abort) && bwd_wait(&sm.qdo_full[0][0], 0, abort))) break;
+      if (i < 8) {                                   // K, V: (half, panel) = (i & 1, (i >> 1) & 1)
+        const int half = i & 1, panel = (i >> 1) & 1;
+        const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
+        tma_load_5d((i < 4 ? sm.k : sm.v) + off, i < 4 ? &map_k : &map_v, &sm.kv_full, 0, k0 + 64 * half, panel, h, b);
+      } else if (i < 16) {                           // step 0: half (i - 8) / 4, then Q panel 0, 1, dO panel 0, 1
+        const int half = (i - 8) >> 2, panel = i & 1, is_do = (i >> 1) & 1;
+        const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
+        qdo_coords(0, half, row, head);
+        tma_load_5d((is_do ? sm.dO[0] : sm.q[0]) + off, is_do ? &map_do : &map_q, &sm.qdo_full[0][half], 0, row, panel, head, b);
+      } else if (i < 20) {                           // O tile of step 0
+        const int half = i & 1, panel = (i >> 1) & 1;
+        const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
+        qdo_coords(0, half, row, head);
+        tma_load_5d(sm.o + off, &map_o, &sm.o_full, 0, row, panel, head, b);
+      } else {                                       // step 1, as step 0
+        const int half = (i - 20) >> 2, panel = i & 1, is_do = (i >> 1) & 1;
+        const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
+        qdo_coords(1, half, row, head);
+        tma_load_5d((is_do ? sm.dO[1] : sm.q[1]) + off, is_do ? &map_do : &map_q, &sm.qdo_full[1][half], 0, row, panel, head, b);
+      }
+    }
+  }
+  __syncwarp();
+
   if (warp == 0) {
-    // ------------------------------------------------------------------ producer
-    // A copy is latency-bound per box, so every tile travels as four boxes of 64 rows x one 64-element
-    // panel (8 KB each), issued by up to twelve lanes at once: lanes 0-3 K or Q, lanes 4-7 V or dO, lanes 8-11 O.
-    const int half = lane & 1, panel = (lane >> 1) & 1;
-    const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)half * 8192;
+    // ------------------------------------------------------------------ producer (Q and dO from the third step on)
     if (lane == 0) {
       prefetch_tensormap(&map_q); prefetch_tensormap(&map_do);
-      prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); prefetch_tensormap(&map_o);
-      mbar_arrive_expect_tx(&sm.kv_full, 2 * kTile);
     }
-    __syncwarp();
-    if (lane < 4) tma_load_5d(sm.k + off, &map_k, &sm.kv_full, 0, k0 + 64 * half, panel, h, b);
-    else if (lane < 8) tma_load_5d(sm.v + off, &map_v, &sm.kv_full, 0, k0 + 64 * half, panel, h, b);
     bool ok = true;
-    int issued = 0, o_issued = 0;
-    for (int m = 0; m < n_steps; ++m) {
+    int issued = n_steps > 1 ? 4 : 2;                // half-steps whose copies have been issued
+    for (int m = 2; m < n_steps && ok; ++m) {
       const int st = m & 1;
-      const Step sp = step_of(m);
-      const int r = sp.r0 + 64 * half;
-      const int row = sp.qb * dm.Bq + r % dm.Bq, head = h * dm.G + r / dm.Bq;
-      // the O tile of step m: its single buffer is free once the statistics warps have read step m-1's
-      if (lane == 0 && m >= 1) ok = bwd_wait(&sm.o_empty, (m - 1) & 1, abort);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      if (lane == 0) mbar_arrive_expect_tx(&sm.o_full, kTile);
-      __syncwarp();
-      if (lane >= 8 && lane < 12) tma_load_5d(sm.o + off, &map_o, &sm.o_full, 0, row, panel, head, b);
-      o_issued = m + 1;
-      if (lane == 0 && m >= 2) ok = bwd_wait(&sm.qdo_empty[st], ((m >> 1) - 1) & 1, abort);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      if (lane == 0) mbar_arrive_expect_tx(&sm.qdo_full[st], 2 * kTile);
-      __syncwarp();
-      if (lane < 4) tma_load_5d(sm.q[st] + off, &map_q, &sm.qdo_full[st], 0, row, panel, head, b);
-      else if (lane < 8) tma_load_5d(sm.dO[st] + off, &map_do, &sm.qdo_full[st], 0, row, panel, head, b);
-      issued = m + 1;
-      HGA_TRACE_POINT(2);
+      // one half of the rows (Q panel 0, 1, dO panel 0, 1: lanes 0-3) at a time: a half is free again as soon
+      // as the GEMMs of its half-step two steps ago are done
+      for (int hf = 0; hf < 2 && ok; ++hf) {
+        if (lane == 0) ok = bwd_wait(&sm.qdo_empty[st][hf], ((m >> 1) - 1) & 1, abort);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        if (lane == 0) mbar_arrive_expect_tx(&sm.qdo_full[st][hf], kTile);
+        __syncwarp();
+        if (lane < 4) {
+          const int panel = lane & 1, is_do = lane >> 1;
+          const uint32_t off = (uint32_t)panel * 16384 + (uint32_t)hf * 8192;
+          int row, head;
+          qdo_coords(m, hf, row, head);
+          tma_load_5d((is_do ? sm.dO[st] : sm.q[st]) + off, is_do ? &map_do : &map_q, &sm.qdo_full[st][hf], 0, row, panel, head, b);
+        }
+        issued = 2 * m + hf + 1;
+        HGA_TRACE_POINT(2);
+      }
     }
     if (*abort && lane == 0) {
       // giving up: let the copies still in flight land before shared memory is released
       mbar_wait(&sm.kv_full, 0);
-      for (int m = issued > 2 ? issued - 2 : 0; m < issued; ++m) mbar_wait(&sm.qdo_full[m & 1], (m >> 1) & 1);
-      if (o_issued > 0) mbar_wait(&sm.o_full, (o_issued - 1) & 1);
+      for (int hs = issued > 4 ? issued - 4 : 0; hs < issued; ++hs)
+        mbar_wait(&sm.qdo_full[(hs >> 1) & 1][hs & 1], (hs >> 2) & 1);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -167,17 +207,18 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
       auto mma_wait = [&](uint64_t* bar, uint32_t parity, volatile int* ab) {
         return __all_sync(0xffffffffu, bwd_wait(bar, parity, ab));
       };
-      constexpr uint32_t idesc_t = idesc_bf16_f32(128, 128, 0, 0);     // keys x rows: A, B K-major (head_dim runs along K)
+      constexpr uint32_t idesc_t = idesc_bf16_f32(128, 64, 0, 0);      // keys x 64 rows: A, B K-major (head_dim runs along K)
       constexpr uint32_t idesc_g = idesc_bf16_f32(128, kD, 0, 1);      // keys x head_dim: A from TMEM, B MN-major
       // every tile is [panel][128 rows][128 B]: K-major with 8-row groups 1024 B apart and the second
-      // panel 16 KB on; MN-major (head_dim along N, rows along K) with panels 16 KB and 8-row groups 1024 B apart
+      // panel 16 KB on; MN-major (head_dim along N, rows along K) with panels 16 KB and 8-row groups 1024 B apart.
+      // The rows of half-step hf start 64 * 128 B = 8 KB into each panel.
       const uint64_t k_k = smem_desc_sw128(smem_u32(sm.k), 16, 1024);
       const uint64_t v_k = smem_desc_sw128(smem_u32(sm.v), 16, 1024);
       const uint64_t q_k0 = smem_desc_sw128(smem_u32(sm.q[0]), 16, 1024);
       const uint64_t do_k0 = smem_desc_sw128(smem_u32(sm.dO[0]), 16, 1024);
       const uint64_t q_mn0 = smem_desc_sw128(smem_u32(sm.q[0]), 16384, 1024);
       const uint64_t do_mn0 = smem_desc_sw128(smem_u32(sm.dO[0]), 16384, 1024);
-      // acc (keys x rows) = a (K or V tile) x b^T (Q or dO tile), both K-major
+      // acc (keys x 64 rows) = a (K or V tile) x b^T (64 rows of the Q or dO tile), both K-major
       auto issue_t = [&](uint32_t acc, uint64_t a, uint64_t bq) {
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
@@ -185,44 +226,49 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
           mma_ss_w(acc, desc_advance(a, off), desc_advance(bq, off), idesc_t, kk > 0);
         }
       };
-      // acc (keys x head_dim) += a (keys x rows, bf16 in TMEM: rows 0-63 at columns 0-31, rows 64-127 at
-      // columns 64-95 of its region) x b (Q or dO tile: rows along K, 16 rows per instruction)
+      // acc (keys x head_dim) += a (keys x 64 rows, bf16 in TMEM: rows 0-31 at columns 0-15, rows 32-63 at
+      // columns 32-47 of its S^T or dP^T part) x b (64 rows of the Q or dO tile: rows along K, 16 per instruction)
       auto issue_g = [&](uint32_t acc, uint32_t a_tmem, uint64_t bmn, bool accumulate) {
 #pragma unroll
-        for (int kk = 0; kk < 128 / 16; ++kk)
-          mma_ts_w(acc, a_tmem + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), desc_advance(bmn, kk * 2048), idesc_g,
-                 (accumulate || kk > 0));
+        for (int kk = 0; kk < 64 / 16; ++kk)
+          mma_ts_w(acc, a_tmem + (kk < 2 ? 8 * kk : 32 + 8 * (kk - 2)), desc_advance(bmn, kk * 2048), idesc_g,
+                   (accumulate || kk > 0));
       };
-      bool ok = mma_wait(&sm.kv_full, 0, abort) && mma_wait(&sm.qdo_full[0], 0, abort);
-      if (ok) {
+      // S^T and dP^T of half-step hf of the M-tile in ring stage st, into region hf
+      auto issue_sdp = [&](uint32_t st, uint32_t hf) {
+        const uint32_t region = tmem + hf * kRegion, off = st * kTile + hf * 8192;
+        issue_t(region + kColS, k_k, desc_advance(q_k0, off));
+        issue_t(region + kColDP, v_k, desc_advance(do_k0, off));
+        mma_commit_w(&sm.sdp_full[hf]);
+      };
+      const int n_half = 2 * n_steps;
+      bool ok = mma_wait(&sm.kv_full, 0, abort);
+      for (uint32_t hf = 0; hf < 2 && ok; ++hf) {
+        ok = mma_wait(&sm.qdo_full[0][hf], 0, abort);
+        if (!ok) break;
         tc_fence_after_sync();
-        issue_t(tmem + kColS, k_k, q_k0);
-        mma_commit_w(&sm.s_full);
-        issue_t(tmem + kColDP, v_k, do_k0);
-        mma_commit_w(&sm.dp_full);
+        issue_sdp(0, hf);
       }
       HGA_TRACE_POINT(3);
-      for (int m = 0; m < n_steps && ok; ++m) {
-        const uint32_t st = (uint32_t)(m & 1), st_n = st ^ 1u;
-        const bool more = m + 1 < n_steps;
-        ok = mma_wait(&sm.pds_full, m & 1, abort);               // P^T and dS^T of step m are in TMEM
+      for (int hs = 0; hs < n_half && ok; ++hs) {
+        const int m = hs >> 1;
+        const uint32_t st = (uint32_t)(m & 1), hf = (uint32_t)(hs & 1);
+        ok = mma_wait(&sm.pds_full[hf], m & 1, abort);           // P^T and dS^T of this half-step are in TMEM
         if (!ok) break;
         tc_fence_after_sync();
         HGA_TRACE_POINT(5);
-        issue_g(tmem + kColDV, tmem + kColS, desc_advance(do_mn0, st * kTile), m > 0);
-        if (more) {
-          // S^T of the next M-tile overwrites P^T: the in-order tensor pipe runs it after the dV GEMM above
-          ok = mma_wait(&sm.qdo_full[st_n], ((m + 1) >> 1) & 1, abort);
+        const uint32_t region = tmem + hf * kRegion, off = st * kTile + hf * 8192;
+        issue_g(tmem + kColDV, region + kColS, desc_advance(do_mn0, off), hs > 0);
+        issue_g(tmem + kColDK, region + kColDP, desc_advance(q_mn0, off), hs > 0);
+        mma_commit_w(&sm.qdo_empty[st][hf]);                     // these 64 rows of Q and dO are consumed
+        if (hs + 2 < n_half) {
+          // the same half of the next M-tile reuses this region: the in-order tensor pipe runs its GEMMs after
+          // the two above, which read P^T and dS^T from it
+          const uint32_t st_n = st ^ 1u;
+          ok = mma_wait(&sm.qdo_full[st_n][hf], ((m + 1) >> 1) & 1, abort);
           if (!ok) break;
           tc_fence_after_sync();
-          issue_t(tmem + kColS, k_k, desc_advance(q_k0, st_n * kTile));
-          mma_commit_w(&sm.s_full);
-        }
-        issue_g(tmem + kColDK, tmem + kColDP, desc_advance(q_mn0, st * kTile), m > 0);
-        mma_commit_w(&sm.qdo_empty[st]);                           // Q and dO of step m are consumed
-        if (more) {
-          issue_t(tmem + kColDP, v_k, desc_advance(do_k0, st_n * kTile));
-          mma_commit_w(&sm.dp_full);
+          issue_sdp(st_n, hf);
         }
         HGA_TRACE_POINT(7);
       }
@@ -230,85 +276,76 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
     }
   } else if (warp < 10) {
     // ------------------------------------------------------------------ one thread per key
-    const int wg = (warp - 2) >> 2;                  // query rows 64*wg .. 64*wg+63 of each M-tile
+    const int wg = (warp - 2) >> 2;                  // query rows 32*wg .. 32*wg+31 of every half-step
     const int quarter = warp & 3;                    // TMEM lanes this warp may touch
     const int key = quarter * 32 + lane;
     const int kp = k0 + key;                         // absolute position of this thread's key
     const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
-    const uint32_t s_addr = lane_base + kColS + 64 * wg, dp_addr = lane_base + kColDP + 64 * wg;
     const float sl2 = dm.scale * 1.4426950408889634f;
     const uint64_t sl2_2 = pack_f32x2(sl2, sl2), scale_2 = pack_f32x2(dm.scale, dm.scale);
     bool ok = true;
-    for (int m = 0; m < n_steps; ++m) {
+    for (int hs = 0; hs < 2 * n_steps; ++hs) {
+      const int m = hs >> 1, hf = hs & 1;
       const Step sp = step_of(m);
       const Window w = window_of(dm, sp.qb);
-      // the warpgroup's 64 columns are 64 consecutive positions of one query head (Bq is a multiple of 64);
+      // the warpgroup's 32 columns are 32 consecutive positions of one query head (Bq is a multiple of 64);
       // column i is visible to this key iff the key is inside the block's band and not after the query
-      const int qp0 = w.p0 + (sp.r0 + 64 * wg) % dm.Bq;
-      const int imin = (kp < w.ls || kp >= k_end) ? 64 : kp - qp0;       // first visible column (may be <= 0)
-      const bool none = __all_sync(0xffffffffu, imin >= 64);
+      const int r_first = 64 * hf + 32 * wg;         // first of those rows inside the M-tile
+      const int qp0 = w.p0 + (sp.r0 + r_first) % dm.Bq;
+      const int imin = (kp < w.ls || kp >= k_end) ? 32 : kp - qp0;       // first visible column (may be <= 0)
+      const bool none = __all_sync(0xffffffffu, imin >= 32);
       const bool masked = __any_sync(0xffffffffu, imin > 0);
-      const uint32_t nlse_a = smem_u32(&sm.nlse[64 * wg]), nds_a = smem_u32(&sm.nds[64 * wg]);
-      uint32_t pk[32];                               // P of this key against 64 query rows, packed bf16
-      ok = __all_sync(0xffffffffu, bwd_wait(&sm.s_full, m & 1, abort));
-      if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.stat_full, m & 1, abort));
+      const uint32_t nlse_a = smem_u32(&sm.nlse[r_first]), nds_a = smem_u32(&sm.nds[r_first]);
+      const uint32_t s_addr = lane_base + hf * kRegion + kColS + 32 * wg;
+      const uint32_t dp_addr = lane_base + hf * kRegion + kColDP + 32 * wg;
+      uint32_t pk[16];                               // P of this key against 32 query rows, packed bf16
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full[hf], m & 1, abort));
+      if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.stat_full[hf], m & 1, abort));
       if (!ok) break;
       tc_fence_after_sync();
       HGA_TRACE_POINT(11);
       if (none) {
-        // no key of this warp is visible to any row of the half tile: zeros, no exponentials
+        // no key of this warp is visible to any of the 32 rows: zeros, no exponentials
 #pragma unroll
-        for (int i = 0; i < 32; ++i) pk[i] = 0u;
-      }
+        for (int i = 0; i < 16; ++i) pk[i] = 0u;
+      } else {
+        uint32_t x[32];
+        tmem_ld32(s_addr, x);
+        tmem_wait_ld();
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        if (!none) {
-          uint32_t x[32];
-          tmem_ld32(s_addr + 32 * c, x);
-          tmem_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 16; i += 2) {
-            uint32_t n0, n1, n2, n3;                 // -LSE*log2e of four consecutive columns
-            ld_shared_v4(nlse_a + (32 * c + 2 * i) * 4, n0, n1, n2, n3);
-            float a0, a1, a2, a3;
-            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1])), sl2_2,
-                                   pack_f32x2(__uint_as_float(n0), __uint_as_float(n1))), a0, a1);
-            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i + 2]), __uint_as_float(x[2 * i + 3])), sl2_2,
-                                   pack_f32x2(__uint_as_float(n2), __uint_as_float(n3))), a2, a3);
-            float p0 = fast_exp2(a0), p1 = fast_exp2(a1), p2 = fast_exp2(a2), p3 = fast_exp2(a3);
-            if (masked) {
-              const int col = 32 * c + 2 * i;
-              if (col < imin) p0 = 0.f;
-              if (col + 1 < imin) p1 = 0.f;
-              if (col + 2 < imin) p2 = 0.f;
-              if (col + 3 < imin) p3 = 0.f;
-            }
-            pk[16 * c + i] = pack_bf16(p0, p1);
-            pk[16 * c + i + 1] = pack_bf16(p2, p3);
+        for (int i = 0; i < 16; i += 2) {
+          uint32_t n0, n1, n2, n3;                   // -LSE*log2e of four consecutive columns
+          ld_shared_v4(nlse_a + (2 * i) * 4, n0, n1, n2, n3);
+          float a0, a1, a2, a3;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1])), sl2_2,
+                                 pack_f32x2(__uint_as_float(n0), __uint_as_float(n1))), a0, a1);
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i + 2]), __uint_as_float(x[2 * i + 3])), sl2_2,
+                                 pack_f32x2(__uint_as_float(n2), __uint_as_float(n3))), a2, a3);
+          float p0 = fast_exp2(a0), p1 = fast_exp2(a1), p2 = fast_exp2(a2), p3 = fast_exp2(a3);
+          if (masked) {
+            const int col = 2 * i;
+            if (col < imin) p0 = 0.f;
+            if (col + 1 < imin) p1 = 0.f;
+            if (col + 2 < imin) p2 = 0.f;
+            if (col + 3 < imin) p3 = 0.f;
           }
+          pk[i] = pack_bf16(p0, p1);
+          pk[i + 1] = pack_bf16(p2, p3);
         }
-        // P^T (bf16) over the S^T columns just read: 16 columns per 32 query rows
-        uint32_t out[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) out[i] = pk[16 * c + i];
-        tmem_st16(s_addr + 16 * c, out);
       }
-      ok = __all_sync(0xffffffffu, bwd_wait(&sm.dp_full, m & 1, abort));
-      if (!ok) break;
-      tc_fence_after_sync();
+      tmem_st16(s_addr, pk);                         // P^T (bf16) over the first 16 of the S^T columns just read
       HGA_TRACE_POINT(13);
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      {
         uint32_t out[16];
         if (!none) {
           uint32_t x[32];
-          tmem_ld32(dp_addr + 32 * c, x);
+          tmem_ld32(dp_addr, x);
           tmem_wait_ld();
 #pragma unroll
           for (int i = 0; i < 16; i += 2) {
             uint32_t n0, n1, n2, n3;                 // -delta*scale of four consecutive columns
-            ld_shared_v4(nds_a + (32 * c + 2 * i) * 4, n0, n1, n2, n3);
-            const uint32_t pa = pk[16 * c + i], pb = pk[16 * c + i + 1];
+            ld_shared_v4(nds_a + (2 * i) * 4, n0, n1, n2, n3);
+            const uint32_t pa = pk[i], pb = pk[i + 1];
             const uint64_t g0 = fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1])), scale_2,
                                           pack_f32x2(__uint_as_float(n0), __uint_as_float(n1)));
             const uint64_t g1 = fma_f32x2(pack_f32x2(__uint_as_float(x[2 * i + 2]), __uint_as_float(x[2 * i + 3])), scale_2,
@@ -323,11 +360,11 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
 #pragma unroll
           for (int i = 0; i < 16; ++i) out[i] = 0u;
         }
-        tmem_st16(dp_addr + 16 * c, out);            // dS^T (bf16) over the dP^T columns just read
+        tmem_st16(dp_addr, out);                     // dS^T (bf16) over the first 16 of the dP^T columns just read
       }
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(&sm.pds_full);
+      mbar_arrive(&sm.pds_full[hf]);
       HGA_TRACE_POINT(14);
     }
     if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.acc_done, 0, abort));
@@ -371,13 +408,16 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
     };
     float lse_next = lse_of(0);
     bool ok = true;
+    int o_issued = 1;                                // O tiles whose copies have been issued
     for (int m = 0; m < n_steps; ++m) {
       const int st = m & 1;
       const float lse = lse_next;
       if (m + 1 < n_steps) lse_next = lse_of(m + 1);
-      ok = __all_sync(0xffffffffu, bwd_wait(&sm.qdo_full[st], (m >> 1) & 1, abort));
+      ok = __all_sync(0xffffffffu, bwd_wait(&sm.qdo_full[st][j >> 6], (m >> 1) & 1, abort));   // (this row's half of dO)
+      HGA_TRACE_POINT(11);
       if (ok) ok = __all_sync(0xffffffffu, bwd_wait(&sm.o_full, m & 1, abort));
       if (!ok) break;
+      HGA_TRACE_POINT(13);
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
       const uint32_t do_line = smem_u32(sm.dO[st]) + (uint32_t)j * 128, o_line = smem_u32(sm.o) + (uint32_t)j * 128;
 #pragma unroll
@@ -393,14 +433,34 @@ k_attn_bwd_band_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_co
         }
       }
       mbar_arrive(&sm.o_empty);                      // the O tile may be overwritten by the next step's
+      if (warp == 13 && m + 1 < n_steps) {
+        // ... which this warp -- the one whose rows of dO arrive last -- fetches as soon as all four
+        // statistics warps have read this one
+        if (lane == 0) ok = bwd_wait(&sm.o_empty, m & 1, abort);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        if (lane == 0) mbar_arrive_expect_tx(&sm.o_full, kTile);
+        __syncwarp();
+        if (lane < 4) {
+          const int half = lane & 1, panel = lane >> 1;
+          int row, head;
+          qdo_coords(m + 1, half, row, head);
+          tma_load_5d(sm.o + (uint32_t)panel * 16384 + (uint32_t)half * 8192, &map_o, &sm.o_full, 0, row, panel, head, b);
+        }
+        o_issued = m + 2;
+      }
       const float delta = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-      // the key threads read the previous step's statistics until they hand its P^T and dS^T over
-      if (m > 0) ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_full, (m - 1) & 1, abort));
+      HGA_TRACE_POINT(15);
+      // the key threads read the previous step's statistics of this half until they hand its P^T and dS^T over
+      if (m > 0) ok = __all_sync(0xffffffffu, bwd_wait(&sm.pds_full[j >> 6], (m - 1) & 1, abort));
       if (!ok) break;
       sm.nlse[j] = -lse * 1.4426950408889634f;
       sm.nds[j] = -delta * dm.scale;
-      mbar_arrive(&sm.stat_full);
+      mbar_arrive(&sm.stat_full[j >> 6]);
+      HGA_TRACE_POINT(14);
     }
+    // giving up: let the O copy still in flight land before shared memory is released
+    if (*abort && warp == 13 && lane == 0) mbar_wait(&sm.o_full, (o_issued - 1) & 1);
   }
   HGA_TRACE_POINT(30);
 
