@@ -68,7 +68,7 @@ struct BwdSmem {
   alignas(1024) uint8_t v[kBwdVStages][kKvTile];
   alignas(1024) uint8_t p[kPdsTile];            // [16 row octets][8 rows][128 B], 128-byte swizzle
   alignas(1024) uint8_t ds[kPdsTile];           // (P and dS pass through shared memory only for dK/dV tiles)
-  uint64_t q_full, k_full[kBwdKStages], k_empty[kBwdKStages], v_full[kBwdVStages], v_empty[kBwdVStages];
+  uint64_t q_full, k_full[kBwdKStages], k_empty[kBwdKStages];   // (dK/dV steps: even stages hold K tiles, odd ones V tiles)
   uint64_t sdp_full, pds_full, dkv_full, dkv_free;      // dK/dV steps
   uint64_t s_full[2], dp_full[4], ds_full[2], s_read[2];   // paired steps (S(u+1) is committed before step u is over: two barriers;
                                                         // dP: four, so that a copy item taken ahead of time cannot mistake an older phase)
@@ -105,7 +105,10 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   HGA_TRACE_DECL;
   const int n_mt_item = dm.rows / 128;
-  const int item = blockIdx.x / n_mt_item;
+  // Launch order: late query blocks first.  They have the most routed keys inside the active segment (the
+  // expensive dK/dV steps), early ones none, so the cheapest CTAs are the ones that fill the last wave.
+  const int unit = blockIdx.x / n_mt_item, n_bh = dm.B * dm.Hkv;
+  const int item = (unit % n_bh) * dm.NQB + (dm.NQB - 1 - unit / n_bh);
   const int mt = blockIdx.x % n_mt_item;
   int b, h, qb;
   item_coords(dm, item, b, h, qb);
@@ -113,9 +116,8 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < kBwdKStages; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
-    for (int s = 0; s < kBwdVStages; ++s) { mbar_init(&sm.v_full[s], 2); mbar_init(&sm.v_empty[s], 1); }   // two V producers
-    mbar_init(&sm.sdp_full, 1); mbar_init(&sm.pds_full, 128);
+    for (int s = 0; s < kBwdKStages; ++s) { mbar_init(&sm.k_full[s], (s & 1) ? 2 : 1); mbar_init(&sm.k_empty[s], 1); }   // (two V producers)
+    mbar_init(&sm.sdp_full, 1); mbar_init(&sm.pds_full, 256);
     mbar_init(&sm.dkv_full, 1); mbar_init(&sm.dkv_free, 128);
     mbar_init(&sm.s_full[0], 1); mbar_init(&sm.s_full[1], 1);
     // (two barriers each, used alternately: S(u+1) and dP(u+1) are issued before the MMA warp waits for the row
@@ -206,10 +208,10 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const int n_act = sm.n_dkv;                       // steps 0 .. n_act-1 are dK/dV steps
   const int dkv_hi = sm.dkv_lo + n_act;
   const int n_pairs = (n_tiles - n_act + 1) / 2;    // paired steps; the last may hold one tile only
-  // Ring slots: dK/dV step s uses slot s; the paired steps start on an even slot (a pair of stages is
-  // one contiguous operand), so after an odd number of dK/dV steps one slot passes unused: the
-  // producers complete its full barriers without a copy, the MMA thread releases it at once.
-  const int n_act_even = n_pairs > 0 ? (n_act + 1) & ~1 : n_act;
+  // Ring slots: dK/dV step s takes TWO slots of the K ring, 2s for its K tile and 2s+1 for its V tile, so that
+  // the V ring proper stays free and the first V pair of the paired steps is copied while the dK/dV steps
+  // still run; the paired steps continue the slot numbering (a pair of stages is one contiguous operand).
+  const int n_act_even = 2 * n_act;
   const int red_hi = w.ls;
   // Step order: the dK/dV tiles first (descending), so their atomics drain while the rest is
   // computed; then every other tile, descending.
@@ -223,14 +225,12 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (warp == 0 || warp >= 14) {
     // ------------------------------------------------------------------ producers
-    // K and V advance independently (their rings differ in depth, and a V tile is released long
-    // before the K tile of the same step): warp 0 copies the K tiles (eight octet boxes, one per
-    // lane) and runs several steps ahead; warps 14 and 15 copy the V tiles (four boxes each), whose
-    // short ring is refilled only after the dP GEMM of the previous pair, so their issue time is on
-    // the critical path.  Issuing a box costs the issuing warp on the order of a hundred cycles;
+    // K and V advance independently (a V tile is released long before the K tile of the same step):
+    // warp 0 copies the K tiles (eight octet boxes, one per lane) and runs several steps ahead; warps 14
+    // and 15 copy the V tiles (four boxes each); in the paired steps their short ring is refilled only
+    // after the dP GEMM of the pair before the previous one, so their issue time is on the critical path.  Issuing a box costs the issuing warp on the order of a hundred cycles;
     // different warps issue in parallel.
     const bool is_v = warp != 0;
-    const int n_stages = is_v ? kBwdVStages : kBwdKStages;
     const CUtensorMap* map = is_v ? &map_v : &map_k;
     bool ok = true;
     // ---- slots of the dK/dV steps: one tile per slot, one full/empty barrier pair per stage
@@ -238,23 +238,18 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const int oct_in_tile = is_v ? (warp == 14 ? lane : 4 + lane) : lane;
       const bool copy_lane = is_v ? lane < 4 : lane < 8;
       const uint32_t my_bytes = (uint32_t)(is_v ? 4 : 8) * kOct;
-      for (int slot = 0; slot < n_act_even && ok; ++slot) {
-        const int st = slot % n_stages;
-        uint64_t* full = is_v ? &sm.v_full[st] : &sm.k_full[st];
-        uint64_t* empty = is_v ? &sm.v_empty[st] : &sm.k_empty[st];
-        uint8_t* dst = is_v ? sm.v[st] : sm.k[st];
-        const bool skipped = slot >= n_act;
+      for (int step = 0; step < n_act && ok; ++step) {
+        const int slot = 2 * step + (is_v ? 1 : 0);
+        const int st = slot % kBwdKStages;
         int row = dm.L;                                      // past the list: zeros
-        if (!skipped) {
-          const int o = 8 * tile_of_step(slot) + oct_in_tile;
-          if (o < n_oct) row = sm.oct_row[o];
-        }
-        if (lane == 0 && slot >= n_stages) ok = bwd_wait(empty, (uint32_t)(slot / n_stages - 1) & 1, abort);
+        const int o = 8 * tile_of_step(step) + oct_in_tile;
+        if (o < n_oct) row = sm.oct_row[o];
+        if (lane == 0 && slot >= kBwdKStages) ok = bwd_wait(&sm.k_empty[st], (uint32_t)(slot / kBwdKStages - 1) & 1, abort);
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
-        if (lane == 0) { if (skipped) mbar_arrive(full); else mbar_arrive_expect_tx(full, my_bytes); }
+        if (lane == 0) mbar_arrive_expect_tx(&sm.k_full[st], my_bytes);
         __syncwarp();
-        if (copy_lane && !skipped) tma_load_5d(dst + oct_in_tile * kOct, map, full, 0, row, 0, h, b);
+        if (copy_lane) tma_load_5d(sm.k[st] + oct_in_tile * kOct, map, &sm.k_full[st], 0, row, 0, h, b);
         HGA_TRACE_POINT(2);
       }
     }
@@ -280,8 +275,9 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         if (lane == 0) {
           if (is_v) {
-            // first use: the dK/dV steps (which read V stages, P and dS) must be over; later: dP of pair p-2 is done
-            if (p < 2) { if (n_act > 0) ok = bwd_wait(&sm.phase_a_done, 0, abort); }
+            // first pair: the V ring is free from the start; second: the dK/dV steps (which use the P and dS
+            // tiles) must be over; later: dP of pair p-2 is done
+            if (p < 2) { if (p == 1 && n_act > 0) ok = bwd_wait(&sm.phase_a_done, 0, abort); }
             else ok = bwd_wait(&sm.dp_full[(p - 2) & 3], (uint32_t)((p - 2) >> 2) & 1, abort);
           } else if (p < n_ps) {
             // first paired use of these stages: if a dK/dV step used them, those steps must be over
@@ -331,7 +327,6 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const uint64_t pd = smem_desc_sw128(smem_u32(sm.p), 16, 1024);         // P : MN-major B (dV^T)
       // (arguments are ring slots)
       auto wait_k = [&](int s) { return mma_wait(&sm.k_full[s % kBwdKStages], (s / kBwdKStages) & 1, abort); };
-      auto wait_v = [&](int s) { return mma_wait(&sm.v_full[s % kBwdVStages], (s / kBwdVStages) & 1, abort); };
       // acc (128 rows x N keys) = a (Q or dO, K-major) x b^T (key tiles at ring stage st, K-major)
       auto issue_qk = [&](uint32_t acc, uint64_t a, uint64_t b0, int st, uint32_t idesc) {   // st: ring stage
         const uint64_t bd = desc_advance(b0, (uint32_t)st * kKvTile);
@@ -342,22 +337,28 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       };
       bool ok = mma_wait(&sm.q_full, 0, abort);
+      HGA_TRACE_POINT(40);
       bool dq_started = false;
       // ---- dK/dV steps: one at a time, every operand from shared memory.  The tensor pipe runs in
       // issue order and a commit covers everything issued before it, so sdp_full of step s+1 also
       // tells the row threads that the GEMMs reading P/dS of step s are done.
       for (int s = 0; s < n_act && ok; ++s) {
-        const int st = s % kBwdKStages, vst = s % kBwdVStages;
-        ok = wait_k(s) && wait_v(s);
+        const int st = (2 * s) % kBwdKStages, vst = (2 * s + 1) % kBwdKStages;      // K tile, V tile
+        ok = wait_k(2 * s);
+        HGA_TRACE_POINT(41);
+        ok = ok && wait_k(2 * s + 1);
+        HGA_TRACE_POINT(42);
         if (!ok) break;
         tc_fence_after_sync();
         issue_qk(tmem + region(0), q_k, k_k0, st, idesc_sdp);
-        issue_qk(tmem + region(0) + 64, do_k, v_k0, vst, idesc_sdp);
+        issue_qk(tmem + region(0) + 64, do_k, k_k0, vst, idesc_sdp);
         mma_commit_w(&sm.sdp_full);
-        mma_commit_w(&sm.v_empty[vst]);
+        mma_commit_w(&sm.k_empty[vst]);
+        HGA_TRACE_POINT(44);
         ok = mma_wait(&sm.pds_full, s & 1, abort);
         if (!ok) break;
         tc_fence_after_sync();
+        HGA_TRACE_POINT(45);
         const uint64_t kmn = desc_advance(k_mn0, (uint32_t)st * kKvTile);
 #pragma unroll
         for (int kk = 0; kk < kKT / 16; ++kk)   // dQ += dS K : 16 keys per MMA
@@ -382,17 +383,10 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // ---- paired steps.  Step u covers ring stages st, st+1 (contiguous); S(u) lives in region
       // (2u)%3, dP(u) and later dS(u) in region (2u+1)%3.
       if (ok && n_pairs > 0) {
-        if (n_act_even > n_act) {
-          // the unused slot: observe its (copy-less) full barriers and release it
-          ok = wait_k(n_act) && wait_v(n_act);
-          if (ok) {
-            mma_commit_w(&sm.k_empty[n_act % kBwdKStages]);
-            mma_commit_w(&sm.v_empty[n_act % kBwdVStages]);
-          }
-        }
         if (ok && n_act_even > 0) mma_commit_w(&sm.phase_a_done);
         const int ps0 = (n_act_even / 2) % (kBwdKStages / 2);
         if (ok) ok = mma_wait(&sm.kp_full[ps0], 0, abort);
+        HGA_TRACE_POINT(43);
         if (ok) {
           tc_fence_after_sync();
           issue_qk(tmem + region(0), q_k, k_k0, 2 * ps0, idesc_sdp2);
@@ -492,14 +486,14 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     uint32_t d_lo, d_hi;
     tmem_ld2(lane_base + kColDQ, d_lo, d_hi);
     tmem_wait_ld();
-    // (the first dQ GEMM of a dK/dV step follows the arrivals of warpgroup 0 alone: it must not overwrite
-    // these two columns before warpgroup 1 has read them)
+    // (the first dQ GEMM must not overwrite these two columns before every row thread has read them)
     tc_fence_before_sync();
     asm volatile("bar.sync 3, 256;" ::: "memory");
     const float neg_delta_s = -(__uint_as_float(d_lo) + __uint_as_float(d_hi)) * dm.scale;
     HGA_TRACE_POINT(10);
-    if (wg == 0) {
-      // ---- dK/dV steps (warpgroup 0): P and dS go to shared memory as operands of dV^T / dK^T / dQ
+    {
+      // ---- dK/dV steps: P and dS go to shared memory as operands of dV^T / dK^T / dQ; warpgroup wg takes
+      // keys 32*wg .. 32*wg+31 of the tile.
       // this row's 128-byte line inside the P / dS buffers, and its swizzle key
       const uint32_t line = (uint32_t)(row_in_tile >> 3) * 1024 + (uint32_t)(row_in_tile & 7) * 128;
       const uint32_t key = (uint32_t)(row_in_tile & 7);
@@ -509,9 +503,10 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ok = __all_sync(0xffffffffu, bwd_wait(&sm.sdp_full, s & 1, abort));
         if (!ok) break;
         tc_fence_after_sync();
+        HGA_TRACE_POINT(12);
         const int vis = limit - kKT * tile_of_step(s);
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {             // 16 columns (keys) at a time
+        for (int q4 = 2 * wg; q4 < 2 * wg + 2; ++q4) {   // 16 columns (keys) at a time
           uint32_t sv[16], dp[16];
           tmem_ld16(sdp_addr + q4 * 16, sv);
           tmem_ld16(sdp_addr + 64 + q4 * 16, dp);
@@ -540,6 +535,7 @@ k_attn_bwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tc_fence_before_sync();
         fence_proxy_async_smem();
         mbar_arrive(&sm.pds_full);
+        HGA_TRACE_POINT(17);
       }
     }
     // ---- paired steps: warpgroup wg owns the wg-th tile of each pair (64 of the 128 columns)

@@ -85,7 +85,10 @@ k_attn_fwd_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   // in their own TMEM lanes and are never stored)
   const int bq_pad = bq_padded(dm), rows_pad = rows_padded(dm);
   const int n_mt_item = (rows_pad + 127) / 128;
-  const int item = blockIdx.x / n_mt_item;
+  // Launch order: late query blocks first -- where the history is short they see the most keys, so the
+  // cheapest CTAs are the ones that fill the last wave.
+  const int unit = blockIdx.x / n_mt_item, n_bh = dm.B * dm.Hkv;
+  const int item = (unit % n_bh) * dm.NQB + (dm.NQB - 1 - unit / n_bh);
   const int mt0 = blockIdx.x % n_mt_item;               // this CTA's M-tile inside the item
   int b, h, qb;
   item_coords(dm, item, b, h, qb);
