@@ -55,7 +55,7 @@ __device__ __forceinline__ uint32_t rt_orderable(float f) {
 
 template <int D, int STAGES, int ACCS>
 __global__ void __launch_bounds__(kRtThreads, 2)
-k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_cs,
+k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_ct,
               const __grid_constant__ CUtensorMap map_gs, Dims dm, int32_t* __restrict__ chunk_idx,
               int32_t* __restrict__ group_idx, int32_t* __restrict__ n_groups,
               float* __restrict__ chunk_scores, float* __restrict__ group_scores, int q_bytes,
@@ -93,22 +93,26 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   uint32_t col_mask = 0;                                       // bit i: column i of a block of 32 is a real query row
   for (int i = 0; i < 32; ++i) col_mask |= (uint32_t)((i % bq_pad) < dm.Bq) << i;
 
-  // Copies one 128-row summary tile (16 octet boxes, one per lane) into its ring stage; all lanes of warp 0.
+  // Copies one 128-row summary tile into its ring stage; all lanes of warp 0.  The candidate chunks are
+  // consecutive rows of the summary table, so a tile of them is 64-row x one-panel boxes (8 KB each: two or four
+  // per tile, laid out [panel][128 rows][128 B]); the opened chunks' group summaries are gathered octet by octet
+  // (16 boxes, [octet][panel][8 rows][128 B]).  A box costs the issuing warp on the order of a hundred cycles.
   int tiles_issued = 0;                 // warp 0's count of summary tiles whose copies were started
   auto issue_tile = [&](int tg, int t, bool phase2) {
     const int s = tg % STAGES;
     tiles_issued = tg + 1;
     if (lane == 0) mbar_arrive_expect_tx(&sm.a_full[s], Smem::kTile);
     __syncwarp();
-    if (lane < 16) {
-      if (!phase2) {
-        const int row = j0 + 128 * t + 8 * lane;              // rows past the table read as zeros
-        tma_load_5d(sm.a[s] + lane * kOctBytes, &map_cs, &sm.a_full[s], 0, row, 0, h, b);
-      } else {
-        const int oc = 16 * t + lane, r = oc / opc;
-        const int row = r < k_sel ? sm.sorted[r] * dm.per + 8 * (oc % opc) : dm.Ng;
-        tma_load_5d(sm.a[s] + lane * kOctBytes, &map_gs, &sm.a_full[s], 0, row, 0, h, b);
+    if (!phase2) {
+      if (lane < 2 * (D / 64)) {
+        const int half = lane & 1, panel = lane >> 1;
+        const int row = j0 + 128 * t + 64 * half;             // rows past the table read as zeros
+        tma_load_5d(sm.a[s] + panel * 16384 + half * 8192, &map_ct, &sm.a_full[s], 0, row, panel, h, b);
       }
+    } else if (lane < 16) {
+      const int oc = 16 * t + lane, r = oc / opc;
+      const int row = r < k_sel ? sm.sorted[r] * dm.per + 8 * (oc % opc) : dm.Ng;
+      tma_load_5d(sm.a[s] + lane * kOctBytes, &map_gs, &sm.a_full[s], 0, row, 0, h, b);
     }
   };
   const int n_pre = k_sel > 0 ? (n_ct < STAGES ? n_ct : STAGES) : 0;   // chunk tiles copied ahead of the CTA barrier
@@ -122,7 +126,7 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       sm.abort = 0;
       sm.n_sel = 0;
       fence_barrier_init();
-      prefetch_tensormap(&map_q); prefetch_tensormap(&map_cs); prefetch_tensormap(&map_gs);
+      prefetch_tensormap(&map_q); prefetch_tensormap(&map_ct); prefetch_tensormap(&map_gs);
     }
     __syncwarp();
     // the first chunk tiles depend on nothing: their copies start before the CTA meets
@@ -191,13 +195,16 @@ k_route_sm100(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             if (use > 0) ok = mma_wait(&sm.acc_free[buf], (use - 1) & 1, abort);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint64_t ad = smem_desc_sw128(smem_u32(sm.a[s]), 16, kOctBytes);
+            // A: the summary tile -- 8-row groups 1024 B apart and panels 16 KB apart for the chunk tiles,
+            // octets (8 rows x all panels) for the gathered group tiles; B: the query rows, octets
+            const uint64_t ad = smem_desc_sw128(smem_u32(sm.a[s]), 16, phase2 ? kOctBytes : 1024);
+            const uint32_t a_panel = phase2 ? 1024u : 16384u;
             const uint64_t bd = smem_desc_sw128(
                 smem_u32(q_smem) + (uint32_t)hf * (uint32_t)(rows_half / 8) * kOctBytes, 16, kOctBytes);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
-              const uint32_t off = (kk >> 2) * 1024 + (kk & 3) * 32;
-              mma_ss_w(tmem + buf * kAccCols, desc_advance(ad, off), desc_advance(bd, off), idesc, kk > 0);
+              const uint32_t a_off = (kk >> 2) * a_panel + (kk & 3) * 32, b_off = (kk >> 2) * 1024 + (kk & 3) * 32;
+              mma_ss_w(tmem + buf * kAccCols, desc_advance(ad, a_off), desc_advance(bd, b_off), idesc, kk > 0);
             }
             mma_commit_w(&sm.acc_full[buf]);
           }
@@ -491,6 +498,7 @@ static int launch_route(const Dims& dm, const void* Q, const void* chunk_sum, co
                         float* group_scores, cudaStream_t st) {
   CUtensorMap mq, mc, mg;
   const uint32_t box[5] = {64, 8, (uint32_t)(D / 64), 1, 1};
+  const uint32_t box_ct[5] = {64, 64, 1, 1, 1};            // half a chunk tile, one panel
   const uint64_t dq[5] = {64, (uint64_t)dm.S, (uint64_t)(D / 64), (uint64_t)dm.Hq, (uint64_t)dm.B};
   const uint64_t dc[5] = {64, (uint64_t)dm.Nc, (uint64_t)(D / 64), (uint64_t)dm.Hkv, (uint64_t)dm.B};
   const uint64_t dg[5] = {64, (uint64_t)dm.Ng, (uint64_t)(D / 64), (uint64_t)dm.Hkv, (uint64_t)dm.B};
@@ -498,7 +506,7 @@ static int launch_route(const Dims& dm, const void* Q, const void* chunk_sum, co
   const uint64_t sc[4] = {(uint64_t)D * 2, 128, (uint64_t)dm.NcS * D * 2, (uint64_t)dm.Hkv * dm.NcS * D * 2};
   const uint64_t sg[4] = {(uint64_t)D * 2, 128, (uint64_t)dm.NgS * D * 2, (uint64_t)dm.Hkv * dm.NgS * D * 2};
   if (encode_tensor_map_bf16(&mq, Q, 5, dq, sq, box, true) ||
-      encode_tensor_map_bf16(&mc, chunk_sum, 5, dc, sc, box, true) ||
+      encode_tensor_map_bf16(&mc, chunk_sum, 5, dc, sc, box_ct, true) ||
       encode_tensor_map_bf16(&mg, group_sum, 5, dg, sg, box, true))
     return HGA_ERR_UNSUPPORTED;
   const int max_cand = route_max_cand(dm);
