@@ -27,8 +27,10 @@ def sample_items(cfg, full_head, extra, seed):
 
 # routed keys per item (a data-independent count) for the last query block of each config
 ROUTED_KEYS_LAST_BLOCK = {1: 320, 2: 512, 3: 768, 4: 768, 5: 2560, 6: 768}
-# per configuration: (items that may carry an excused chunk, chunks that may carry an excused group)
-EXCUSED_BOUNDS = {1: (1, 1), 2: (2, 2), 3: (2, 2), 4: (2, 2), 5: (8, 8), 6: (2, 2)}
+# per configuration: (items that may carry an excused chunk, chunks that may carry an excused group).  Observed
+# on the sampled items: none on any configuration (the counts are printed); one is allowed for a change of
+# accumulation order, two on the i.i.d. configuration 5, where near ties are the most likely.
+EXCUSED_BOUNDS = {1: (1, 1), 2: (1, 1), 3: (1, 1), 4: (1, 1), 5: (2, 2), 6: (1, 1)}
 
 
 @pytest.mark.parametrize("n,full_head,extra", [(1, (0, 0), 4), (2, (0, 5), 12), (3, (0, 3), 12),
