@@ -9,7 +9,12 @@
 //
 // Tags (see the kernels): 1 set-up done; 2 a producer issued a tile; 3 first GEMMs issued; 5/6/7/8 the
 // issuing warp (barrier observed / S issued / dQ or PV issued / dP issued); 11/13/14/15 a row or key
-// thread (S observed / second operand observed / results handed over); 20/21 epilogue; 30 role finished.
+// thread (S observed / second operand observed / results handed over); 20/21 epilogue; 30 role finished, 31
+// past the final block barrier.  Sweep only: 4 a dK/dV step issued; 10 delta known; 12/17 a row thread in a
+// dK/dV step (S, dP observed / P, dS written); 16/18 a reduction warp (accumulators observed / atomics issued);
+// 40-45 the issuing warp before the pairs (Q and dO / K tile / V tile / first K pair arrived, S and dP of a dK/dV
+// step issued, its P and dS observed).  Band only: 11/13/15/14 in the statistics warps = dO rows arrived / O tile
+// arrived / delta computed / statistics published.
 // Built with -DHGA_TRACE; includes the kernels' translation units directly, so it needs no library.
 #include <algorithm>
 #include <array>
